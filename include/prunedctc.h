@@ -1,0 +1,153 @@
+/*
+ * prunedctc.h -- C ABI of the Pruned-CTC head-and-loss library for NVIDIA B200 (sm_100a).
+ *
+ * One call evaluates Algorithm 1 of the paper ("Pruned CTC"): the CTC loss of a
+ * batch under a full-vocabulary softmax head, and the gradients of the sum of
+ * the utterance losses with respect to the head input and the head, without
+ * ever holding a frames-by-vocabulary array.
+ *
+ * All device work is enqueued on the caller's stream.  Every buffer is owned by
+ * the caller; the library keeps no pointers and no state between calls and,
+ * except where an entry point says otherwise, allocates nothing.
+ * Functions return a status code and never throw or abort.
+ */
+#ifndef PRUNEDCTC_H_
+#define PRUNEDCTC_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum {
+  PCTC_OK = 0,
+  PCTC_ERR_INVALID_ARG = 1,         /* null pointer, non-positive size, length out of range      */
+  PCTC_ERR_WORKSPACE_TOO_SMALL = 2, /* workspace_bytes below pctc_workspace_bytes()              */
+  PCTC_ERR_UNSUPPORTED = 3,         /* dtype/shape the kernels do not cover (see each function)  */
+  PCTC_ERR_CUDA = 4,                /* a CUDA runtime or driver call failed (launch errors)      */
+  PCTC_ERR_BAD_TARGET = 5,          /* reserved: bad targets are reported per utterance instead  */
+  PCTC_ERR_TIMEOUT = 6              /* a bounded device-side wait gave up (see pctc_last_device_status) */
+} pctc_status_t;
+
+typedef enum { PCTC_BF16 = 0, PCTC_FP32 = 1 } pctc_dtype_t;
+
+/* Which contraction kernels run.  AUTO: tcgen05 tensor-core kernels for bf16,
+ * fp32 FMA kernels for fp32.  SIMT: the FMA kernels for either dtype (bf16
+ * operands are widened to fp32; used to cross-check the tensor-core path). */
+typedef enum { PCTC_GEMM_AUTO = 0, PCTC_GEMM_SIMT = 1 } pctc_gemm_path_t;
+
+/* Per-utterance flags written to `utt_flags` (Appendix B.1, "Loss aggregation"). */
+#define PCTC_UTT_INFEASIBLE 1 /* T_n < |y_n| + (adjacent equal pairs): no alignment exists  */
+#define PCTC_UTT_NONFINITE 2  /* loss not finite (NaN/Inf input, or empty retained lattice)  */
+#define PCTC_UTT_BAD_TARGET 4 /* a token equals blank_id or lies outside [0, V)              */
+
+/*
+ * The problem of Section 3.1 / Algorithm 1, line 1.
+ *   hidden  [N, T, D]  padded head-input states; utterance n has T_n valid frames
+ *   W       [V, D]     head weight, bias [V] optional; logits Z = X W^T + 1 b^T
+ *   targets [N, target_stride] blank-free token ids, first U_n entries of row n count
+ */
+typedef struct {
+  int32_t N;             /* utterances                                                        */
+  int32_t T;             /* padded frames per utterance (row count of hidden[n])              */
+  int32_t D;             /* head input width; bf16 tensor-core path needs D % 8 == 0          */
+  int64_t V;             /* classes, blank included; bf16 tensor-core path needs V % 8 == 0   */
+  int32_t dtype;         /* pctc_dtype_t of hidden, W, bias, dH, dW, dbias; loss is fp32      */
+  int32_t blank_id;      /* in [0, V)                                                         */
+  float   beam;          /* alignment beam in nats (Section 3.3); <= 0 or +inf: no pruning    */
+  int32_t chunk;         /* vocabulary chunk width C (Algorithm 1); 0: library default        */
+  int32_t target_stride; /* row pitch of targets and relabeled_out                            */
+  int32_t gemm_path;     /* pctc_gemm_path_t                                                  */
+} pctc_problem_t;
+
+/*
+ * Workspace size for a problem (host-only; touches no device).
+ * input_lengths_host [N]: 1 <= T_n <= T.  target_lengths_host [N]: 0 <= U_n <= target_stride.
+ * The size depends on M = sum T_n, D, sum U_n and the chunk width, and on V only
+ * through O(V) index tables: there is no M*V term (Section 3.4, activation storage).
+ */
+pctc_status_t pctc_workspace_bytes(const pctc_problem_t* problem,
+                                   const int32_t* input_lengths_host,
+                                   const int32_t* target_lengths_host,
+                                   size_t* bytes_out);
+
+/*
+ * Algorithm 1, forward and backward in one call.
+ *
+ * Steps, all on `stream`:
+ *   line 2-3  U = blank followed by the ascending distinct target labels; K = |U|;
+ *             targets relabelled by their index in U               -> subset_out, K_out, relabeled_out
+ *   line 4    the M = sum T_n valid frames are stacked             (workspace)
+ *   line 5    lambda_m = log sum_v exp Z[m,v], online over vocabulary chunks (Eq. "lognorm")
+ *   line 6    S = X W_U^T + 1 b_U^T - lambda 1^T                   (workspace, fp32)
+ *   line 7-9  per utterance: loss = -log sum over (retained) alignments; loss of an
+ *             infeasible, bad-target or non-finite utterance is 0  -> loss, utt_flags
+ *   line 10   occupancies gamma (G = -gamma)                       (workspace, fp32)
+ *   line 11-17 per vocabulary chunk: recompute Z, dZ = w_m (exp(Z - lambda) - scatter_U(gamma))
+ *             (Eq. "vjp" with unit weights; w_m = 0 on frames of excluded utterances),
+ *             dH += dZ W_c, dW_c = dZ^T X, db_c = dZ^T 1           -> dH, dW, dbias
+ *
+ * Pointers (device unless marked HOST; all contiguous, row-major):
+ *   hidden [N,T,D], W [V,D], bias [V] or NULL, targets [N,target_stride] int32,
+ *   input_lengths HOST [N], target_lengths HOST [N],
+ *   loss [N] fp32 (per-utterance, not normalised),
+ *   dH [N,T,D] (padded frames are written as zero), dW [V,D] (overwritten),
+ *   dbias [V] or NULL (ignored when bias is NULL),
+ *   subset_out [1 + sum U_n] or NULL, K_out [1] or NULL,
+ *   relabeled_out [N,target_stride] or NULL (entries past U_n and bad tokens: -1),
+ *   utt_flags [N] or NULL,
+ *   workspace: >= pctc_workspace_bytes(), 256-byte aligned.
+ * hidden, W, dH, dW must be 16-byte aligned.
+ *
+ * Gradients are those of the plain sum of the utterance losses (no division by
+ * token or frame counts).  With a finite beam the retained lattice is treated
+ * as fixed (Section 3.3).
+ *
+ * Errors: host-detectable problems return before anything is launched and leave
+ * the outputs untouched.  Bad targets and non-finite losses never fault; they are
+ * reported in utt_flags.  The return value covers launch errors only: the call
+ * does not synchronise.
+ */
+pctc_status_t pruned_ctc_fwd_bwd(const pctc_problem_t* problem,
+                                 const void* hidden, const void* W, const void* bias,
+                                 const int32_t* targets,
+                                 const int32_t* input_lengths, const int32_t* target_lengths,
+                                 float* loss, void* dH, void* dW, void* dbias,
+                                 int32_t* subset_out, int32_t* K_out, int32_t* relabeled_out,
+                                 int32_t* utt_flags,
+                                 void* workspace, size_t workspace_bytes, void* stream);
+
+/*
+ * Contraction kernel on its own, for validation of the tensor-core path:
+ *   C[i,j] = sum_k A(i,k) B(j,k),  i < m, j < n, k < k,  C fp32 [m, n] row-major.
+ * a_mn_major == 0: A is stored [m, k] (k contiguous); else A is stored [k, m].
+ * b_mn_major == 0: B is stored [n, k] (k contiguous); else B is stored [k, n].
+ * Operands are bf16 device arrays, 16-byte aligned, with the contiguous extent a
+ * multiple of 8.  gemm_path as in pctc_problem_t.  Not part of Algorithm 1: it is
+ * the building block of lines 5, 6 and 13-16.
+ */
+pctc_status_t pctc_gemm_bf16(const void* A, const void* B, float* C,
+                             int32_t m, int32_t n, int32_t k,
+                             int32_t a_mn_major, int32_t b_mn_major,
+                             int32_t gemm_path,
+                             int32_t* device_status, /* device [1] or NULL; see below */
+                             void* stream);
+
+/*
+ * Device-side status word.  Every wait inside a kernel (on an mbarrier) is
+ * bounded; a wait that gives up stores a non-zero code and the kernel returns
+ * cleanly instead of hanging.  pruned_ctc_fwd_bwd keeps the word at the start of
+ * its workspace (zeroed by each call); this function copies it to the host after
+ * synchronising `stream`.  0 means no wait gave up.  PCTC_ERR_TIMEOUT is returned
+ * when it is non-zero.
+ */
+pctc_status_t pctc_workspace_status(const void* workspace, void* stream, int32_t* status_host);
+
+const char* pctc_status_string(pctc_status_t status);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* PRUNEDCTC_H_ */

@@ -1,0 +1,195 @@
+"""ctypes binding of libprunedctc: argument marshalling only.
+
+Every step of the computation runs in the library's CUDA kernels; torch is
+used for device memory and the current stream.  There is no CPU path: calls
+raise if the library is missing or returns an error status.
+"""
+
+from __future__ import annotations
+
+import ctypes
+import os
+from typing import Optional
+
+import numpy as np
+
+HERE = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(HERE, "libprunedctc.so")
+
+PCTC_BF16, PCTC_FP32 = 0, 1
+GEMM_AUTO, GEMM_SIMT = 0, 1
+UTT_INFEASIBLE, UTT_NONFINITE, UTT_BAD_TARGET = 1, 2, 4
+
+EXPORTS = ("pctc_workspace_bytes", "pruned_ctc_fwd_bwd", "pctc_gemm_bf16", "pctc_workspace_status",
+           "pctc_status_string")
+
+
+class Problem(ctypes.Structure):
+    _fields_ = [
+        ("N", ctypes.c_int32), ("T", ctypes.c_int32), ("D", ctypes.c_int32),
+        ("V", ctypes.c_int64),
+        ("dtype", ctypes.c_int32), ("blank_id", ctypes.c_int32),
+        ("beam", ctypes.c_float),
+        ("chunk", ctypes.c_int32), ("target_stride", ctypes.c_int32), ("gemm_path", ctypes.c_int32),
+    ]
+
+
+class PctcError(RuntimeError):
+    def __init__(self, status: int, what: str):
+        super().__init__(f"{what}: status {status} ({status_string(status)})")
+        self.status = status
+
+
+_lib = None
+
+
+def load() -> ctypes.CDLL:
+    """Load the shared library (no build here; see build.build())."""
+    global _lib
+    if _lib is not None:
+        return _lib
+    if not os.path.exists(LIB_PATH):
+        raise RuntimeError(f"{LIB_PATH} is missing: run paper_2609_33645_b200.build.build() first; "
+                           "there is no fallback implementation")
+    lib = ctypes.CDLL(LIB_PATH)
+    vp, i32p = ctypes.c_void_p, ctypes.POINTER(ctypes.c_int32)
+    lib.pctc_workspace_bytes.restype = ctypes.c_int
+    lib.pctc_workspace_bytes.argtypes = [ctypes.POINTER(Problem), i32p, i32p, ctypes.POINTER(ctypes.c_size_t)]
+    lib.pruned_ctc_fwd_bwd.restype = ctypes.c_int
+    lib.pruned_ctc_fwd_bwd.argtypes = [ctypes.POINTER(Problem), vp, vp, vp, vp, i32p, i32p,
+                                       vp, vp, vp, vp, vp, vp, vp, vp, vp, ctypes.c_size_t, vp]
+    lib.pctc_gemm_bf16.restype = ctypes.c_int
+    lib.pctc_gemm_bf16.argtypes = [vp, vp, vp, ctypes.c_int32, ctypes.c_int32, ctypes.c_int32,
+                                   ctypes.c_int32, ctypes.c_int32, ctypes.c_int32, vp, vp]
+    lib.pctc_workspace_status.restype = ctypes.c_int
+    lib.pctc_workspace_status.argtypes = [vp, vp, i32p]
+    lib.pctc_status_string.restype = ctypes.c_char_p
+    lib.pctc_status_string.argtypes = [ctypes.c_int]
+    _lib = lib
+    return lib
+
+
+def status_string(status: int) -> str:
+    return load().pctc_status_string(int(status)).decode()
+
+
+def _i32(a) -> np.ndarray:
+    return np.ascontiguousarray(np.asarray(a), dtype=np.int32)
+
+
+def _ptr_i32(a: np.ndarray):
+    return a.ctypes.data_as(ctypes.POINTER(ctypes.c_int32))
+
+
+def make_problem(N, T, D, V, dtype, blank_id, beam=0.0, chunk=0, target_stride=0, gemm_path=GEMM_AUTO) -> Problem:
+    return Problem(int(N), int(T), int(D), int(V), int(dtype), int(blank_id), float(beam), int(chunk),
+                   int(target_stride), int(gemm_path))
+
+
+def workspace_bytes(problem: Problem, input_lengths, target_lengths) -> int:
+    il, tl = _i32(input_lengths), _i32(target_lengths)
+    out = ctypes.c_size_t(0)
+    st = load().pctc_workspace_bytes(ctypes.byref(problem), _ptr_i32(il), _ptr_i32(tl), ctypes.byref(out))
+    if st != 0:
+        raise PctcError(st, "pctc_workspace_bytes")
+    return int(out.value)
+
+
+def _dptr(t) -> Optional[int]:
+    return None if t is None else ctypes.c_void_p(t.data_ptr())
+
+
+def pruned_ctc_fwd_bwd(hidden, W, bias, targets, input_lengths, target_lengths, blank_id, *, beam=0.0,
+                       chunk=0, gemm_path=GEMM_AUTO, workspace=None, out=None, check_status=False):
+    """Algorithm 1 on CUDA tensors.
+
+    hidden [N,T,D], W [V,D], bias [V] or None (bf16 or fp32, same dtype), targets
+    [N,stride] int32 on the device; input_lengths / target_lengths are host
+    integer sequences.  Returns a dict of device tensors: loss [N] fp32, dH, dW,
+    dbias (or None), subset [1+sum U], K [1], relabeled [N,stride], flags [N],
+    plus "workspace" (reusable) and "workspace_bytes".  `out` may carry
+    preallocated tensors from an earlier call with the same shapes.
+    """
+    import torch
+
+    lib = load()
+    if not (hidden.is_cuda and W.is_cuda and hidden.is_contiguous() and W.is_contiguous()):
+        raise ValueError("hidden and W must be contiguous CUDA tensors")
+    if hidden.dtype != W.dtype or hidden.dtype not in (torch.bfloat16, torch.float32):
+        raise ValueError("hidden and W must both be bf16 or both fp32")
+    dt = PCTC_BF16 if hidden.dtype == torch.bfloat16 else PCTC_FP32
+    N, T, D = hidden.shape
+    V = W.shape[0]
+    il, tl = _i32(input_lengths), _i32(target_lengths)
+    if targets is None:
+        targets = torch.zeros((N, 1), dtype=torch.int32, device=hidden.device)
+    if targets.dtype != torch.int32 or not targets.is_contiguous():
+        raise ValueError("targets must be a contiguous int32 CUDA tensor")
+    stride = targets.shape[1]
+    prob = make_problem(N, T, D, V, dt, blank_id, beam, chunk, stride, gemm_path)
+    need = workspace_bytes(prob, il, tl)
+    dev = hidden.device
+    if workspace is None or workspace.numel() < need:
+        workspace = torch.empty(need, dtype=torch.uint8, device=dev)
+    o = out or {}
+
+    def buf(name, shape, dtype):
+        t = o.get(name)
+        if t is None or tuple(t.shape) != tuple(shape) or t.dtype != dtype:
+            t = torch.empty(shape, dtype=dtype, device=dev)
+        return t
+
+    ksum = int(tl.sum()) + 1
+    res = dict(
+        loss=buf("loss", (N,), torch.float32),
+        dH=buf("dH", (N, T, D), hidden.dtype),
+        dW=buf("dW", (V, D), hidden.dtype),
+        dbias=buf("dbias", (V,), hidden.dtype) if bias is not None else None,
+        subset=buf("subset", (ksum,), torch.int32),
+        K=buf("K", (1,), torch.int32),
+        relabeled=buf("relabeled", (N, stride), torch.int32),
+        flags=buf("flags", (N,), torch.int32),
+        workspace=workspace, workspace_bytes=need,
+    )
+    stream = ctypes.c_void_p(torch.cuda.current_stream(dev).cuda_stream)
+    st = lib.pruned_ctc_fwd_bwd(
+        ctypes.byref(prob), _dptr(hidden), _dptr(W), _dptr(bias), _dptr(targets), _ptr_i32(il), _ptr_i32(tl),
+        _dptr(res["loss"]), _dptr(res["dH"]), _dptr(res["dW"]), _dptr(res["dbias"]),
+        _dptr(res["subset"]), _dptr(res["K"]), _dptr(res["relabeled"]), _dptr(res["flags"]),
+        _dptr(workspace), ctypes.c_size_t(workspace.numel()), stream)
+    if st != 0:
+        raise PctcError(st, "pruned_ctc_fwd_bwd")
+    if check_status:
+        code = workspace_status(workspace)
+        if code != 0:
+            raise PctcError(6, f"device status word {code}")
+    return res
+
+
+def workspace_status(workspace) -> int:
+    """Synchronise the current stream and return the device status word (0: no wait gave up)."""
+    import torch
+
+    host = ctypes.c_int32(0)
+    stream = ctypes.c_void_p(torch.cuda.current_stream(workspace.device).cuda_stream)
+    st = load().pctc_workspace_status(_dptr(workspace), stream, ctypes.byref(host))
+    if st not in (0, 6):
+        raise PctcError(st, "pctc_workspace_status")
+    return int(host.value)
+
+
+def gemm_bf16(A, B, m, n, k, a_mn_major=False, b_mn_major=False, gemm_path=GEMM_AUTO):
+    """C[m,n] (fp32) = sum_k A(i,k) B(j,k) for bf16 CUDA tensors; see prunedctc.h."""
+    import torch
+
+    C = torch.empty((m, n), dtype=torch.float32, device=A.device)
+    status = torch.zeros(64, dtype=torch.int32, device=A.device)
+    stream = ctypes.c_void_p(torch.cuda.current_stream(A.device).cuda_stream)
+    st = load().pctc_gemm_bf16(_dptr(A), _dptr(B), _dptr(C), m, n, k, int(a_mn_major), int(b_mn_major),
+                               int(gemm_path), _dptr(status), stream)
+    if st != 0:
+        raise PctcError(st, "pctc_gemm_bf16")
+    code = int(status[0].item())
+    if code != 0:
+        raise PctcError(6, f"device status word {code}")
+    return C

@@ -1,0 +1,355 @@
+// C ABI of libprunedctc: argument validation, workspace layout and the stream
+// order of Algorithm 1.  All arithmetic happens in the kernels this file launches.
+#include "../../include/prunedctc.h"
+#include "pctc_internal.h"
+
+#include <cmath>
+#include <cstring>
+#include <vector>
+
+namespace {
+
+using namespace pctc;
+
+constexpr size_t ALIGN = 256;
+inline size_t up(size_t x, size_t a = ALIGN) { return (x + a - 1) / a * a; }
+
+struct Plan {
+  int N, T, D, M, Usum, Kcap, Lmax, chunk, nsplit, nchunks;
+  long long V, cells;
+  size_t ldS;
+  int elem;          // bytes per element of hidden/W
+  bool bf16, use_umma, beam;
+  // byte offsets into the workspace
+  size_t o_status, o_meta_i, o_cell0, o_bitmap, o_wrank, o_vmap, o_U, o_K, o_rel, o_flags, o_X, o_lambda,
+      o_partial, o_WU, o_S, o_G, o_roww, o_alpha, o_beta, o_va, o_vb, o_offa, o_offb, o_best, o_chunk, o_dHacc;
+  size_t total;
+  size_t meta_ints;  // T_n[N] | U_n[N] | row0[N+1] | row_utt[M]
+};
+
+int default_chunk(bool /*bf16*/) { return 4096; }
+
+pctc_status_t make_plan(const pctc_problem_t* p, const int32_t* Tn, const int32_t* Un, Plan* pl) {
+  if (!p || !Tn || !Un) return PCTC_ERR_INVALID_ARG;
+  if (p->N <= 0 || p->T <= 0 || p->D <= 0 || p->V <= 0 || p->target_stride < 0) return PCTC_ERR_INVALID_ARG;
+  if (p->V > 0x7fffffffLL) return PCTC_ERR_UNSUPPORTED;
+  if (p->blank_id < 0 || (long long)p->blank_id >= p->V) return PCTC_ERR_INVALID_ARG;
+  if (p->dtype != PCTC_BF16 && p->dtype != PCTC_FP32) return PCTC_ERR_UNSUPPORTED;
+  if (p->gemm_path != PCTC_GEMM_AUTO && p->gemm_path != PCTC_GEMM_SIMT) return PCTC_ERR_INVALID_ARG;
+  if (p->chunk < 0) return PCTC_ERR_INVALID_ARG;
+  if (std::isnan(p->beam)) return PCTC_ERR_INVALID_ARG;
+  long long M = 0, Usum = 0, cells = 0;
+  int Umax = 0;
+  for (int n = 0; n < p->N; ++n) {
+    if (Tn[n] < 1 || Tn[n] > p->T) return PCTC_ERR_INVALID_ARG;
+    if (Un[n] < 0 || Un[n] > p->target_stride) return PCTC_ERR_INVALID_ARG;
+    M += Tn[n];
+    Usum += Un[n];
+    cells += (long long)Tn[n] * (2LL * Un[n] + 1);
+    if (Un[n] > Umax) Umax = Un[n];
+  }
+  if (M > 0x7fffffffLL / 2 || Usum > 0x3fffffffLL) return PCTC_ERR_UNSUPPORTED;
+  pl->N = p->N; pl->T = p->T; pl->D = p->D; pl->V = p->V;
+  pl->M = (int)M; pl->Usum = (int)Usum; pl->Kcap = (int)Usum + 1; pl->cells = cells;
+  pl->Lmax = 2 * Umax + 1;
+  if (pl->Lmax > dp_max_states()) return PCTC_ERR_UNSUPPORTED;
+  pl->bf16 = (p->dtype == PCTC_BF16);
+  pl->elem = pl->bf16 ? 2 : 4;
+  pl->use_umma = pl->bf16 && p->gemm_path == PCTC_GEMM_AUTO && (p->D % 8 == 0) && (p->V % 8 == 0);
+  pl->beam = (p->beam > 0.f) && std::isfinite(p->beam);
+  int chunk = p->chunk > 0 ? p->chunk : default_chunk(pl->bf16);
+  if (pl->use_umma) chunk = (chunk + 127) / 128 * 128;   // operand tiles of the tensor-core path
+  if ((long long)chunk > p->V) chunk = (int)(pl->use_umma ? (p->V + 7) / 8 * 8 : p->V);
+  pl->chunk = chunk;
+  pl->nchunks = (int)((p->V + chunk - 1) / chunk);
+  pl->nsplit = 32;
+  pl->ldS = up((size_t)pl->Kcap, 4);
+  pl->meta_ints = (size_t)2 * pl->N + (pl->N + 1) + pl->M;
+
+  const size_t nwords = (size_t)((p->V + 31) / 32);
+  size_t o = 0;
+  auto take = [&](size_t bytes) { size_t r = o; o = up(o + bytes); return r; };
+  pl->o_status = take(256);
+  pl->o_meta_i = take(pl->meta_ints * 4);
+  pl->o_cell0 = take((size_t)pl->N * 8);
+  pl->o_bitmap = take(nwords * 4);
+  pl->o_wrank = take(nwords * 4);
+  pl->o_vmap = take((size_t)p->V * 4);
+  pl->o_U = take((size_t)pl->Kcap * 4);
+  pl->o_K = take(4);
+  pl->o_rel = take((size_t)pl->N * (size_t)(p->target_stride > 0 ? p->target_stride : 1) * 4);
+  pl->o_flags = take((size_t)pl->N * 4);
+  pl->o_X = take((size_t)pl->M * pl->D * pl->elem);
+  pl->o_lambda = take((size_t)pl->M * 4);
+  pl->o_partial = take((size_t)pl->M * pl->nsplit * 8);
+  pl->o_WU = take((size_t)pl->Kcap * pl->D * pl->elem);
+  pl->o_S = take((size_t)pl->M * pl->ldS * 4);
+  pl->o_G = take((size_t)pl->M * pl->ldS * 4);
+  pl->o_roww = take((size_t)pl->M * 4);
+  pl->o_alpha = take((size_t)cells * 4);
+  pl->o_beta = take((size_t)cells * 4);
+  pl->o_va = pl->o_vb = pl->o_offa = pl->o_offb = pl->o_best = 0;
+  if (pl->beam) {
+    pl->o_va = take((size_t)cells * 4);
+    pl->o_vb = take((size_t)cells * 4);
+    pl->o_offa = take((size_t)pl->M * 8);
+    pl->o_offb = take((size_t)pl->M * 8);
+    pl->o_best = take((size_t)pl->N * 8);
+  }
+  pl->o_chunk = take((size_t)pl->M * pl->chunk * pl->elem);
+  pl->o_dHacc = take((size_t)pl->M * pl->D * 4);
+  pl->total = o;
+  return PCTC_OK;
+}
+
+struct GemmCall {
+  const void* A; long long lda; bool a_mn;
+  const void* B; long long ldb; bool b_mn;
+  int m, n, k;
+};
+
+cudaError_t run_gemm(bool use_umma, bool bf16, const GemmCall& c, const Epilogue& e, int* status,
+                     cudaStream_t stream) {
+  if (c.m <= 0 || c.n <= 0) return cudaSuccess;
+  if (use_umma)
+    return umma_gemm((const __nv_bfloat16*)c.A, c.lda, c.a_mn, (const __nv_bfloat16*)c.B, c.ldb, c.b_mn,
+                     c.m, c.n, c.k, e, status, stream);
+  GemmShape g;
+  g.m = c.m; g.n = c.n; g.k = c.k;
+  g.a_i = c.a_mn ? 1 : c.lda; g.a_k = c.a_mn ? c.lda : 1;
+  g.b_j = c.b_mn ? 1 : c.ldb; g.b_k = c.b_mn ? c.ldb : 1;
+  return simt_gemm(c.A, c.B, bf16, g, e, stream);
+}
+
+}  // namespace
+
+extern "C" {
+
+const char* pctc_status_string(pctc_status_t s) {
+  switch (s) {
+    case PCTC_OK: return "ok";
+    case PCTC_ERR_INVALID_ARG: return "invalid argument";
+    case PCTC_ERR_WORKSPACE_TOO_SMALL: return "workspace too small";
+    case PCTC_ERR_UNSUPPORTED: return "unsupported dtype or shape";
+    case PCTC_ERR_CUDA: return "CUDA error";
+    case PCTC_ERR_BAD_TARGET: return "bad target";
+    case PCTC_ERR_TIMEOUT: return "bounded device wait gave up";
+  }
+  return "unknown status";
+}
+
+pctc_status_t pctc_workspace_bytes(const pctc_problem_t* problem, const int32_t* input_lengths_host,
+                                   const int32_t* target_lengths_host, size_t* bytes_out) {
+  if (!bytes_out) return PCTC_ERR_INVALID_ARG;
+  Plan pl;
+  pctc_status_t st = make_plan(problem, input_lengths_host, target_lengths_host, &pl);
+  if (st != PCTC_OK) return st;
+  *bytes_out = pl.total;
+  return PCTC_OK;
+}
+
+pctc_status_t pctc_workspace_status(const void* workspace, void* stream, int32_t* status_host) {
+  if (!workspace || !status_host) return PCTC_ERR_INVALID_ARG;
+  cudaStream_t s = (cudaStream_t)stream;
+  if (cudaMemcpyAsync(status_host, workspace, 4, cudaMemcpyDeviceToHost, s) != cudaSuccess) return PCTC_ERR_CUDA;
+  if (cudaStreamSynchronize(s) != cudaSuccess) return PCTC_ERR_CUDA;
+  return *status_host ? PCTC_ERR_TIMEOUT : PCTC_OK;
+}
+
+pctc_status_t pctc_gemm_bf16(const void* A, const void* B, float* C, int32_t m, int32_t n, int32_t k,
+                             int32_t a_mn_major, int32_t b_mn_major, int32_t gemm_path,
+                             int32_t* device_status, void* stream) {
+  if (!A || !B || !C || m <= 0 || n <= 0 || k <= 0) return PCTC_ERR_INVALID_ARG;
+  if (gemm_path != PCTC_GEMM_AUTO && gemm_path != PCTC_GEMM_SIMT) return PCTC_ERR_INVALID_ARG;
+  const long long lda = a_mn_major ? m : k, ldb = b_mn_major ? n : k;
+  const bool umma = gemm_path == PCTC_GEMM_AUTO;
+  if (umma && ((lda % 8) || (ldb % 8) || ((size_t)A & 15) || ((size_t)B & 15))) return PCTC_ERR_UNSUPPORTED;
+  if (umma && !umma_available()) return PCTC_ERR_CUDA;
+  Epilogue e;
+  e.kind = EPI_STORE_F32;
+  e.out = C;
+  e.ld = n;
+  GemmCall c{A, lda, a_mn_major != 0, B, ldb, b_mn_major != 0, m, n, k};
+  cudaError_t err = run_gemm(umma, true, c, e, device_status, (cudaStream_t)stream);
+  return err == cudaSuccess ? PCTC_OK : PCTC_ERR_CUDA;
+}
+
+pctc_status_t pruned_ctc_fwd_bwd(const pctc_problem_t* p, const void* hidden, const void* W, const void* bias,
+                                 const int32_t* targets, const int32_t* input_lengths,
+                                 const int32_t* target_lengths, float* loss, void* dH, void* dW, void* dbias,
+                                 int32_t* subset_out, int32_t* K_out, int32_t* relabeled_out,
+                                 int32_t* utt_flags, void* workspace, size_t workspace_bytes, void* stream_v) {
+  Plan pl;
+  pctc_status_t st = make_plan(p, input_lengths, target_lengths, &pl);
+  if (st != PCTC_OK) return st;
+  if (!hidden || !W || !loss || !dH || !dW || !workspace) return PCTC_ERR_INVALID_ARG;
+  if (!targets && pl.Usum > 0) return PCTC_ERR_INVALID_ARG;
+  if (workspace_bytes < pl.total) return PCTC_ERR_WORKSPACE_TOO_SMALL;
+  if (((size_t)workspace & (ALIGN - 1)) || ((size_t)hidden & 15) || ((size_t)W & 15) || ((size_t)dH & 15) ||
+      ((size_t)dW & 15))
+    return PCTC_ERR_INVALID_ARG;
+  if (pl.use_umma && !umma_available()) return PCTC_ERR_CUDA;
+  cudaStream_t stream = (cudaStream_t)stream_v;
+  char* ws = (char*)workspace;
+  const int N = pl.N, M = pl.M, D = pl.D;
+  const long long V = pl.V;
+
+#define PCTC_CUDA(call)                          \
+  do {                                           \
+    if ((call) != cudaSuccess) return PCTC_ERR_CUDA; \
+  } while (0)
+
+  // ---- batch description: lengths, first stacked row, first trellis cell, row -> utterance ----
+  std::vector<int> meta(pl.meta_ints);
+  std::vector<long long> cell0(N);
+  {
+    int* Tn = meta.data();
+    int* Un = Tn + N;
+    int* row0 = Un + N;
+    int* row_utt = row0 + N + 1;
+    long long cells = 0;
+    int r = 0;
+    for (int n = 0; n < N; ++n) {
+      Tn[n] = input_lengths[n];
+      Un[n] = target_lengths[n];
+      row0[n] = r;
+      cell0[n] = cells;
+      for (int t = 0; t < Tn[n]; ++t) row_utt[r + t] = n;
+      r += Tn[n];
+      cells += (long long)Tn[n] * (2LL * Un[n] + 1);
+    }
+    row0[N] = r;
+  }
+  int* d_meta = (int*)(ws + pl.o_meta_i);
+  long long* d_cell0 = (long long*)(ws + pl.o_cell0);
+  PCTC_CUDA(cudaMemcpyAsync(d_meta, meta.data(), pl.meta_ints * 4, cudaMemcpyHostToDevice, stream));
+  PCTC_CUDA(cudaMemcpyAsync(d_cell0, cell0.data(), (size_t)N * 8, cudaMemcpyHostToDevice, stream));
+  PCTC_CUDA(cudaMemsetAsync(ws + pl.o_status, 0, 256, stream));
+  BatchMeta bm;
+  bm.T_n = d_meta;
+  bm.U_n = d_meta + N;
+  bm.row0 = d_meta + 2 * N;
+  bm.row_utt = d_meta + 3 * N + 1;
+  bm.cell0 = d_cell0;
+
+  int* d_status = (int*)(ws + pl.o_status);
+  unsigned* d_bitmap = (unsigned*)(ws + pl.o_bitmap);
+  int* d_wrank = (int*)(ws + pl.o_wrank);
+  int* d_vmap = (int*)(ws + pl.o_vmap);
+  int* d_U = (int*)(ws + pl.o_U);
+  int* d_K = (int*)(ws + pl.o_K);
+  int* d_rel = (int*)(ws + pl.o_rel);
+  int* d_flags = (int*)(ws + pl.o_flags);
+  void* d_X = ws + pl.o_X;
+  float* d_lambda = (float*)(ws + pl.o_lambda);
+  float2* d_partial = (float2*)(ws + pl.o_partial);
+  void* d_WU = ws + pl.o_WU;
+  float* d_S = (float*)(ws + pl.o_S);
+  float* d_G = (float*)(ws + pl.o_G);
+  void* d_chunk = ws + pl.o_chunk;
+  float* d_dHacc = (float*)(ws + pl.o_dHacc);
+  DpBuffers dp{};
+  dp.alpha = (float*)(ws + pl.o_alpha);
+  dp.beta = (float*)(ws + pl.o_beta);
+  dp.roww = (float*)(ws + pl.o_roww);
+  if (pl.beam) {
+    dp.va = (float*)(ws + pl.o_va);
+    dp.vb = (float*)(ws + pl.o_vb);
+    dp.off_a = (double*)(ws + pl.o_offa);
+    dp.off_b = (double*)(ws + pl.o_offb);
+    dp.best = (double*)(ws + pl.o_best);
+  }
+
+  // ---- Algorithm 1 lines 2-3: subset and relabelling ----
+  PCTC_CUDA(cudaMemsetAsync(d_U, 0xFF, (size_t)pl.Kcap * 4, stream));   // entries past K read -1
+  PCTC_CUDA(subset_and_relabel(targets, p->target_stride, bm.U_n, N, V, p->blank_id, d_bitmap, d_wrank, d_vmap,
+                               d_U, d_K, d_rel, d_flags, stream));
+  // ---- line 4: stack the valid frames ----
+  PCTC_CUDA(stack_frames(hidden, d_X, N, pl.T, D, pl.elem, bm.row_utt, bm.row0, M, stream));
+
+  // ---- line 5: normaliser, online over the vocabulary ----
+  {
+    Epilogue e;
+    e.kind = EPI_LSE_PARTIAL;
+    e.bias = bias;
+    e.partial = d_partial;
+    e.nsplit = pl.nsplit;
+    GemmCall c{d_X, D, false, W, D, false, M, (int)V, D};
+    PCTC_CUDA(run_gemm(pl.use_umma, pl.bf16, c, e, d_status, stream));
+    PCTC_CUDA(lse_combine(d_partial, pl.nsplit, M, d_lambda, stream));
+  }
+  // ---- line 6: log-probabilities of the selected classes ----
+  {
+    PCTC_CUDA(gather_rows(W, d_WU, d_U, d_K, pl.Kcap, D, pl.elem, stream));
+    Epilogue e;
+    e.kind = EPI_SUBSET_LOGP;
+    e.out = d_S;
+    e.ld = (long long)pl.ldS;
+    e.lambda = d_lambda;
+    e.bias = bias;
+    e.U = d_U;
+    e.Kdev = d_K;
+    GemmCall c{d_X, D, false, d_WU, D, false, M, pl.Kcap, D};
+    PCTC_CUDA(run_gemm(pl.use_umma, pl.bf16, c, e, d_status, stream));
+  }
+  // ---- lines 7-10: alignment DP, losses, occupancies ----
+  PCTC_CUDA(alignment_dp(d_S, (long long)pl.ldS, d_rel, p->target_stride, bm, N, M, pl.Lmax,
+                         pl.beam ? p->beam : 0.f, dp, d_G, (long long)pl.ldS, d_K, loss, d_flags, stream));
+
+  // ---- lines 11-17: backward, one vocabulary chunk at a time ----
+  for (int ci = 0; ci < pl.nchunks; ++ci) {
+    const long long v0 = (long long)ci * pl.chunk;
+    const int Cc = (int)((V - v0 < pl.chunk) ? (V - v0) : pl.chunk);
+    const char* Wc = (const char*)W + (size_t)v0 * D * pl.elem;
+    {
+      Epilogue e;                      // recompute Z_c and form Eq. "vjp"
+      e.kind = EPI_DLOGITS;
+      e.out = d_chunk;
+      e.ld = pl.chunk;
+      e.out_is_bf16 = pl.bf16;
+      e.lambda = d_lambda;
+      e.bias = bias;
+      e.v0 = v0;
+      e.vmap = d_vmap;
+      e.gamma = d_G;
+      e.ld_gamma = (long long)pl.ldS;
+      e.roww = dp.roww;
+      GemmCall c{d_X, D, false, Wc, D, false, M, Cc, D};
+      PCTC_CUDA(run_gemm(pl.use_umma, pl.bf16, c, e, d_status, stream));
+    }
+    {
+      Epilogue e;                      // dX += dZ_c W_c
+      e.kind = EPI_ACCUM_F32;
+      e.out = d_dHacc;
+      e.ld = D;
+      e.accumulate = ci > 0;
+      GemmCall c{d_chunk, pl.chunk, false, Wc, D, true, M, D, Cc};
+      PCTC_CUDA(run_gemm(pl.use_umma, pl.bf16, c, e, d_status, stream));
+    }
+    {
+      Epilogue e;                      // rows of dW: dZ_c^T X
+      e.kind = EPI_STORE_OUT;
+      e.out = (char*)dW + (size_t)v0 * D * pl.elem;
+      e.ld = D;
+      e.out_is_bf16 = pl.bf16;
+      GemmCall c{d_chunk, pl.chunk, true, d_X, D, true, Cc, D, M};
+      PCTC_CUDA(run_gemm(pl.use_umma, pl.bf16, c, e, d_status, stream));
+    }
+    if (bias && dbias)
+      PCTC_CUDA(column_sums(d_chunk, pl.bf16, pl.chunk, M, Cc, dbias, pl.bf16, v0, stream));
+  }
+  PCTC_CUDA(unstack_cast(d_dHacc, dH, N, pl.T, D, pl.bf16, bm.T_n, bm.row0, stream));
+
+  // ---- optional integer outputs ----
+  if (subset_out)
+    PCTC_CUDA(cudaMemcpyAsync(subset_out, d_U, (size_t)pl.Kcap * 4, cudaMemcpyDeviceToDevice, stream));
+  if (K_out) PCTC_CUDA(cudaMemcpyAsync(K_out, d_K, 4, cudaMemcpyDeviceToDevice, stream));
+  if (relabeled_out && p->target_stride > 0)
+    PCTC_CUDA(cudaMemcpyAsync(relabeled_out, d_rel, (size_t)N * p->target_stride * 4, cudaMemcpyDeviceToDevice,
+                              stream));
+  if (utt_flags) PCTC_CUDA(cudaMemcpyAsync(utt_flags, d_flags, (size_t)N * 4, cudaMemcpyDeviceToDevice, stream));
+#undef PCTC_CUDA
+  return PCTC_OK;
+}
+
+}  // extern "C"

@@ -1,0 +1,122 @@
+// Internal declarations shared by the translation units of libprunedctc.
+// Host-callable launch wrappers only; every wrapper enqueues on `stream` and
+// returns the cudaError_t of its launch.
+#pragma once
+
+#include <cuda_runtime.h>
+#include <cuda_bf16.h>
+#include <stdint.h>
+
+namespace pctc {
+
+// ---------------------------------------------------------------------------
+// Contractions:  acc(i,j) = sum_k A(i,k) * B(j,k),  then an epilogue.
+// ---------------------------------------------------------------------------
+
+enum EpiKind : int {
+  EPI_STORE_F32 = 0,    // C[i*ld + j] = acc                                  (validation GEMM)
+  EPI_LSE_PARTIAL = 1,  // running (max, sum exp) of z = acc + bias[j] over a column range
+  EPI_SUBSET_LOGP = 2,  // S[i*ld + j] = acc + bias[U[j]] - lambda[i],  j < K  (Algorithm 1 line 6)
+  EPI_DLOGITS = 3,      // chunk[i*ld + j] = w_i (exp(acc + bias[v0+j] - lambda[i]) - gamma[i, vmap[v0+j]])
+  EPI_ACCUM_F32 = 4,    // acc_out[i*ld + j] (+)= acc                          (dH across chunks)
+  EPI_STORE_OUT = 5     // out[i*ld + j] = T(acc)                              (rows of dW)
+};
+
+struct Epilogue {
+  int kind = EPI_STORE_F32;
+  void* out = nullptr;          // destination (type depends on kind)
+  long long ld = 0;             // its row pitch in elements
+  const float* lambda = nullptr;
+  const void* bias = nullptr;   // [V] in the operand dtype, or null
+  long long v0 = 0;             // vocabulary index of column 0 (EPI_DLOGITS / EPI_LSE_PARTIAL)
+  const int* vmap = nullptr;    // [V] class -> index in U, or -1
+  const float* gamma = nullptr; // [M, ld_gamma]
+  long long ld_gamma = 0;
+  const float* roww = nullptr;  // [M] 1 for frames of utterances in N+, else 0
+  const int* U = nullptr;       // [K] selected classes
+  const int* Kdev = nullptr;    // device scalar K
+  float2* partial = nullptr;    // [M, nsplit] (max, sum)
+  int nsplit = 1;
+  int accumulate = 0;           // EPI_ACCUM_F32: add to the destination instead of overwriting
+  int out_is_bf16 = 0;          // EPI_DLOGITS / EPI_STORE_OUT destination type
+};
+
+struct GemmShape {
+  int m = 0, n = 0, k = 0;      // extents of i, j, k
+  // element strides: A(i,k) at A[i*a_i + k*a_k], B(j,k) at B[j*b_j + k*b_k]
+  long long a_i = 0, a_k = 0, b_j = 0, b_k = 0;
+};
+
+// fp32-FMA contraction (operands fp32 or bf16 widened to fp32).
+cudaError_t simt_gemm(const void* A, const void* B, bool operands_bf16, const GemmShape& g,
+                      const Epilogue& e, cudaStream_t stream);
+
+// tcgen05 tensor-core contraction, bf16 operands.  A is [m,k] (a_mn_major=0) or [k,m];
+// B is [n,k] (b_mn_major=0) or [k,n]; row pitches lda/ldb in elements (multiples of 8).
+// status: device word receiving a non-zero code if a bounded wait gives up.
+cudaError_t umma_gemm(const __nv_bfloat16* A, long long lda, bool a_mn_major,
+                      const __nv_bfloat16* B, long long ldb, bool b_mn_major,
+                      int m, int n, int k, const Epilogue& e, int* status, cudaStream_t stream);
+bool umma_available();   // the driver entry point for tensor maps could be resolved
+
+// Combine LSE partials: lambda[i] = log sum over splits.
+cudaError_t lse_combine(const float2* partial, int nsplit, int M, float* lambda, cudaStream_t stream);
+
+// ---------------------------------------------------------------------------
+// Integer / copy steps
+// ---------------------------------------------------------------------------
+
+struct BatchMeta {              // device arrays describing the batch
+  const int* T_n;               // [N]
+  const int* U_n;               // [N]
+  const int* row0;              // [N+1] first stacked row of each utterance
+  const long long* cell0;       // [N] first trellis cell of each utterance
+  const int* row_utt;           // [M] utterance of each stacked row
+};
+
+// Algorithm 1 lines 2-3.  bitmap: ceil(V/32) words (zeroed here), vmap: [V].
+cudaError_t subset_and_relabel(const int* targets, int target_stride, const int* U_n_dev, int N,
+                               long long V, int blank, unsigned* bitmap, int* word_rank,
+                               int* vmap, int* U_out, int* K_out, int* relabeled, int* utt_flags,
+                               cudaStream_t stream);
+
+// Algorithm 1 line 4: X[row0[n] + t] = hidden[n, t], t < T_n.
+cudaError_t stack_frames(const void* hidden, void* X, int N, int T, int D, int elem_bytes,
+                         const int* row_utt, const int* row0, int M, cudaStream_t stream);
+
+// dH[n,t,:] = T(acc[row0[n]+t,:]) for t < T_n, zero for padded frames.
+cudaError_t unstack_cast(const float* acc, void* dH, int N, int T, int D, bool out_bf16,
+                         const int* T_n, const int* row0, cudaStream_t stream);
+
+// W_U[j,:] = W[U[j],:] for j < K (rows K.. of the [Kcap, D] buffer are zeroed).
+cudaError_t gather_rows(const void* W, void* W_U, const int* U, const int* Kdev, int Kcap, int D,
+                        int elem_bytes, cudaStream_t stream);
+
+// db[v0 + j] = sum_i chunk[i*ld + j]
+cudaError_t column_sums(const void* chunk, bool chunk_bf16, long long ld, int M, int cols,
+                        void* db, bool db_bf16, long long v0, cudaStream_t stream);
+
+// ---------------------------------------------------------------------------
+// Alignment dynamic program (Algorithm 1 lines 7-10; Section 3.3 for the beam)
+// ---------------------------------------------------------------------------
+
+struct DpBuffers {
+  float* alpha;        // [cells]  forward scores, per-frame normalised
+  float* beta;         // [cells]
+  float* va;           // [cells]  best-alignment forward scores (beam only)
+  float* vb;           // [cells]
+  double* off_a;       // [M] per-frame offsets of va   (beam only)
+  double* off_b;       // [M]
+  double* best;        // [N] best alignment score (beam only)
+  float* roww;         // [M]
+};
+
+// Largest trellis width the DP kernels cover.
+int dp_max_states();
+
+cudaError_t alignment_dp(const float* S, long long ldS, const int* relabeled, int target_stride,
+                         const BatchMeta& meta, int N, int M, int Lmax, float beam,
+                         const DpBuffers& buf, float* gamma, long long ld_gamma, const int* Kdev,
+                         float* loss, int* utt_flags, cudaStream_t stream);
+
+}  // namespace pctc

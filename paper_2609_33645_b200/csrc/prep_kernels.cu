@@ -1,0 +1,221 @@
+// Integer and copy steps of Algorithm 1: batch-union subset and relabelling
+// (lines 2-3), stacking of the valid frames (line 4), the gather of the selected
+// head rows (line 6), and the small reductions around the contractions.
+#include "pctc_internal.h"
+
+#include <math_constants.h>
+
+namespace pctc {
+
+namespace {
+
+// --- Algorithm 1 line 2: mark every target token in a V-bit set -------------------------------
+__global__ void k_mark_targets(const int* __restrict__ targets, int stride, const int* __restrict__ U_n,
+                               int N, long long V, int blank, unsigned* bitmap, int* utt_flags) {
+  int idx = blockIdx.x * blockDim.x + threadIdx.x;
+  if (idx >= N * stride) return;
+  int n = idx / stride, i = idx - n * stride;
+  if (i >= U_n[n]) return;
+  int tok = targets[idx];
+  if (tok == blank || tok < 0 || (long long)tok >= V) {
+    atomicOr(&utt_flags[n], 4);      // bad target: never enters U
+  } else {
+    atomicOr(&bitmap[tok >> 5], 1u << (tok & 31));
+  }
+}
+
+// --- rank the set bits: U = blank, then ascending ids; vmap[id] = position in U ----------------
+// One CTA: each thread owns a contiguous run of bitmap words, a block-wide exclusive scan of the
+// per-thread popcounts gives every run its first rank.
+__global__ void k_rank_subset(const unsigned* __restrict__ bitmap, int nwords, int blank, int* word_rank,
+                              int* vmap, int* U_out, int* K_out) {
+  __shared__ int s_scan[1024];
+  const int tid = threadIdx.x, nt = blockDim.x;
+  const int per = (nwords + nt - 1) / nt;
+  const int w0 = min(nwords, tid * per), w1 = min(nwords, w0 + per);
+  int cnt = 0;
+  for (int w = w0; w < w1; ++w) cnt += __popc(bitmap[w]);
+  s_scan[tid] = cnt;
+  __syncthreads();
+  for (int off = 1; off < nt; off <<= 1) {       // inclusive Hillis-Steele scan
+    int v = (tid >= off) ? s_scan[tid - off] : 0;
+    __syncthreads();
+    s_scan[tid] += v;
+    __syncthreads();
+  }
+  int rank = s_scan[tid] - cnt;                  // exclusive prefix
+  for (int w = w0; w < w1; ++w) {
+    unsigned bits = bitmap[w];
+    word_rank[w] = rank;
+    while (bits) {
+      int b = __ffs(bits) - 1;
+      bits &= bits - 1;
+      int id = (w << 5) + b;
+      U_out[1 + rank] = id;
+      vmap[id] = 1 + rank;
+      ++rank;
+    }
+  }
+  if (tid == nt - 1) {
+    *K_out = 1 + s_scan[tid];
+    U_out[0] = blank;
+    vmap[blank] = 0;
+  }
+}
+
+// --- Algorithm 1 line 3: relabel ----------------------------------------------------------------
+__global__ void k_relabel(const int* __restrict__ targets, int stride, const int* __restrict__ U_n, int N,
+                          long long V, int blank, const int* __restrict__ vmap, int* relabeled) {
+  int idx = blockIdx.x * blockDim.x + threadIdx.x;
+  if (idx >= N * stride) return;
+  int n = idx / stride, i = idx - n * stride;
+  int out = -1;
+  if (i < U_n[n]) {
+    int tok = targets[idx];
+    if (tok != blank && tok >= 0 && (long long)tok < V) out = vmap[tok];
+  }
+  relabeled[idx] = out;
+}
+
+// --- row copies ---------------------------------------------------------------------------------
+__device__ __forceinline__ void copy_row(const char* __restrict__ src, char* __restrict__ dst, size_t bytes) {
+  if ((((size_t)src | (size_t)dst | bytes) & 15) == 0) {
+    const uint4* s = reinterpret_cast<const uint4*>(src);
+    uint4* d = reinterpret_cast<uint4*>(dst);
+    for (size_t i = threadIdx.x; i < bytes / 16; i += blockDim.x) d[i] = s[i];
+  } else {
+    for (size_t i = threadIdx.x; i < bytes; i += blockDim.x) dst[i] = src[i];
+  }
+}
+
+__device__ __forceinline__ void zero_row(char* __restrict__ dst, size_t bytes) {
+  if ((((size_t)dst | bytes) & 15) == 0) {
+    uint4* d = reinterpret_cast<uint4*>(dst);
+    for (size_t i = threadIdx.x; i < bytes / 16; i += blockDim.x) d[i] = make_uint4(0, 0, 0, 0);
+  } else {
+    for (size_t i = threadIdx.x; i < bytes; i += blockDim.x) dst[i] = 0;
+  }
+}
+
+__global__ void k_stack_frames(const char* __restrict__ hidden, char* __restrict__ X, int T, size_t row_bytes,
+                               const int* __restrict__ row_utt, const int* __restrict__ row0) {
+  const int m = blockIdx.x;
+  const int n = row_utt[m];
+  const int t = m - row0[n];
+  copy_row(hidden + ((size_t)n * T + t) * row_bytes, X + (size_t)m * row_bytes, row_bytes);
+}
+
+template <typename TOut>
+__global__ void k_unstack_cast(const float* __restrict__ acc, TOut* __restrict__ dH, int T, int D,
+                               const int* __restrict__ T_n, const int* __restrict__ row0) {
+  const int n = blockIdx.x / T, t = blockIdx.x - n * T;
+  TOut* dst = dH + ((size_t)n * T + t) * D;
+  if (t >= T_n[n]) {
+    zero_row(reinterpret_cast<char*>(dst), (size_t)D * sizeof(TOut));
+    return;
+  }
+  const float* src = acc + ((size_t)row0[n] + t) * D;
+  for (int d = threadIdx.x; d < D; d += blockDim.x) dst[d] = TOut(src[d]);
+}
+
+__global__ void k_gather_rows(const char* __restrict__ W, char* __restrict__ W_U, const int* __restrict__ U,
+                              const int* __restrict__ Kdev, size_t row_bytes) {
+  const int j = blockIdx.x;
+  char* dst = W_U + (size_t)j * row_bytes;
+  if (j < *Kdev) copy_row(W + (size_t)U[j] * row_bytes, dst, row_bytes);
+  else zero_row(dst, row_bytes);
+}
+
+// --- db_c = dZ_c^T 1 (Algorithm 1 line 16): fixed summation order, no atomics -------------------
+template <typename TIn, typename TOut>
+__global__ void k_column_sums(const TIn* __restrict__ chunk, long long ld, int M, int cols,
+                              TOut* __restrict__ db, long long v0) {
+  __shared__ float s_part[32][33];
+  const int cx = threadIdx.x, ry = threadIdx.y;
+  const int j = blockIdx.x * 32 + cx;
+  float acc = 0.f;
+  if (j < cols)
+    for (int i = ry; i < M; i += 32) acc += float(chunk[(size_t)i * ld + j]);
+  s_part[ry][cx] = acc;
+  __syncthreads();
+  if (ry == 0 && j < cols) {
+    float tot = 0.f;
+    for (int r = 0; r < 32; ++r) tot += s_part[r][cx];
+    db[v0 + j] = TOut(tot);
+  }
+}
+
+__global__ void k_lse_combine(const float2* __restrict__ partial, int nsplit, int M, float* __restrict__ lambda) {
+  int i = blockIdx.x * blockDim.x + threadIdx.x;
+  if (i >= M) return;
+  float mx = -CUDART_INF_F;
+  for (int s = 0; s < nsplit; ++s) mx = fmaxf(mx, partial[(size_t)i * nsplit + s].x);
+  float sum = 0.f;
+  for (int s = 0; s < nsplit; ++s) {
+    float2 p = partial[(size_t)i * nsplit + s];
+    if (!(p.y <= 0.f)) sum += p.y * __expf(p.x - mx);
+  }
+  lambda[i] = mx + logf(sum);
+}
+
+}  // namespace
+
+cudaError_t subset_and_relabel(const int* targets, int target_stride, const int* U_n_dev, int N,
+                               long long V, int blank, unsigned* bitmap, int* word_rank,
+                               int* vmap, int* U_out, int* K_out, int* relabeled, int* utt_flags,
+                               cudaStream_t stream) {
+  const int nwords = (int)((V + 31) / 32);
+  cudaError_t e;
+  if ((e = cudaMemsetAsync(bitmap, 0, (size_t)nwords * 4, stream)) != cudaSuccess) return e;
+  if ((e = cudaMemsetAsync(vmap, 0xFF, (size_t)V * 4, stream)) != cudaSuccess) return e;
+  if ((e = cudaMemsetAsync(utt_flags, 0, (size_t)N * 4, stream)) != cudaSuccess) return e;
+  const int total = N * target_stride;
+  const int blocks = (total + 255) / 256;
+  if (total > 0)
+    k_mark_targets<<<blocks, 256, 0, stream>>>(targets, target_stride, U_n_dev, N, V, blank, bitmap, utt_flags);
+  k_rank_subset<<<1, 1024, 0, stream>>>(bitmap, nwords, blank, word_rank, vmap, U_out, K_out);
+  if (total > 0)
+    k_relabel<<<blocks, 256, 0, stream>>>(targets, target_stride, U_n_dev, N, V, blank, vmap, relabeled);
+  return cudaGetLastError();
+}
+
+cudaError_t stack_frames(const void* hidden, void* X, int N, int T, int D, int elem_bytes,
+                         const int* row_utt, const int* row0, int M, cudaStream_t stream) {
+  (void)N;
+  k_stack_frames<<<M, 128, 0, stream>>>((const char*)hidden, (char*)X, T, (size_t)D * elem_bytes, row_utt, row0);
+  return cudaGetLastError();
+}
+
+cudaError_t unstack_cast(const float* acc, void* dH, int N, int T, int D, bool out_bf16,
+                         const int* T_n, const int* row0, cudaStream_t stream) {
+  if (out_bf16)
+    k_unstack_cast<__nv_bfloat16><<<N * T, 128, 0, stream>>>(acc, (__nv_bfloat16*)dH, T, D, T_n, row0);
+  else
+    k_unstack_cast<float><<<N * T, 128, 0, stream>>>(acc, (float*)dH, T, D, T_n, row0);
+  return cudaGetLastError();
+}
+
+cudaError_t gather_rows(const void* W, void* W_U, const int* U, const int* Kdev, int Kcap, int D,
+                        int elem_bytes, cudaStream_t stream) {
+  k_gather_rows<<<Kcap, 128, 0, stream>>>((const char*)W, (char*)W_U, U, Kdev, (size_t)D * elem_bytes);
+  return cudaGetLastError();
+}
+
+cudaError_t column_sums(const void* chunk, bool chunk_bf16, long long ld, int M, int cols,
+                        void* db, bool db_bf16, long long v0, cudaStream_t stream) {
+  dim3 block(32, 32), grid((cols + 31) / 32);
+  if (chunk_bf16 && db_bf16)
+    k_column_sums<<<grid, block, 0, stream>>>((const __nv_bfloat16*)chunk, ld, M, cols, (__nv_bfloat16*)db, v0);
+  else if (!chunk_bf16 && !db_bf16)
+    k_column_sums<<<grid, block, 0, stream>>>((const float*)chunk, ld, M, cols, (float*)db, v0);
+  else
+    return cudaErrorInvalidValue;
+  return cudaGetLastError();
+}
+
+cudaError_t lse_combine(const float2* partial, int nsplit, int M, float* lambda, cudaStream_t stream) {
+  k_lse_combine<<<(M + 127) / 128, 128, 0, stream>>>(partial, nsplit, M, lambda);
+  return cudaGetLastError();
+}
+
+}  // namespace pctc

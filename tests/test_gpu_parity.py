@@ -1,0 +1,155 @@
+"""GPU parity: the CUDA library against the float64 oracle, element by element,
+on seeded batches small enough for the oracle (several tiles and ragged tails in
+every dimension), for both arithmetic paths and the edge cases of the method."""
+
+import dataclasses
+
+import numpy as np
+import pytest
+
+from paper_2609_33645_b200 import workloads as wl
+from tests import helpers as H
+
+pytestmark = pytest.mark.gpu
+
+SIMT, AUTO = 1, 0
+
+
+def small(name, **kw):
+    return wl.reduced(wl.CONFIGS[name], name=name + "-small", **kw)
+
+
+def test_c1_fp32_full_config(lib):
+    batch = wl.make_batch(wl.CONFIGS["c1"])
+    gpu = H.run_gpu(lib, batch)
+    ref = H.run_oracle(batch)
+    errs = H.assert_parity(gpu, ref, batch)
+    assert max(errs.values()) < 1e-4
+
+
+def test_fp32_with_bias_ragged_chunks_blank_nonzero(lib):
+    cfg = dataclasses.replace(wl.CONFIGS["c1"], name="c1-var", N=5, T_lo=9, T_hi=70, V=1531, D=72, blank=17,
+                              U_lo=0, U_hi=12, seed=77)
+    batch = wl.make_batch(cfg, with_bias=True, poison_padding=True)
+    gpu = H.run_gpu(lib, batch, chunk=500)
+    ref = H.run_oracle(batch)
+    H.assert_parity(gpu, ref, batch)
+    assert abs(float(gpu["dbias"].sum())) < 1e-3       # every frame's dlogits sum to zero
+
+
+@pytest.mark.parametrize("path", [SIMT, AUTO])
+@pytest.mark.parametrize("name,kw", [
+    ("c2", dict(V=8192, N=6, T_div=4)),                 # D=512, several row and column tiles
+    ("c3", dict(V=12288 + 384, D=256, N=4, T_div=4, U_div=2)),   # ragged last chunk, RMS-normalised frames
+])
+def test_bf16_reduced_configs(lib, path, name, kw):
+    batch = wl.make_batch(small(name, **kw), permute_ids=True, poison_padding=True)
+    gpu = H.run_gpu(lib, batch, gemm_path=path)
+    ref = H.run_oracle(batch)
+    H.assert_parity(gpu, ref, batch)
+
+
+@pytest.mark.parametrize("path", [SIMT, AUTO])
+def test_bf16_bias_blank_nonzero_small_chunk(lib, path):
+    cfg = small("c2", V=5000 if path == SIMT else 5000 - 5000 % 8, D=192, N=5, T_div=6, U_div=3, blank=4097)
+    batch = wl.make_batch(cfg, with_bias=True, permute_ids=True, poison_padding=True)
+    gpu = H.run_gpu(lib, batch, gemm_path=path, chunk=1024)
+    ref = H.run_oracle(batch)
+    H.assert_parity(gpu, ref, batch)
+
+
+@pytest.mark.parametrize("path", [SIMT, AUTO])
+def test_edge_cases_excluded_utterances(lib, path):
+    cfg = small("c2", V=2048, D=64, N=6, T_div=20, U_div=6)
+    batch = wl.make_batch(cfg, poison_padding=True)
+    tl, il, tg = batch.target_lengths, batch.input_lengths, batch.targets
+    tl[0] = 0                                   # empty target: only the all-blank alignment
+    tg[1, :tl[1]] = 7                           # all labels equal: needs 2U-1 frames
+    il[1] = 2 * tl[1] - 2                       # one frame short -> infeasible
+    batch.hidden[1, il[1]:] = 3e4
+    tg[2, 1] = batch.blank                      # blank inside a target -> bad target
+    tg[3, 0] = cfg.V + 5                        # id out of range -> bad target
+    il[4] = tl[4]                               # T = U with no repeats: exactly one alignment ...
+    row = np.arange(1, tl[4] + 1) * 3
+    tg[4, :tl[4]] = row                         # ... (distinct labels)
+    batch.hidden[4, il[4]:] = -3e4
+    gpu = H.run_gpu(lib, batch, gemm_path=path)
+    ref = H.run_oracle(batch)
+    assert list(ref["flags"]) == [0, 1, 4, 4, 0, 0]
+    H.assert_parity(gpu, ref, batch)
+
+
+def test_single_frame_and_single_utterance(lib):
+    cfg = dataclasses.replace(wl.CONFIGS["c1"], name="one", N=1, T_lo=1, T_hi=1, U_lo=1, U_hi=1, V=264, D=8, seed=5)
+    batch = wl.make_batch(cfg)
+    gpu = H.run_gpu(lib, batch)
+    ref = H.run_oracle(batch)
+    H.assert_parity(gpu, ref, batch)
+
+
+@pytest.mark.parametrize("U,T", [(14, 40), (30, 90), (60, 150), (120, 300), (250, 520), (500, 1010), (1000, 2005)])
+def test_every_trellis_width_of_the_dp(lib, U, T):
+    # one utterance per DP kernel configuration (32 ... 2048 positions), with adjacent repeats
+    cfg = dataclasses.replace(wl.CONFIGS["c1"], name=f"dp{U}", N=2, T_lo=T - 3, T_hi=T, U_lo=U - 2, U_hi=U,
+                              V=300, D=16, zipf_s=1.0, seed=U)
+    batch = wl.make_batch(cfg)
+    gpu = H.run_gpu(lib, batch)
+    ref = H.run_oracle(batch)
+    H.assert_parity(gpu, ref, batch, tol=(1e-5, 2e-4))
+
+
+@pytest.mark.parametrize("beam", [2.0, 8.0, 16.0, 64.0])
+@pytest.mark.parametrize("path", [SIMT])
+def test_finite_beam_matches_oracle_at_the_same_beam(lib, beam, path):
+    cfg = dataclasses.replace(wl.CONFIGS["c1"], name="beam", N=4, T_lo=60, T_hi=140, U_lo=5, U_hi=40,
+                              V=1000, D=64, zipf_s=1.0, seed=31)
+    batch = wl.make_batch(cfg)
+    batch.hidden *= 3.0                      # sharper posteriors so that the beams prune
+    gpu = H.run_gpu(lib, batch, beam=beam, gemm_path=path)
+    ref = H.run_oracle(batch, beam=beam)
+    H.assert_parity(gpu, ref, batch, tol=(1e-5, 5e-4))
+    exact = H.run_oracle(batch)
+    Delta, delta = H.O.discarded_mass(ref["loss"], exact["loss"])
+    assert np.all(Delta >= -1e-9)
+    if beam <= 2.0:
+        assert Delta.max() > 1e-6            # the case does prune
+    # loss stays an upper bound of the exact loss on the GPU too
+    assert np.all(gpu["loss"] >= exact["loss"] * (1 - 1e-5))
+
+
+def test_beam_bf16_reduced_c5_shape(lib):
+    cfg = small("c5", V=4096, D=128, N=3, T_div=10, U_div=10)
+    batch = wl.make_batch(cfg)
+    for beam in (8.0, 16.0):
+        gpu = H.run_gpu(lib, batch, beam=beam)
+        ref = H.run_oracle(batch, beam=beam)
+        H.assert_parity(gpu, ref, batch)
+
+
+def test_two_calls_are_bitwise_identical_and_workspace_is_reusable(lib):
+    import torch
+    batch = wl.make_batch(small("c2", V=4096, D=128, N=4, T_div=8, U_div=4))
+    a = H.run_gpu(lib, batch)
+    b = H.run_gpu(lib, batch)
+    for k in ("loss", "dH", "dW", "subset", "relabeled"):
+        np.testing.assert_array_equal(a[k], b[k])
+    torch.cuda.synchronize()
+
+
+@pytest.mark.parametrize("a_mn", [False, True])
+@pytest.mark.parametrize("b_mn", [False, True])
+@pytest.mark.parametrize("m,n,k", [(128, 256, 64), (200, 264, 328), (1000, 520, 1032), (72, 8, 4096)])
+def test_tensor_core_contraction_all_operand_layouts(lib, a_mn, b_mn, m, n, k):
+    import torch
+    g = torch.Generator(device="cpu").manual_seed(m * 7 + n * 3 + k)
+    A = torch.randn((m, k), generator=g).to(torch.bfloat16)
+    B = torch.randn((n, k), generator=g).to(torch.bfloat16)
+    ref = A.double() @ B.double().T
+    Ad = (A.T.contiguous() if a_mn else A).cuda()
+    Bd = (B.T.contiguous() if b_mn else B).cuda()
+    if (a_mn and m % 8) or (b_mn and n % 8):
+        pytest.skip("contiguous extent must be a multiple of 8")
+    for path in (SIMT, AUTO):
+        C = lib.gemm_bf16(Ad, Bd, m, n, k, a_mn, b_mn, gemm_path=path).cpu().double()
+        err = (C - ref).abs().max().item()
+        assert err <= 2e-3 * (k ** 0.5), (path, err)

@@ -356,7 +356,7 @@ cudaError_t launch_sweep(const SweepArgs& a, int N, cudaStream_t stream) {
   constexpr int NX = (MODE == MODE_MASKED) ? (2 * SPL + 2) : 0;
   const size_t smem = (size_t)DEPTH * (NE + NX) * W * 32 * sizeof(float);
   auto kern = k_ctc_sweep<W, SPL, DEPTH, MODE>;
-  if (smem > 48 * 1024) {
+  if (smem + 2048 > 48 * 1024) {
     cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
     if (e != cudaSuccess) return e;
   }

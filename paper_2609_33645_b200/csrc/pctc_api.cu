@@ -62,7 +62,7 @@ pctc_status_t make_plan(const pctc_problem_t* p, const int32_t* Tn, const int32_
   if ((long long)chunk > p->V) chunk = (int)(pl->use_umma ? (p->V + 7) / 8 * 8 : p->V);
   pl->chunk = chunk;
   pl->nchunks = (int)((p->V + chunk - 1) / chunk);
-  pl->nsplit = 32;
+  pl->nsplit = 64;            // capacity of the partial buffer; the launch may use fewer
   pl->ldS = up((size_t)pl->Kcap, 4);
   pl->meta_ints = (size_t)2 * pl->N + (pl->N + 1) + pl->M;
 
@@ -273,10 +273,10 @@ pctc_status_t pruned_ctc_fwd_bwd(const pctc_problem_t* p, const void* hidden, co
     e.kind = EPI_LSE_PARTIAL;
     e.bias = bias;
     e.partial = d_partial;
-    e.nsplit = pl.nsplit;
+    e.nsplit = pl.use_umma ? umma_lse_splits(M, (int)V) : 32;
     GemmCall c{d_X, D, false, W, D, false, M, (int)V, D};
     PCTC_CUDA(run_gemm(pl.use_umma, pl.bf16, c, e, d_status, stream));
-    PCTC_CUDA(lse_combine(d_partial, pl.nsplit, M, d_lambda, stream));
+    PCTC_CUDA(lse_combine(d_partial, e.nsplit, M, d_lambda, stream));
   }
   // ---- line 6: log-probabilities of the selected classes ----
   {

@@ -1,8 +1,572 @@
+// tcgen05 tensor-core contraction for sm_100a with the fused epilogues of
+// Algorithm 1:  acc(i,j) = sum_k A(i,k) B(j,k), bf16 operands, fp32 accumulators
+// in tensor memory.
+//
+// One persistent CTA per SM, 192 threads in three roles:
+//   warp 0      TMA producer: 128-byte-swizzled operand tiles into a 4-stage ring
+//   warp 1      MMA issuer: tcgen05.mma 128x256x16 from shared-memory descriptors
+//               into one of two 256-column accumulators in tensor memory
+//   warps 2..5  epilogue: tcgen05.ld (one accumulator row per thread), the fused
+//               arithmetic, global stores; runs while the next tile's MMAs issue
+// Operands may be K-major (k contiguous) or MN-major (the transposed storage),
+// chosen at run time through the descriptors, so that dX += dZ W and
+// dW = dZ^T X need no transposed copies.
+//
+// Every mbarrier wait is bounded: after about two seconds a wait stores a code
+// in the caller's status word, raises a CTA-wide abort flag and every role
+// leaves its loop; the CTA then drains its own copies, frees its tensor memory
+// and returns.
 #include "pctc_internal.h"
+
+#include <cuda.h>
+#include <math_constants.h>
+
 namespace pctc {
-bool umma_available() { return false; }
-cudaError_t umma_gemm(const __nv_bfloat16*, long long, bool, const __nv_bfloat16*, long long, bool, int, int, int,
-                      const Epilogue&, int*, cudaStream_t) {
-  return cudaErrorNotSupported;
+
+namespace {
+
+constexpr int BM = 128, BN = 256, BK = 64, STAGES = 4;
+constexpr int A_STAGE_BYTES = BM * BK * 2;
+constexpr int B_STAGE_BYTES = BN * BK * 2;
+constexpr int NUM_THREADS = 192;
+constexpr int TMEM_COLS = 512;
+constexpr int MN_GROUP_BYTES = 64 * BK * 2;          // one 64-wide MN group of an MN-major tile
+constexpr long long WAIT_LIMIT_CYCLES = 4000000000LL;
+constexpr float LOG2E = 1.4426950408889634f;
+constexpr float LN2 = 0.6931471805599453f;
+
+struct UmmaArgs {
+  int m, n, k;
+  int a_mn, b_mn;
+  int nsplit;          // EPI_LSE_PARTIAL: column splits per row tile
+  int* status;
+  Epilogue e;
+};
+
+struct SharedTail {   // after the operand ring
+  unsigned long long full[STAGES];
+  unsigned long long empty[STAGES];
+  unsigned long long tmem_full[2];
+  unsigned long long tmem_empty[2];
+  unsigned long long done;
+  unsigned tmem_base;
+  int abort;
+  float bias[4][BN];       // per epilogue warp: bias of the tile's columns
+  int2 list[4][BN];        // per epilogue warp: (column, index in U) of the selected classes
+};
+
+constexpr size_t SMEM_BYTES = 1024 + (size_t)STAGES * (A_STAGE_BYTES + B_STAGE_BYTES) + sizeof(SharedTail);
+
+// ---------------------------------------------------------------------------------------------
+// PTX wrappers
+// ---------------------------------------------------------------------------------------------
+__device__ __forceinline__ unsigned smem_u32(const void* p) { return (unsigned)__cvta_generic_to_shared(p); }
+
+__device__ __forceinline__ void mbar_init(unsigned long long* bar, unsigned count) {
+  asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(smem_u32(bar)), "r"(count) : "memory");
 }
+__device__ __forceinline__ void mbar_expect_tx(unsigned long long* bar, unsigned bytes) {
+  asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(smem_u32(bar)), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive(unsigned long long* bar) {
+  asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(smem_u32(bar)) : "memory");
+}
+__device__ __forceinline__ bool mbar_try(unsigned long long* bar, unsigned parity) {
+  unsigned ok;
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+      "selp.u32 %0, 1, 0, p;\n\t}"
+      : "=r"(ok)
+      : "r"(smem_u32(bar)), "r"(parity)
+      : "memory");
+  return ok != 0;
+}
+// Bounded wait.  Returns false if the CTA is aborting or the limit ran out (then it raises the abort).
+__device__ __forceinline__ bool mbar_wait(unsigned long long* bar, unsigned parity, volatile int* abort_flag,
+                                          int* status, int code, long long limit = WAIT_LIMIT_CYCLES) {
+  if (mbar_try(bar, parity)) return true;
+  const long long t0 = clock64();
+  for (unsigned it = 1;; ++it) {
+    if (mbar_try(bar, parity)) return true;
+    if ((it & 255u) == 0u) {
+      if (*abort_flag) return false;
+      if (clock64() - t0 > limit) {
+        *abort_flag = 1;
+        if (status) atomicCAS(status, 0, code);
+        return false;
+      }
+    }
+  }
+}
+
+__device__ __forceinline__ void tma_load_2d(void* smem_dst, const CUtensorMap* map, int c0, int c1,
+                                            unsigned long long* bar) {
+  asm volatile(
+      "cp.async.bulk.tensor.2d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
+      ::"r"(smem_u32(smem_dst)), "l"(map), "r"(c0), "r"(c1), "r"(smem_u32(bar))
+      : "memory");
+}
+
+__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
+
+__device__ __forceinline__ void tc_commit(unsigned long long* bar) {
+  asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(smem_u32(bar))
+               : "memory");
+}
+
+__device__ __forceinline__ void tc_mma_bf16(unsigned tmem_d, unsigned long long adesc, unsigned long long bdesc,
+                                            unsigned idesc, unsigned accumulate) {
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "setp.ne.b32 p, %4, 0;\n\t"
+      "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
+      ::"r"(tmem_d), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate)
+      : "memory");
+}
+
+// 32 lanes x 32 consecutive 32-bit columns: thread `lane` of the warp receives its row.
+__device__ __forceinline__ void tmem_ld32(unsigned taddr, float* v) {
+  unsigned r[32];
+  asm volatile(
+      "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
+      "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
+      "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];"
+      : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]),
+        "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]),
+        "=r"(r[16]), "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]),
+        "=r"(r[24]), "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
+      : "r"(taddr)
+      : "memory");
+  asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+#pragma unroll
+  for (int i = 0; i < 32; ++i) v[i] = __uint_as_float(r[i]);
+}
+__device__ __forceinline__ float tmem_ld1(unsigned taddr) {
+  unsigned r;
+  asm volatile("tcgen05.ld.sync.aligned.32x32b.x1.b32 {%0}, [%1];" : "=r"(r) : "r"(taddr) : "memory");
+  asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+  return __uint_as_float(r);
+}
+
+__device__ __forceinline__ float ex2(float x) {
+  float y;
+  asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+  return y;
+}
+
+// Shared-memory matrix descriptor of a 128-byte-swizzled bf16 tile.
+//   K-major : rows of 64 k (128 bytes); 8-row groups 1024 bytes apart (stride byte offset).
+//   MN-major: rows of 64 m/n (128 bytes), one row per k; 8-k groups 1024 bytes apart (stride byte
+//             offset); 64-wide m/n groups MN_GROUP_BYTES apart (leading byte offset).
+__device__ __forceinline__ unsigned long long make_smem_desc(unsigned addr, bool mn_major) {
+  unsigned long long d = 0;
+  d |= (unsigned long long)((addr & 0x3FFFFu) >> 4);
+  d |= (unsigned long long)(mn_major ? (MN_GROUP_BYTES >> 4) : 1) << 16;
+  d |= (unsigned long long)(1024 >> 4) << 32;
+  d |= 1ull << 46;     // descriptor version of sm_100
+  d |= 2ull << 61;     // 128-byte swizzle
+  return d;
+}
+
+__device__ __forceinline__ void split_range(int n_tiles, int splits, int sp, int& start, int& cnt) {
+  const int base = n_tiles / splits, rem = n_tiles % splits;
+  cnt = base + (sp < rem ? 1 : 0);
+  start = sp * base + min(sp, rem);
+}
+
+// ---------------------------------------------------------------------------------------------
+// The kernel
+// ---------------------------------------------------------------------------------------------
+template <int EPI>
+__global__ void __launch_bounds__(NUM_THREADS, 1)
+k_umma_gemm(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB, UmmaArgs a) {
+  extern __shared__ unsigned char smem_raw[];
+  unsigned char* smem = (unsigned char*)(((size_t)smem_raw + 1023) & ~(size_t)1023);
+  unsigned char* sA = smem;
+  unsigned char* sB = smem + (size_t)STAGES * A_STAGE_BYTES;
+  SharedTail* st = (SharedTail*)(smem + (size_t)STAGES * (A_STAGE_BYTES + B_STAGE_BYTES));
+
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+
+  // problem decomposition, identical in every role
+  int n_eff = a.n;
+  if (EPI == EPI_SUBSET_LOGP) n_eff = min(a.n, *a.e.Kdev);
+  const int m_tiles = (a.m + BM - 1) / BM;
+  const int n_tiles = (n_eff + BN - 1) / BN;
+  const int splits = (EPI == EPI_LSE_PARTIAL) ? a.nsplit : n_tiles;
+  const int units = m_tiles * splits;
+  const int k_blocks = (a.k + BK - 1) / BK;
+
+  if (threadIdx.x == 0) {
+    for (int s = 0; s < STAGES; ++s) { mbar_init(&st->full[s], 1); mbar_init(&st->empty[s], 1); }
+    for (int s = 0; s < 2; ++s) { mbar_init(&st->tmem_full[s], 1); mbar_init(&st->tmem_empty[s], 4); }
+    mbar_init(&st->done, 1);
+    st->abort = 0;
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+  }
+  if (warp == 1) {
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&st->tmem_base)),
+                 "r"(TMEM_COLS)
+                 : "memory");
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+  }
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const unsigned tmem_base = st->tmem_base;
+  volatile int* abort_flag = &st->abort;
+
+  if (warp == 0) {
+    // ===================== TMA producer =====================
+    if (lane == 0) {
+      unsigned g = 0;
+      bool ok = true;
+      for (int u = blockIdx.x; u < units && ok; u += gridDim.x) {
+        const int mt = u % m_tiles, sp = u / m_tiles;
+        int nt0, cnt;
+        split_range(n_tiles, splits, sp, nt0, cnt);
+        for (int nt = nt0; nt < nt0 + cnt && ok; ++nt) {
+          for (int kb = 0; kb < k_blocks; ++kb, ++g) {
+            const int s = g % STAGES;
+            const unsigned ph = (g / STAGES) & 1u;
+            if (!mbar_wait(&st->empty[s], ph ^ 1u, abort_flag, a.status, 1)) { ok = false; break; }
+            mbar_expect_tx(&st->full[s], A_STAGE_BYTES + B_STAGE_BYTES);
+            unsigned char* dA = sA + (size_t)s * A_STAGE_BYTES;
+            unsigned char* dB = sB + (size_t)s * B_STAGE_BYTES;
+            if (!a.a_mn) {
+              tma_load_2d(dA, &tmA, kb * BK, mt * BM, &st->full[s]);
+            } else {
+#pragma unroll
+              for (int q = 0; q < BM / 64; ++q)
+                tma_load_2d(dA + q * MN_GROUP_BYTES, &tmA, mt * BM + q * 64, kb * BK, &st->full[s]);
+            }
+            if (!a.b_mn) {
+              tma_load_2d(dB, &tmB, kb * BK, nt * BN, &st->full[s]);
+            } else {
+#pragma unroll
+              for (int q = 0; q < BN / 64; ++q)
+                tma_load_2d(dB + q * MN_GROUP_BYTES, &tmB, nt * BN + q * 64, kb * BK, &st->full[s]);
+            }
+          }
+        }
+      }
+      // drain: every copy this thread issued has landed before the CTA may exit
+      const unsigned issued = g;
+      for (unsigned j = (issued > STAGES ? issued - STAGES : 0); j < issued; ++j)
+        mbar_wait(&st->full[j % STAGES], (j / STAGES) & 1u, abort_flag, nullptr, 0, 200000000LL);
+    }
+  } else if (warp == 1) {
+    // ===================== MMA issuer =====================
+    if (lane == 0) {
+      const unsigned idesc = (1u << 4) | (1u << 7) | (1u << 10) | ((unsigned)(a.a_mn ? 1 : 0) << 15) |
+                             ((unsigned)(a.b_mn ? 1 : 0) << 16) | ((unsigned)(BN >> 3) << 17) |
+                             ((unsigned)(BM >> 4) << 24);
+      const unsigned a_step = a.a_mn ? (2048u >> 4) : (32u >> 4);   // descriptor advance per 16 k
+      const unsigned b_step = a.b_mn ? (2048u >> 4) : (32u >> 4);
+      unsigned g = 0, it = 0;
+      bool ok = true;
+      for (int u = blockIdx.x; u < units && ok; u += gridDim.x) {
+        const int sp = u / m_tiles;
+        int nt0, cnt;
+        split_range(n_tiles, splits, sp, nt0, cnt);
+        for (int nt = nt0; nt < nt0 + cnt && ok; ++nt, ++it) {
+          const unsigned acc = it & 1u, aph = (it >> 1) & 1u;
+          if (!mbar_wait(&st->tmem_empty[acc], aph ^ 1u, abort_flag, a.status, 2)) { ok = false; break; }
+          tc_fence_after();
+          const unsigned d_tmem = tmem_base + acc * BN;
+          for (int kb = 0; kb < k_blocks; ++kb, ++g) {
+            const int s = g % STAGES;
+            const unsigned ph = (g / STAGES) & 1u;
+            if (!mbar_wait(&st->full[s], ph, abort_flag, a.status, 3)) { ok = false; break; }
+            tc_fence_after();
+            const unsigned long long adesc = make_smem_desc(smem_u32(sA + (size_t)s * A_STAGE_BYTES), a.a_mn);
+            const unsigned long long bdesc = make_smem_desc(smem_u32(sB + (size_t)s * B_STAGE_BYTES), a.b_mn);
+#pragma unroll
+            for (int kk = 0; kk < BK / 16; ++kk)
+              tc_mma_bf16(d_tmem, adesc + (unsigned long long)(kk * a_step), bdesc + (unsigned long long)(kk * b_step),
+                          idesc, (kb | kk) != 0 ? 1u : 0u);
+            tc_commit(&st->empty[s]);        // frees the stage once these MMAs have read it
+          }
+          if (ok) tc_commit(&st->tmem_full[acc]);
+        }
+      }
+      // all MMAs issued by this thread have completed before tensor memory is freed
+      tc_commit(&st->done);
+      mbar_wait(&st->done, 0, abort_flag, nullptr, 0, 200000000LL);
+    }
+  } else {
+    // ===================== epilogue warps =====================
+    const int ew = warp - 2;                 // private staging slot
+    const int q = warp & 3;                  // tensor-memory lane quarter this warp may read
+    const int r = q * 32 + lane;             // accumulator row of this thread
+    float* sb = st->bias[ew];
+    int2* sl = st->list[ew];
+    unsigned it = 0;
+    bool ok = true;
+    for (int u = blockIdx.x; u < units && ok; u += gridDim.x) {
+      const int mt = u % m_tiles, sp = u / m_tiles;
+      int nt0, cnt;
+      split_range(n_tiles, splits, sp, nt0, cnt);
+      const int i = mt * BM + r;
+      const bool row_ok = i < a.m;
+      float lam2 = 0.f, lam = 0.f, w = 0.f;
+      if ((EPI == EPI_SUBSET_LOGP || EPI == EPI_DLOGITS) && row_ok) { lam = a.e.lambda[i]; lam2 = lam * LOG2E; }
+      if (EPI == EPI_DLOGITS && row_ok) w = a.e.roww[i];
+      float run_max2 = -CUDART_INF_F, run_sum = 0.f;     // EPI_LSE_PARTIAL, base-2 domain
+
+      for (int nt = nt0; nt < nt0 + cnt && ok; ++nt, ++it) {
+        const unsigned acc = it & 1u, aph = (it >> 1) & 1u;
+        const int n0 = nt * BN;
+        int nsel = 0;
+        // ---- warp-private staging of per-column data (overlaps the MMAs of this tile) ----
+        if (EPI == EPI_LSE_PARTIAL || EPI == EPI_DLOGITS || EPI == EPI_SUBSET_LOGP) {
+          const __nv_bfloat16* bias = (const __nv_bfloat16*)a.e.bias;
+#pragma unroll
+          for (int c = lane; c < BN; c += 32) {
+            const int j = n0 + c;
+            float b = 0.f;
+            if (bias && j < n_eff) {
+              if (EPI == EPI_SUBSET_LOGP) b = __bfloat162float(bias[a.e.U[j]]);
+              else b = __bfloat162float(bias[a.e.v0 + j]);
+            }
+            sb[c] = b;
+          }
+        }
+        if (EPI == EPI_DLOGITS) {
+          for (int c0 = 0; c0 < BN; c0 += 32) {
+            const int j = n0 + c0 + lane;
+            const int jj = (j < n_eff) ? a.e.vmap[a.e.v0 + j] : -1;
+            const unsigned mask = __ballot_sync(0xffffffffu, jj >= 0);
+            if (jj >= 0) sl[nsel + __popc(mask & ((1u << lane) - 1u))] = make_int2(c0 + lane, jj);
+            nsel += __popc(mask);
+          }
+        }
+        __syncwarp();
+
+        int got = 0;
+        if (lane == 0) got = mbar_wait(&st->tmem_full[acc], aph, abort_flag, a.status, 4) ? 1 : 0;
+        got = __shfl_sync(0xffffffffu, got, 0);
+        if (!got) { ok = false; break; }
+        tc_fence_after();
+        const unsigned taddr = tmem_base + ((unsigned)(q * 32) << 16) + acc * BN;
+
+#pragma unroll 1
+        for (int cg = 0; cg < BN / 32; ++cg) {
+          if (n0 + cg * 32 >= n_eff) break;          // warp-uniform
+          float v[32];
+          tmem_ld32(taddr + cg * 32, v);
+          const int j0 = n0 + cg * 32;
+          if (EPI == EPI_STORE_F32) {
+            if (row_ok) {
+              float* dst = (float*)a.e.out + (long long)i * a.e.ld + j0;
+#pragma unroll
+              for (int c = 0; c < 32; ++c)
+                if (j0 + c < n_eff) dst[c] = v[c];
+            }
+          } else if (EPI == EPI_ACCUM_F32) {
+            if (row_ok) {
+              float4* dst = (float4*)((float*)a.e.out + (long long)i * a.e.ld + j0);
+#pragma unroll
+              for (int c4 = 0; c4 < 8; ++c4) {
+                if (j0 + c4 * 4 < n_eff) {
+                  float4 o = make_float4(v[c4 * 4], v[c4 * 4 + 1], v[c4 * 4 + 2], v[c4 * 4 + 3]);
+                  if (a.e.accumulate) {
+                    const float4 old = dst[c4];
+                    o.x += old.x; o.y += old.y; o.z += old.z; o.w += old.w;
+                  }
+                  dst[c4] = o;
+                }
+              }
+            }
+          } else if (EPI == EPI_STORE_OUT || EPI == EPI_DLOGITS) {
+            if (EPI == EPI_DLOGITS) {
+#pragma unroll
+              for (int c = 0; c < 32; ++c)
+                v[c] = w * ex2(fmaf(v[c] + sb[cg * 32 + c], LOG2E, -lam2));
+            }
+            if (row_ok) {
+              uint4* dst = (uint4*)((__nv_bfloat16*)a.e.out + (long long)i * a.e.ld + j0);
+#pragma unroll
+              for (int c8 = 0; c8 < 4; ++c8) {
+                if (j0 + c8 * 8 < n_eff) {
+                  uint4 o;
+                  __nv_bfloat162 p0 = __floats2bfloat162_rn(v[c8 * 8 + 0], v[c8 * 8 + 1]);
+                  __nv_bfloat162 p1 = __floats2bfloat162_rn(v[c8 * 8 + 2], v[c8 * 8 + 3]);
+                  __nv_bfloat162 p2 = __floats2bfloat162_rn(v[c8 * 8 + 4], v[c8 * 8 + 5]);
+                  __nv_bfloat162 p3 = __floats2bfloat162_rn(v[c8 * 8 + 6], v[c8 * 8 + 7]);
+                  o.x = *(unsigned*)&p0; o.y = *(unsigned*)&p1; o.z = *(unsigned*)&p2; o.w = *(unsigned*)&p3;
+                  dst[c8] = o;
+                }
+              }
+            }
+          } else if (EPI == EPI_SUBSET_LOGP) {
+            if (row_ok) {
+              float* dst = (float*)a.e.out + (long long)i * a.e.ld + j0;
+#pragma unroll
+              for (int c = 0; c < 32; ++c)
+                if (j0 + c < n_eff) dst[c] = v[c] + sb[cg * 32 + c] - lam;
+            }
+          } else if (EPI == EPI_LSE_PARTIAL) {
+            float gmax = -CUDART_INF_F;
+#pragma unroll
+            for (int c = 0; c < 32; ++c) {
+              v[c] = (j0 + c < n_eff) ? (v[c] + sb[cg * 32 + c]) * LOG2E : -CUDART_INF_F;
+              gmax = fmaxf(gmax, v[c]);
+            }
+            if (gmax > run_max2) {
+              run_sum *= ex2(run_max2 - gmax);     // ex2(-inf) = 0 on the first group
+              run_max2 = gmax;
+            }
+            float s = 0.f;
+#pragma unroll
+            for (int c = 0; c < 32; ++c) s += ex2(v[c] - run_max2);
+            run_sum += s;
+            if (gmax != gmax) run_sum = gmax;      // NaN logits poison the normaliser
+          }
+        }
+
+        if (EPI == EPI_DLOGITS) {
+          // selected classes: subtract the occupancy in fp32, before the rounding to bf16
+          for (int e = 0; e < nsel; ++e) {
+            const int2 cj = sl[e];
+            const float z = tmem_ld1(taddr + cj.x);
+            if (row_ok) {
+              const float p = ex2(fmaf(z + sb[cj.x], LOG2E, -lam2));
+              const float g = a.e.gamma[(long long)i * a.e.ld_gamma + cj.y];
+              ((__nv_bfloat16*)a.e.out)[(long long)i * a.e.ld + n0 + cj.x] = __float2bfloat16_rn(w * (p - g));
+            }
+          }
+        }
+
+        tc_fence_before();
+        __syncwarp();
+        if (lane == 0) mbar_arrive(&st->tmem_empty[acc]);
+      }
+
+      if (EPI == EPI_LSE_PARTIAL && ok && row_ok)
+        a.e.partial[(long long)i * a.nsplit + sp] = make_float2(run_max2 * LN2, run_sum);
+    }
+  }
+
+  tc_fence_before();
+  __syncthreads();
+  if (warp == 1) {
+    tc_fence_after();
+    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(TMEM_COLS) : "memory");
+  }
+}
+
+// ---------------------------------------------------------------------------------------------
+// Host side
+// ---------------------------------------------------------------------------------------------
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+EncodeTiledFn encode_fn() {
+  static EncodeTiledFn fn = [] {
+    void* p = nullptr;
+    cudaDriverEntryPointQueryResult q;
+    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &q) != cudaSuccess ||
+        q != cudaDriverEntryPointSuccess)
+      p = nullptr;
+    return (EncodeTiledFn)p;
+  }();
+  return fn;
+}
+
+// 2-D bf16 tensor map: `inner` contiguous elements per row, `rows` rows of pitch `ld` elements.
+bool make_map(CUtensorMap* map, const void* base, unsigned long long inner, unsigned long long rows,
+              unsigned long long ld, unsigned box_inner, unsigned box_rows) {
+  EncodeTiledFn fn = encode_fn();
+  if (!fn) return false;
+  cuuint64_t dims[2] = {inner, rows};
+  cuuint64_t strides[1] = {ld * 2};
+  cuuint32_t box[2] = {box_inner, box_rows};
+  cuuint32_t estr[2] = {1, 1};
+  return fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(base), dims, strides, box, estr,
+            CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+            CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+int sm_count() {
+  static int n = [] {
+    int dev = 0, v = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess) return 148;
+    if (cudaDeviceGetAttribute(&v, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || v <= 0) return 148;
+    return v;
+  }();
+  return n;
+}
+
+template <int EPI>
+cudaError_t launch(const CUtensorMap& tmA, const CUtensorMap& tmB, const UmmaArgs& a, int grid, cudaStream_t stream) {
+  static bool configured = false;
+  if (!configured) {
+    cudaError_t e = cudaFuncSetAttribute(k_umma_gemm<EPI>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)SMEM_BYTES);
+    if (e != cudaSuccess) return e;
+    configured = true;
+  }
+  k_umma_gemm<EPI><<<grid, NUM_THREADS, SMEM_BYTES, stream>>>(tmA, tmB, a);
+  return cudaGetLastError();
+}
+
+}  // namespace
+
+bool umma_available() { return encode_fn() != nullptr; }
+
+int umma_lse_splits(int m, int n) {
+  // column splits per row tile such that the (row tile, split) units fill whole waves of CTAs
+  const int sms = sm_count();
+  const int m_tiles = (m + BM - 1) / BM, n_tiles = (n + BN - 1) / BN;
+  int best = 1;
+  double best_cost = 1e30;
+  for (int s = 1; s <= 64 && s <= n_tiles; ++s) {
+    const long long units = (long long)m_tiles * s;
+    const long long waves = (units + sms - 1) / sms;
+    const int per = (n_tiles + s - 1) / s;                 // column tiles of the largest split
+    const double cost = (double)waves * per + 0.05 * waves; // tile-times on the critical CTA + per-unit overhead
+    if (cost < best_cost - 1e-9) { best_cost = cost; best = s; }
+  }
+  return best;
+}
+
+cudaError_t umma_gemm(const __nv_bfloat16* A, long long lda, bool a_mn_major,
+                      const __nv_bfloat16* B, long long ldb, bool b_mn_major,
+                      int m, int n, int k, const Epilogue& e, int* status, cudaStream_t stream) {
+  if (m <= 0 || n <= 0 || k <= 0) return cudaSuccess;
+  if ((lda % 8) || (ldb % 8) || ((size_t)A & 15) || ((size_t)B & 15)) return cudaErrorInvalidValue;
+  alignas(64) CUtensorMap tmA, tmB;
+  bool ok = true;
+  if (!a_mn_major) ok = ok && make_map(&tmA, A, (unsigned long long)k, (unsigned long long)m, lda, BK, BM);
+  else ok = ok && make_map(&tmA, A, (unsigned long long)m, (unsigned long long)k, lda, 64, BK);
+  if (!b_mn_major) ok = ok && make_map(&tmB, B, (unsigned long long)k, (unsigned long long)n, ldb, BK, BN);
+  else ok = ok && make_map(&tmB, B, (unsigned long long)n, (unsigned long long)k, ldb, 64, BK);
+  if (!ok) return cudaErrorInvalidValue;
+
+  UmmaArgs a;
+  a.m = m; a.n = n; a.k = k;
+  a.a_mn = a_mn_major ? 1 : 0;
+  a.b_mn = b_mn_major ? 1 : 0;
+  a.nsplit = e.nsplit;
+  a.status = status;
+  a.e = e;
+  const int m_tiles = (m + BM - 1) / BM, n_tiles = (n + BN - 1) / BN;
+  long long units = (long long)m_tiles * (e.kind == EPI_LSE_PARTIAL ? e.nsplit : n_tiles);
+  if (e.kind == EPI_LSE_PARTIAL && (e.nsplit < 1 || e.nsplit > n_tiles)) return cudaErrorInvalidValue;
+  const int grid = (int)(units < sm_count() ? units : sm_count());
+  switch (e.kind) {
+    case EPI_STORE_F32: return launch<EPI_STORE_F32>(tmA, tmB, a, grid, stream);
+    case EPI_LSE_PARTIAL: return launch<EPI_LSE_PARTIAL>(tmA, tmB, a, grid, stream);
+    case EPI_SUBSET_LOGP: return launch<EPI_SUBSET_LOGP>(tmA, tmB, a, grid, stream);
+    case EPI_DLOGITS: return launch<EPI_DLOGITS>(tmA, tmB, a, grid, stream);
+    case EPI_ACCUM_F32: return launch<EPI_ACCUM_F32>(tmA, tmB, a, grid, stream);
+    case EPI_STORE_OUT: return launch<EPI_STORE_OUT>(tmA, tmB, a, grid, stream);
+  }
+  return cudaErrorInvalidValue;
+}
+
 }  // namespace pctc

@@ -1,0 +1,382 @@
+#!/usr/bin/env python
+"""Benchmark of the Pruned-CTC head-and-loss hot path (Algorithm 1, forward + backward).
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--config c4] [--impl ours|reference]
+
+A step is one complete pruned_ctc_fwd_bwd call (subset, stacking, chunked
+projection + online LSE, subset log-probs, alignment DP, chunked backward) on one
+seeded synthetic batch that stays resident in HBM.  Rank 0 prints one JSON line.
+With N > 1 (launched by torch.distributed.run) every rank works on its own batch
+of the same shape; the path has no exchange step, so there is no collective in
+the timed region (weak scaling).
+
+`--impl reference` times the float64 CPU oracle on the host cores instead, on a
+bounded sample of the same workload.
+"""
+
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import threading
+import time
+
+import numpy as np
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+sys.path.insert(0, ROOT)
+
+from paper_2609_33645_b200 import workloads as wl  # noqa: E402
+
+METRIC = "pruned_ctc_fwd_bwd_frames_per_s"
+UNIT = "frames/s"
+DEFAULT_CHUNK = 4096      # vocabulary chunk width C passed to the library
+
+
+def load_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        with open(path) as f:
+            p = json.load(f)
+        return dict(source="measured", hbm_gbs=p["hbm_gbs"], bf16_tflops=p["bf16_tflops"],
+                    bf16_tflops_sustained=p.get("bf16_tflops_sustained", p["bf16_tflops"]))
+    return dict(source="fallback", hbm_gbs=6650.0, bf16_tflops=1590.0, bf16_tflops_sustained=1400.0)
+
+
+class ClockSampler:
+    """nvidia-smi clocks and throttle reasons, sampled every 200 ms while the timed region runs."""
+
+    Q = ("index,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,"
+         "clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
+         "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, gpu_index: int):
+        self.gpu = gpu_index
+        self.proc = None
+        self.lines = []
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(
+                ["nvidia-smi", f"--query-gpu={self.Q}", "--format=csv,noheader,nounits", "-lms", "200",
+                 "-i", str(self.gpu)], stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+            self.thread = threading.Thread(target=self._read, daemon=True)
+            self.thread.start()
+        except OSError:
+            self.proc = None
+
+    def _read(self):
+        for line in self.proc.stdout:
+            self.lines.append(line.strip())
+
+    def stop(self):
+        if self.proc is None:
+            return dict(sm_mhz=None, sm_max_mhz=None, reasons=["nvidia-smi unavailable"])
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except subprocess.TimeoutExpired:
+            self.proc.kill()
+        sm, smax, power, reasons = [], [], [], set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for ln in self.lines:
+            f = [x.strip() for x in ln.split(",")]
+            if len(f) < 9:
+                continue
+            try:
+                sm.append(float(f[1]))
+                smax.append(float(f[2]))
+                power.append(float(f[3]))
+            except ValueError:
+                continue
+            for name, val in zip(names, f[5:9]):
+                if val.lower().startswith("active"):
+                    reasons.add(name)
+        # samples under load: the upper half by power draw
+        if sm:
+            order = np.argsort(power)[len(power) // 2:]
+            load_sm = [sm[i] for i in order]
+        else:
+            load_sm = []
+        return dict(sm_mhz=statistics.median(load_sm) if load_sm else None,
+                    sm_max_mhz=max(smax) if smax else None,
+                    power_w_max=max(power) if power else None,
+                    samples=len(sm), reasons=sorted(reasons))
+
+
+def oracle_sample(batch, frames: int):
+    """The first `frames` frames of utterance 0 with a proportional prefix of its labels."""
+    n = 0
+    Tn = int(batch.input_lengths[n])
+    f = min(frames, Tn)
+    u = max(1, int(batch.target_lengths[n]) * f // Tn // 2)
+    return (batch.hidden[n:n + 1, :f].astype(np.float64), batch.targets[n:n + 1, :max(u, 1)],
+            np.array([f], dtype=np.int32), np.array([u], dtype=np.int32))
+
+
+def time_oracle(batch, W64, frames: int):
+    from oracle import pruned_ctc_oracle as O
+    H, y, il, tl = oracle_sample(batch, frames)
+    t0 = time.perf_counter()
+    out = O.pruned_ctc_reference(H, W64, None, y, il, tl, batch.blank)
+    dt = time.perf_counter() - t0
+    assert np.isfinite(out["loss"]).all()
+    return dt, int(il[0])
+
+
+def blas_threads():
+    try:
+        from threadpoolctl import threadpool_info
+        return max([p.get("num_threads", 1) for p in threadpool_info()] + [1])
+    except Exception:
+        return len(os.sched_getaffinity(0))
+
+
+def run_reference(args, cfg):
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return 0
+    batch = wl.make_batch(cfg)
+    W64 = batch.W.astype(np.float64)
+    total_steps = args.steps + args.warmup
+    budget = 150.0 / max(1, total_steps)
+    dt8, _ = time_oracle(batch, W64, 8)          # calibration (also the first touch of the BLAS)
+    frames = 8
+    for cand in (16, 32, 64, 128, 256):
+        # the per-call cost is a fixed O(V D) part plus a part linear in the frames
+        if dt8 * (0.6 + 0.4 * cand / 8.0) <= budget:
+            frames = cand
+    for _ in range(args.warmup):
+        time_oracle(batch, W64, frames)
+    times = []
+    t_all = time.perf_counter()
+    for _ in range(args.steps):
+        dt, f = time_oracle(batch, W64, frames)
+        times.append(dt)
+    total = time.perf_counter() - t_all
+    value = frames * args.steps / total
+    cores = blas_threads()
+    sample = (f"oracle fwd+bwd on the first {frames} frames of utterance 0 of {cfg.name} "
+              f"(full V={cfg.V}, D={cfg.D}, full dW); W pre-widened to float64 outside the timed steps")
+    line = dict(impl="reference", metric=METRIC, value=value, unit=UNIT, n_gpus=args.gpus, steps=args.steps,
+                warmup=args.warmup, ms_per_step=1000.0 * total / args.steps, higher_is_better=True,
+                scaling="weak", vs_baseline=None, dtype="f64", data="synthetic",
+                config=dict(workload=cfg.name, N=cfg.N, D=cfg.D, V=cfg.V, sample_frames=frames),
+                cpu_baseline=dict(value=value, unit=UNIT, cores=cores, kind="oracle", sample=sample),
+                e2e=dict(value=value, unit=UNIT, h2d_bytes_per_step=0, d2h_bytes_per_step=0))
+    print(json.dumps(line), flush=True)
+    return 0
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=20)
+    ap.add_argument("--warmup", type=int, default=5)
+    ap.add_argument("--config", default="c4")
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--beam", type=float, default=0.0)
+    ap.add_argument("--chunk", type=int, default=0)
+    ap.add_argument("--e2e-steps", type=int, default=3)
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--cpu-frames", type=int, default=128)
+    args = ap.parse_args()
+    cfg = wl.CONFIGS[args.config]
+
+    if args.impl == "reference":
+        return run_reference(args, cfg)
+
+    import torch
+    from paper_2609_33645_b200 import binding, build
+
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: the hot path has no CPU implementation")
+    torch.cuda.set_device(local_rank)
+    dev = torch.device("cuda", local_rank)
+    if world > 1:
+        import torch.distributed as dist
+        dist.init_process_group("nccl", device_id=dev)
+    if rank == 0:
+        build.build()
+    if world > 1:
+        dist.barrier()
+    binding.load()
+    peaks = load_peaks()
+
+    # ---- the batch: every rank its own utterances, same shape distribution ----
+    batch = wl.make_batch(cfg, seed=cfg.seed + 7919 * rank)
+    tdt = torch.bfloat16 if cfg.dtype == "bf16" else torch.float32
+    h_hidden = torch.from_numpy(batch.hidden).to(tdt).pin_memory()
+    h_W = torch.from_numpy(batch.W).to(tdt).pin_memory()
+    h_targets = torch.from_numpy(batch.targets).pin_memory()
+    hidden = h_hidden.to(dev, non_blocking=True)
+    W = h_W.to(dev, non_blocking=True)
+    targets = h_targets.to(dev, non_blocking=True)
+    il, tl = batch.input_lengths, batch.target_lengths
+    M, D, V, N = batch.M, cfg.D, cfg.V, cfg.N
+    flops_per_step = 8.0 * M * D * V
+
+    chunk = args.chunk or DEFAULT_CHUNK
+    prob = binding.make_problem(N, batch.T, D, V, binding.PCTC_BF16 if cfg.dtype == "bf16" else binding.PCTC_FP32,
+                                batch.blank, args.beam, chunk, batch.targets.shape[1])
+    ws_bytes = binding.workspace_bytes(prob, il, tl)
+    chunk = args.chunk or DEFAULT_CHUNK
+    nchunks = (V + chunk - 1) // chunk
+    call = dict(beam=args.beam, chunk=chunk)
+
+    res = binding.pruned_ctc_fwd_bwd(hidden, W, None, targets, il, tl, batch.blank, check_status=True, **call)
+    torch.cuda.synchronize()
+    for _ in range(max(0, args.warmup - 1)):
+        res = binding.pruned_ctc_fwd_bwd(hidden, W, None, targets, il, tl, batch.blank,
+                                         workspace=res["workspace"], out=res, **call)
+    torch.cuda.synchronize()
+
+    traces = [binding.Trace(binding.Trace.capacity_for(V, chunk)) for _ in range(args.steps)]
+    sampler = ClockSampler(local_rank)
+    if rank == 0:
+        sampler.start()
+        time.sleep(0.25)
+    ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    if world > 1:
+        dist.barrier()
+    torch.cuda.synchronize()
+    ev0.record()
+    for s in range(args.steps):
+        binding.pruned_ctc_fwd_bwd(hidden, W, None, targets, il, tl, batch.blank, workspace=res["workspace"],
+                                   out=res, trace=traces[s], **call)
+    ev1.record()
+    torch.cuda.synchronize()
+    if world > 1:
+        dist.barrier()
+    clocks = sampler.stop() if rank == 0 else None
+    ms_total = ev0.elapsed_time(ev1)
+    status = binding.workspace_status(res["workspace"])
+    if status != 0:
+        raise SystemExit(f"device status word {status}: a bounded wait gave up")
+    if world > 1:
+        t = torch.tensor([ms_total], device=dev, dtype=torch.float64)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        ms_total = float(t.item())
+        mt = torch.tensor([float(M)], device=dev, dtype=torch.float64)
+        dist.all_reduce(mt, op=dist.ReduceOp.SUM)
+        frames_all = float(mt.item())
+        fl = torch.tensor([flops_per_step], device=dev, dtype=torch.float64)
+        dist.all_reduce(fl, op=dist.ReduceOp.SUM)
+        flops_all = float(fl.item())
+    else:
+        frames_all, flops_all = float(M), flops_per_step
+    ms_per_step = ms_total / args.steps
+    value = frames_all / (ms_per_step * 1e-3)
+
+    # ---- per-phase device time from the event timeline of the same timed steps ----
+    phase_ms = {name: 0.0 for name in binding.PHASES}
+    phase_cnt = {name: 0 for name in binding.PHASES}
+    for tr in traces:
+        for kind, ms in tr.spans():
+            phase_ms[binding.PHASES[kind]] += ms
+            phase_cnt[binding.PHASES[kind]] += 1
+    for k in phase_ms:
+        phase_ms[k] /= args.steps
+    gemm_phases = ("lse", "dlogits", "dh", "dw")
+    gemm_ms = sum(phase_ms[k] for k in gemm_phases)
+    gemm_launches = sum(phase_cnt[k] for k in gemm_phases) // args.steps
+    achieved_tflops = flops_per_step / (gemm_ms * 1e-3) / 1e12
+    peak = peaks["bf16_tflops_sustained"]
+    per_kernel = {}
+    split_flops = dict(lse=2.0 * M * D * V, dlogits=2.0 * M * D * V, dh=2.0 * M * D * V, dw=2.0 * M * D * V)
+    for k in gemm_phases:
+        per_kernel[k] = dict(ms=round(phase_ms[k], 4), launches=phase_cnt[k] // args.steps,
+                             tflops=round(split_flops[k] / (phase_ms[k] * 1e-3) / 1e12, 2))
+
+    # kernels launched by the library inside the timed region
+    dp_launches = 3 if args.beam > 0 else 2
+    launches_per_step = 3 + 1 + 2 + 2 + dp_launches + 3 * nchunks + 1
+    gpu_launches = launches_per_step * args.steps
+
+    # ---- end to end through the host-buffer entry point ----
+    e2e = None
+    if args.e2e_steps > 0:
+        h_res = binding.pruned_ctc_fwd_bwd_host(h_hidden, h_W, None, h_targets, il, tl, batch.blank,
+                                                device=dev, **call)
+        torch.cuda.synchronize()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+        e0.record()
+        for _ in range(args.e2e_steps):
+            binding.pruned_ctc_fwd_bwd_host(h_hidden, h_W, None, h_targets, il, tl, batch.blank,
+                                            scratch=h_res["scratch"], out=h_res, device=dev, **call)
+        e1.record()
+        torch.cuda.synchronize()
+        ms_e2e = e0.elapsed_time(e1) / args.e2e_steps
+        if world > 1:
+            t = torch.tensor([ms_e2e], device=dev, dtype=torch.float64)
+            dist.all_reduce(t, op=dist.ReduceOp.MAX)
+            ms_e2e = float(t.item())
+        h2d = h_hidden.numel() * h_hidden.element_size() + h_W.numel() * h_W.element_size() + h_targets.numel() * 4
+        d2h = (N * 4 + h_hidden.numel() * h_hidden.element_size() + h_W.numel() * h_W.element_size()
+               + (int(tl.sum()) + 1) * 4 + 4 + h_targets.numel() * 4 + N * 4)
+        e2e = dict(value=frames_all / (ms_e2e * 1e-3), unit=UNIT, ms_per_step=ms_e2e,
+                   h2d_bytes_per_step=int(h2d), d2h_bytes_per_step=int(d2h), steps=args.e2e_steps,
+                   api="pruned_ctc_fwd_bwd_host (pinned host buffers)")
+        del h_res
+    if rank != 0:
+        if world > 1:
+            dist.destroy_process_group()
+        return 0
+
+    # ---- peak head-and-loss bytes; the workspace does not depend on M*V ----
+    out_bytes = (N * 4 + hidden.numel() * hidden.element_size() + W.numel() * W.element_size())
+    prob_half = binding.make_problem(N, batch.T, D, V // 2 // 8 * 8, prob.dtype, batch.blank, args.beam, chunk,
+                                     batch.targets.shape[1])
+    ws_half = binding.workspace_bytes(prob_half, il, tl)
+
+    # ---- the oracle on the host cores, on a bounded sample ----
+    cpu = None
+    if not args.no_cpu_baseline and world == 1:
+        W64 = batch.W.astype(np.float64)
+        dt, frames = time_oracle(batch, W64, args.cpu_frames)
+        cpu = dict(value=frames / dt, unit=UNIT, cores=blas_threads(), kind="oracle", seconds=round(dt, 2),
+                   sample=(f"oracle fwd+bwd (float64, full V, full dW) on the first {frames} frames of "
+                           f"utterance 0 of {cfg.name}"))
+
+    line = dict(
+        metric=METRIC, value=value, unit=UNIT, n_gpus=world, steps=args.steps, warmup=args.warmup,
+        ms_per_step=ms_per_step, higher_is_better=True, scaling="weak", vs_baseline=None,
+        dtype=cfg.dtype, data="synthetic",
+        config=dict(workload=cfg.name, N=N, T_range=[cfg.T_lo, cfg.T_hi], D=D, V=V, M_frames=M,
+                    K_selected=int(res["K"].item()), beam=args.beam, chunk=chunk,
+                    l2="inputs larger than L2 (W and dW are %.2f GB each)" % (W.numel() * 2 / 1e9),
+                    parallelism="independent utterance batches per GPU, no collective"),
+        tflops=flops_all / (ms_per_step * 1e-3) / 1e12,
+        frac_of_bf16_peak=dict(burst=flops_all / (ms_per_step * 1e-3) / 1e12 / (peaks["bf16_tflops"] * world),
+                               sustained=flops_all / (ms_per_step * 1e-3) / 1e12 / (peak * world),
+                               peaks=peaks["source"]),
+        flops_per_step=flops_per_step,
+        phase_ms={k: round(v, 4) for k, v in phase_ms.items()},
+        roofline=dict(bound="tensor", achieved=achieved_tflops, peak=peak, unit="TFLOP/s",
+                      frac=achieved_tflops / peak, traffic=None,
+                      kernel="k_umma_gemm (all fused-epilogue instances: lse, dlogits, dh, dw)",
+                      launches_per_step=gemm_launches, ms_per_step=gemm_ms,
+                      peak_source="%s bf16_tflops_sustained (kernel timed inside a long step)" % peaks["source"],
+                      per_kernel=per_kernel),
+        peak_bytes=dict(workspace=ws_bytes, outputs=out_bytes, workspace_at_half_V=ws_half,
+                        one_fp32_MxV_array=4 * M * V),
+        e2e=e2e, gpu_launches=gpu_launches, clocks=clocks, cpu_baseline=cpu,
+    )
+    print(json.dumps(line), flush=True)
+    if world > 1:
+        dist.destroy_process_group()
+    return 0
+
+
+if __name__ == "__main__":
+    sys.exit(main())

@@ -28,7 +28,7 @@ typedef enum {
   PCTC_ERR_UNSUPPORTED = 3,         /* dtype/shape the kernels do not cover (see each function)  */
   PCTC_ERR_CUDA = 4,                /* a CUDA runtime or driver call failed (launch errors)      */
   PCTC_ERR_BAD_TARGET = 5,          /* reserved: bad targets are reported per utterance instead  */
-  PCTC_ERR_TIMEOUT = 6              /* a bounded device-side wait gave up (see pctc_last_device_status) */
+  PCTC_ERR_TIMEOUT = 6              /* a bounded device-side wait gave up (see pctc_workspace_status) */
 } pctc_status_t;
 
 typedef enum { PCTC_BF16 = 0, PCTC_FP32 = 1 } pctc_dtype_t;
@@ -118,6 +118,69 @@ pctc_status_t pruned_ctc_fwd_bwd(const pctc_problem_t* problem,
                                  int32_t* subset_out, int32_t* K_out, int32_t* relabeled_out,
                                  int32_t* utt_flags,
                                  void* workspace, size_t workspace_bytes, void* stream);
+
+/*
+ * The same call with a per-phase timeline, for measurement.  The caller creates
+ * `capacity` CUDA events (timing enabled); the call records one at the start of
+ * every phase and one at the end, on `stream`, without synchronising:
+ * events[i], events[i+1] bracket a span of phase kinds[i], for i < used-1.
+ * capacity must be at least 8 + 4 * (number of vocabulary chunks), i.e.
+ * 8 + 4 * ceil(V / chunk); otherwise PCTC_ERR_INVALID_ARG and nothing is launched.
+ * trace == NULL makes the call identical to pruned_ctc_fwd_bwd.  No counterpart
+ * in the paper (its Appendix C times whole steps with a device synchronise).
+ */
+#define PCTC_PHASE_PREP 0        /* Algorithm 1 lines 2-4: subset, relabel, frame stacking       */
+#define PCTC_PHASE_LSE 1         /* line 5: chunked projection with online log-sum-exp            */
+#define PCTC_PHASE_SUBSET_LOGP 2 /* line 6: gather W_U, S = X W_U^T + b_U - lambda                */
+#define PCTC_PHASE_DP 3          /* lines 7-10: alignment DP, losses, occupancies                 */
+#define PCTC_PHASE_DLOGITS 4     /* lines 13-14: recompute Z_c and form Eq. "vjp"                 */
+#define PCTC_PHASE_DH 5          /* line 15: dX += dZ_c W_c                                       */
+#define PCTC_PHASE_DW 6          /* line 16: dW_c = dZ_c^T X                                      */
+#define PCTC_PHASE_DBIAS 7       /* line 16: db_c = dZ_c^T 1                                      */
+#define PCTC_PHASE_FINISH 8      /* un-stacking dX into [N,T,D], integer outputs                  */
+
+typedef struct {
+  void** events;    /* HOST array of cudaEvent_t handles, [capacity]                    */
+  int32_t capacity;
+  int32_t used;     /* out: number of events recorded                                   */
+  int32_t* kinds;   /* HOST [capacity], out: kinds[i] = phase of span (events[i], events[i+1]) */
+} pctc_trace_t;
+
+pctc_status_t pruned_ctc_fwd_bwd_traced(const pctc_problem_t* problem,
+                                        const void* hidden, const void* W, const void* bias,
+                                        const int32_t* targets,
+                                        const int32_t* input_lengths, const int32_t* target_lengths,
+                                        float* loss, void* dH, void* dW, void* dbias,
+                                        int32_t* subset_out, int32_t* K_out, int32_t* relabeled_out,
+                                        int32_t* utt_flags,
+                                        void* workspace, size_t workspace_bytes, void* stream,
+                                        pctc_trace_t* trace);
+
+/*
+ * The same computation for callers whose tensors live in HOST memory (pinned
+ * memory makes the copies asynchronous).  Every data pointer of
+ * pruned_ctc_fwd_bwd is a host pointer here; `device_scratch` is one device
+ * buffer of at least pctc_host_call_scratch_bytes() bytes, 256-byte aligned,
+ * that the call carves into input staging, output staging and the workspace.
+ * Order on `stream`: host-to-device copies of hidden, W, bias, targets; Algorithm
+ * 1; device-to-host copies of loss, dH, dW, dbias and the optional integer
+ * outputs.  The call does not synchronise: the host outputs are valid once
+ * `stream` has been synchronised, and the host inputs must stay unchanged until
+ * then.  Same return codes as pruned_ctc_fwd_bwd.
+ */
+pctc_status_t pctc_host_call_scratch_bytes(const pctc_problem_t* problem,
+                                           const int32_t* input_lengths_host,
+                                           const int32_t* target_lengths_host,
+                                           int32_t has_bias, size_t* bytes_out);
+
+pctc_status_t pruned_ctc_fwd_bwd_host(const pctc_problem_t* problem,
+                                      const void* hidden, const void* W, const void* bias,
+                                      const int32_t* targets,
+                                      const int32_t* input_lengths, const int32_t* target_lengths,
+                                      float* loss, void* dH, void* dW, void* dbias,
+                                      int32_t* subset_out, int32_t* K_out, int32_t* relabeled_out,
+                                      int32_t* utt_flags,
+                                      void* device_scratch, size_t scratch_bytes, void* stream);
 
 /*
  * Contraction kernel on its own, for validation of the tensor-core path:

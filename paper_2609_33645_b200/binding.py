@@ -20,8 +20,11 @@ PCTC_BF16, PCTC_FP32 = 0, 1
 GEMM_AUTO, GEMM_SIMT = 0, 1
 UTT_INFEASIBLE, UTT_NONFINITE, UTT_BAD_TARGET = 1, 2, 4
 
-EXPORTS = ("pctc_workspace_bytes", "pruned_ctc_fwd_bwd", "pctc_gemm_bf16", "pctc_workspace_status",
-           "pctc_status_string")
+EXPORTS = ("pctc_workspace_bytes", "pruned_ctc_fwd_bwd", "pruned_ctc_fwd_bwd_traced", "pctc_gemm_bf16",
+           "pctc_workspace_status", "pctc_status_string", "pctc_host_call_scratch_bytes",
+           "pruned_ctc_fwd_bwd_host")
+
+PHASES = ("prep", "lse", "subset_logp", "dp", "dlogits", "dh", "dw", "dbias", "finish")
 
 
 class Problem(ctypes.Structure):
@@ -32,6 +35,37 @@ class Problem(ctypes.Structure):
         ("beam", ctypes.c_float),
         ("chunk", ctypes.c_int32), ("target_stride", ctypes.c_int32), ("gemm_path", ctypes.c_int32),
     ]
+
+
+class TraceStruct(ctypes.Structure):
+    _fields_ = [("events", ctypes.POINTER(ctypes.c_void_p)), ("capacity", ctypes.c_int32),
+                ("used", ctypes.c_int32), ("kinds", ctypes.POINTER(ctypes.c_int32))]
+
+
+class Trace:
+    """Caller-owned CUDA events for pruned_ctc_fwd_bwd_traced (one timeline per call)."""
+
+    def __init__(self, capacity: int):
+        import torch
+
+        self.capacity = int(capacity)
+        self.events = [torch.cuda.Event(enable_timing=True) for _ in range(self.capacity)]
+        for e in self.events:          # torch creates the CUDA event at its first record
+            e.record()
+        torch.cuda.synchronize()
+        self._handles = (ctypes.c_void_p * self.capacity)(*[int(e.cuda_event) for e in self.events])
+        self._kinds = (ctypes.c_int32 * self.capacity)()
+        self.struct = TraceStruct(ctypes.cast(self._handles, ctypes.POINTER(ctypes.c_void_p)), self.capacity, 0,
+                                  ctypes.cast(self._kinds, ctypes.POINTER(ctypes.c_int32)))
+
+    def spans(self):
+        """[(phase index, milliseconds)] of the last call; synchronise the stream first."""
+        n = self.struct.used
+        return [(int(self._kinds[i]), self.events[i].elapsed_time(self.events[i + 1])) for i in range(n - 1)]
+
+    @staticmethod
+    def capacity_for(V: int, chunk: int) -> int:
+        return 8 + 4 * ((V + chunk - 1) // chunk)
 
 
 class PctcError(RuntimeError):
@@ -58,6 +92,13 @@ def load() -> ctypes.CDLL:
     lib.pruned_ctc_fwd_bwd.restype = ctypes.c_int
     lib.pruned_ctc_fwd_bwd.argtypes = [ctypes.POINTER(Problem), vp, vp, vp, vp, i32p, i32p,
                                        vp, vp, vp, vp, vp, vp, vp, vp, vp, ctypes.c_size_t, vp]
+    lib.pruned_ctc_fwd_bwd_traced.restype = ctypes.c_int
+    lib.pruned_ctc_fwd_bwd_traced.argtypes = lib.pruned_ctc_fwd_bwd.argtypes + [ctypes.POINTER(TraceStruct)]
+    lib.pruned_ctc_fwd_bwd_host.restype = ctypes.c_int
+    lib.pruned_ctc_fwd_bwd_host.argtypes = lib.pruned_ctc_fwd_bwd.argtypes
+    lib.pctc_host_call_scratch_bytes.restype = ctypes.c_int
+    lib.pctc_host_call_scratch_bytes.argtypes = [ctypes.POINTER(Problem), i32p, i32p, ctypes.c_int32,
+                                                 ctypes.POINTER(ctypes.c_size_t)]
     lib.pctc_gemm_bf16.restype = ctypes.c_int
     lib.pctc_gemm_bf16.argtypes = [vp, vp, vp, ctypes.c_int32, ctypes.c_int32, ctypes.c_int32,
                                    ctypes.c_int32, ctypes.c_int32, ctypes.c_int32, vp, vp]
@@ -100,7 +141,8 @@ def _dptr(t) -> Optional[int]:
 
 
 def pruned_ctc_fwd_bwd(hidden, W, bias, targets, input_lengths, target_lengths, blank_id, *, beam=0.0,
-                       chunk=0, gemm_path=GEMM_AUTO, workspace=None, out=None, check_status=False):
+                       chunk=0, gemm_path=GEMM_AUTO, workspace=None, out=None, check_status=False,
+                       trace: Optional[Trace] = None):
     """Algorithm 1 on CUDA tensors.
 
     hidden [N,T,D], W [V,D], bias [V] or None (bf16 or fp32, same dtype), targets
@@ -152,11 +194,14 @@ def pruned_ctc_fwd_bwd(hidden, W, bias, targets, input_lengths, target_lengths, 
         workspace=workspace, workspace_bytes=need,
     )
     stream = ctypes.c_void_p(torch.cuda.current_stream(dev).cuda_stream)
-    st = lib.pruned_ctc_fwd_bwd(
-        ctypes.byref(prob), _dptr(hidden), _dptr(W), _dptr(bias), _dptr(targets), _ptr_i32(il), _ptr_i32(tl),
-        _dptr(res["loss"]), _dptr(res["dH"]), _dptr(res["dW"]), _dptr(res["dbias"]),
-        _dptr(res["subset"]), _dptr(res["K"]), _dptr(res["relabeled"]), _dptr(res["flags"]),
-        _dptr(workspace), ctypes.c_size_t(workspace.numel()), stream)
+    args = [ctypes.byref(prob), _dptr(hidden), _dptr(W), _dptr(bias), _dptr(targets), _ptr_i32(il), _ptr_i32(tl),
+            _dptr(res["loss"]), _dptr(res["dH"]), _dptr(res["dW"]), _dptr(res["dbias"]),
+            _dptr(res["subset"]), _dptr(res["K"]), _dptr(res["relabeled"]), _dptr(res["flags"]),
+            _dptr(workspace), ctypes.c_size_t(workspace.numel()), stream]
+    if trace is None:
+        st = lib.pruned_ctc_fwd_bwd(*args)
+    else:
+        st = lib.pruned_ctc_fwd_bwd_traced(*args, ctypes.byref(trace.struct))
     if st != 0:
         raise PctcError(st, "pruned_ctc_fwd_bwd")
     if check_status:
@@ -193,3 +238,56 @@ def gemm_bf16(A, B, m, n, k, a_mn_major=False, b_mn_major=False, gemm_path=GEMM_
     if code != 0:
         raise PctcError(6, f"device status word {code}")
     return C
+
+
+def pruned_ctc_fwd_bwd_host(hidden, W, bias, targets, input_lengths, target_lengths, blank_id, *, beam=0.0,
+                            chunk=0, gemm_path=GEMM_AUTO, scratch=None, out=None, device=None):
+    """Algorithm 1 on HOST tensors (pinned torch CPU tensors): copies in, computes, copies out.
+
+    Returns host tensors loss, dH, dW, dbias, subset, K, relabeled, flags (pinned; valid after the
+    current stream has been synchronised) plus "scratch", the reusable device buffer.
+    """
+    import torch
+
+    lib = load()
+    dev = torch.device(device or "cuda:0")
+    if hidden.is_cuda or W.is_cuda:
+        raise ValueError("the host entry point takes CPU tensors")
+    dt = PCTC_BF16 if hidden.dtype == torch.bfloat16 else PCTC_FP32
+    N, T, D = hidden.shape
+    V = W.shape[0]
+    il, tl = _i32(input_lengths), _i32(target_lengths)
+    stride = targets.shape[1]
+    prob = make_problem(N, T, D, V, dt, blank_id, beam, chunk, stride, gemm_path)
+    need = ctypes.c_size_t(0)
+    st = lib.pctc_host_call_scratch_bytes(ctypes.byref(prob), _ptr_i32(il), _ptr_i32(tl),
+                                          int(bias is not None), ctypes.byref(need))
+    if st != 0:
+        raise PctcError(st, "pctc_host_call_scratch_bytes")
+    if scratch is None or scratch.numel() < need.value:
+        scratch = torch.empty(need.value, dtype=torch.uint8, device=dev)
+    o = out or {}
+
+    def buf(name, shape, dtype):
+        t = o.get(name)
+        if t is None or tuple(t.shape) != tuple(shape) or t.dtype != dtype:
+            t = torch.empty(shape, dtype=dtype, pin_memory=True)
+        return t
+
+    res = dict(
+        loss=buf("loss", (N,), torch.float32), dH=buf("dH", (N, T, D), hidden.dtype),
+        dW=buf("dW", (V, D), hidden.dtype),
+        dbias=buf("dbias", (V,), hidden.dtype) if bias is not None else None,
+        subset=buf("subset", (int(tl.sum()) + 1,), torch.int32), K=buf("K", (1,), torch.int32),
+        relabeled=buf("relabeled", (N, stride), torch.int32), flags=buf("flags", (N,), torch.int32),
+        scratch=scratch, scratch_bytes=int(need.value),
+    )
+    stream = ctypes.c_void_p(torch.cuda.current_stream(dev).cuda_stream)
+    st = lib.pruned_ctc_fwd_bwd_host(
+        ctypes.byref(prob), _dptr(hidden), _dptr(W), _dptr(bias), _dptr(targets), _ptr_i32(il), _ptr_i32(tl),
+        _dptr(res["loss"]), _dptr(res["dH"]), _dptr(res["dW"]), _dptr(res["dbias"]),
+        _dptr(res["subset"]), _dptr(res["K"]), _dptr(res["relabeled"]), _dptr(res["flags"]),
+        _dptr(scratch), ctypes.c_size_t(scratch.numel()), stream)
+    if st != 0:
+        raise PctcError(st, "pruned_ctc_fwd_bwd_host")
+    return res

@@ -78,7 +78,7 @@ def build(verbose: bool = False, extra_flags=()) -> str:
                 if verbose and out:
                     sys.stderr.write(out)
     if jobs or not os.path.exists(LIB_PATH) or os.path.getmtime(LIB_PATH) < _newest(objs):
-        run([nvcc, "-shared", "-o", LIB_PATH, *objs, "-lcudart"])
+        run([nvcc, "-shared", "-o", LIB_PATH, *objs])   # static cudart (nvcc default)
     return LIB_PATH
 
 

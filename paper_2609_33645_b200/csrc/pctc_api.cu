@@ -179,9 +179,24 @@ pctc_status_t pruned_ctc_fwd_bwd(const pctc_problem_t* p, const void* hidden, co
                                  const int32_t* target_lengths, float* loss, void* dH, void* dW, void* dbias,
                                  int32_t* subset_out, int32_t* K_out, int32_t* relabeled_out,
                                  int32_t* utt_flags, void* workspace, size_t workspace_bytes, void* stream_v) {
+  return pruned_ctc_fwd_bwd_traced(p, hidden, W, bias, targets, input_lengths, target_lengths, loss, dH, dW, dbias,
+                                   subset_out, K_out, relabeled_out, utt_flags, workspace, workspace_bytes,
+                                   stream_v, nullptr);
+}
+
+pctc_status_t pruned_ctc_fwd_bwd_traced(const pctc_problem_t* p, const void* hidden, const void* W,
+                                        const void* bias, const int32_t* targets, const int32_t* input_lengths,
+                                        const int32_t* target_lengths, float* loss, void* dH, void* dW,
+                                        void* dbias, int32_t* subset_out, int32_t* K_out,
+                                        int32_t* relabeled_out, int32_t* utt_flags, void* workspace,
+                                        size_t workspace_bytes, void* stream_v, pctc_trace_t* trace) {
   Plan pl;
   pctc_status_t st = make_plan(p, input_lengths, target_lengths, &pl);
   if (st != PCTC_OK) return st;
+  if (trace) {
+    if (!trace->events || !trace->kinds || trace->capacity < 8 + 4 * pl.nchunks) return PCTC_ERR_INVALID_ARG;
+    trace->used = 0;
+  }
   if (!hidden || !W || !loss || !dH || !dW || !workspace) return PCTC_ERR_INVALID_ARG;
   if (!targets && pl.Usum > 0) return PCTC_ERR_INVALID_ARG;
   if (workspace_bytes < pl.total) return PCTC_ERR_WORKSPACE_TOO_SMALL;
@@ -198,7 +213,17 @@ pctc_status_t pruned_ctc_fwd_bwd(const pctc_problem_t* p, const void* hidden, co
   do {                                           \
     if ((call) != cudaSuccess) return PCTC_ERR_CUDA; \
   } while (0)
+  // start of a span of phase `kind` (kind < 0: end of the timeline)
+#define PCTC_MARK(kind)                                                                              \
+  do {                                                                                               \
+    if (trace) {                                                                                     \
+      PCTC_CUDA(cudaEventRecord((cudaEvent_t)trace->events[trace->used], stream));                   \
+      trace->kinds[trace->used] = (kind);                                                            \
+      ++trace->used;                                                                                 \
+    }                                                                                                \
+  } while (0)
 
+  PCTC_MARK(PCTC_PHASE_PREP);
   // ---- batch description: lengths, first stacked row, first trellis cell, row -> utterance ----
   std::vector<int> meta(pl.meta_ints);
   std::vector<long long> cell0(N);
@@ -268,6 +293,7 @@ pctc_status_t pruned_ctc_fwd_bwd(const pctc_problem_t* p, const void* hidden, co
   PCTC_CUDA(stack_frames(hidden, d_X, N, pl.T, D, pl.elem, bm.row_utt, bm.row0, M, stream));
 
   // ---- line 5: normaliser, online over the vocabulary ----
+  PCTC_MARK(PCTC_PHASE_LSE);
   {
     Epilogue e;
     e.kind = EPI_LSE_PARTIAL;
@@ -279,6 +305,7 @@ pctc_status_t pruned_ctc_fwd_bwd(const pctc_problem_t* p, const void* hidden, co
     PCTC_CUDA(lse_combine(d_partial, e.nsplit, M, d_lambda, stream));
   }
   // ---- line 6: log-probabilities of the selected classes ----
+  PCTC_MARK(PCTC_PHASE_SUBSET_LOGP);
   {
     PCTC_CUDA(gather_rows(W, d_WU, d_U, d_K, pl.Kcap, D, pl.elem, stream));
     Epilogue e;
@@ -293,6 +320,7 @@ pctc_status_t pruned_ctc_fwd_bwd(const pctc_problem_t* p, const void* hidden, co
     PCTC_CUDA(run_gemm(pl.use_umma, pl.bf16, c, e, d_status, stream));
   }
   // ---- lines 7-10: alignment DP, losses, occupancies ----
+  PCTC_MARK(PCTC_PHASE_DP);
   PCTC_CUDA(alignment_dp(d_S, (long long)pl.ldS, d_rel, p->target_stride, bm, N, M, pl.Lmax,
                          pl.beam ? p->beam : 0.f, dp, d_G, (long long)pl.ldS, d_K, loss, d_flags, stream));
 
@@ -301,6 +329,7 @@ pctc_status_t pruned_ctc_fwd_bwd(const pctc_problem_t* p, const void* hidden, co
     const long long v0 = (long long)ci * pl.chunk;
     const int Cc = (int)((V - v0 < pl.chunk) ? (V - v0) : pl.chunk);
     const char* Wc = (const char*)W + (size_t)v0 * D * pl.elem;
+    PCTC_MARK(PCTC_PHASE_DLOGITS);
     {
       Epilogue e;                      // recompute Z_c and form Eq. "vjp"
       e.kind = EPI_DLOGITS;
@@ -317,6 +346,7 @@ pctc_status_t pruned_ctc_fwd_bwd(const pctc_problem_t* p, const void* hidden, co
       GemmCall c{d_X, D, false, Wc, D, false, M, Cc, D};
       PCTC_CUDA(run_gemm(pl.use_umma, pl.bf16, c, e, d_status, stream));
     }
+    PCTC_MARK(PCTC_PHASE_DH);
     {
       Epilogue e;                      // dX += dZ_c W_c
       e.kind = EPI_ACCUM_F32;
@@ -326,6 +356,7 @@ pctc_status_t pruned_ctc_fwd_bwd(const pctc_problem_t* p, const void* hidden, co
       GemmCall c{d_chunk, pl.chunk, false, Wc, D, true, M, D, Cc};
       PCTC_CUDA(run_gemm(pl.use_umma, pl.bf16, c, e, d_status, stream));
     }
+    PCTC_MARK(PCTC_PHASE_DW);
     {
       Epilogue e;                      // rows of dW: dZ_c^T X
       e.kind = EPI_STORE_OUT;
@@ -335,9 +366,12 @@ pctc_status_t pruned_ctc_fwd_bwd(const pctc_problem_t* p, const void* hidden, co
       GemmCall c{d_chunk, pl.chunk, true, d_X, D, true, Cc, D, M};
       PCTC_CUDA(run_gemm(pl.use_umma, pl.bf16, c, e, d_status, stream));
     }
-    if (bias && dbias)
+    if (bias && dbias) {
+      PCTC_MARK(PCTC_PHASE_DBIAS);
       PCTC_CUDA(column_sums(d_chunk, pl.bf16, pl.chunk, M, Cc, dbias, pl.bf16, v0, stream));
+    }
   }
+  PCTC_MARK(PCTC_PHASE_FINISH);
   PCTC_CUDA(unstack_cast(d_dHacc, dH, N, pl.T, D, pl.bf16, bm.T_n, bm.row0, stream));
 
   // ---- optional integer outputs ----
@@ -348,6 +382,99 @@ pctc_status_t pruned_ctc_fwd_bwd(const pctc_problem_t* p, const void* hidden, co
     PCTC_CUDA(cudaMemcpyAsync(relabeled_out, d_rel, (size_t)N * p->target_stride * 4, cudaMemcpyDeviceToDevice,
                               stream));
   if (utt_flags) PCTC_CUDA(cudaMemcpyAsync(utt_flags, d_flags, (size_t)N * 4, cudaMemcpyDeviceToDevice, stream));
+  PCTC_MARK(-1);
+#undef PCTC_MARK
+#undef PCTC_CUDA
+  return PCTC_OK;
+}
+
+namespace {
+struct HostLayout {
+  size_t o_hidden, o_W, o_bias, o_targets, o_loss, o_dH, o_dW, o_dbias, o_subset, o_K, o_rel, o_flags, o_ws;
+  size_t b_hidden, b_W, b_bias, b_targets, b_rel, b_subset, ws_bytes, total;
+};
+pctc_status_t host_layout(const pctc_problem_t* p, const int32_t* Tn, const int32_t* Un, bool has_bias,
+                          HostLayout* h) {
+  Plan pl;
+  pctc_status_t st = make_plan(p, Tn, Un, &pl);
+  if (st != PCTC_OK) return st;
+  size_t o = 0;
+  auto take = [&](size_t bytes) { size_t r = o; o = up(o + bytes); return r; };
+  h->b_hidden = (size_t)pl.N * pl.T * pl.D * pl.elem;
+  h->b_W = (size_t)pl.V * pl.D * pl.elem;
+  h->b_bias = has_bias ? (size_t)pl.V * pl.elem : 0;
+  h->b_targets = (size_t)pl.N * p->target_stride * 4;
+  h->b_rel = h->b_targets;
+  h->b_subset = (size_t)pl.Kcap * 4;
+  h->o_hidden = take(h->b_hidden);
+  h->o_W = take(h->b_W);
+  h->o_bias = take(h->b_bias);
+  h->o_targets = take(h->b_targets);
+  h->o_loss = take((size_t)pl.N * 4);
+  h->o_dH = take(h->b_hidden);
+  h->o_dW = take(h->b_W);
+  h->o_dbias = take(h->b_bias);
+  h->o_subset = take(h->b_subset);
+  h->o_K = take(4);
+  h->o_rel = take(h->b_rel);
+  h->o_flags = take((size_t)pl.N * 4);
+  h->o_ws = take(pl.total);
+  h->ws_bytes = pl.total;
+  h->total = o;
+  return PCTC_OK;
+}
+}  // namespace
+
+pctc_status_t pctc_host_call_scratch_bytes(const pctc_problem_t* problem, const int32_t* input_lengths_host,
+                                           const int32_t* target_lengths_host, int32_t has_bias,
+                                           size_t* bytes_out) {
+  if (!bytes_out) return PCTC_ERR_INVALID_ARG;
+  HostLayout h;
+  pctc_status_t st = host_layout(problem, input_lengths_host, target_lengths_host, has_bias != 0, &h);
+  if (st != PCTC_OK) return st;
+  *bytes_out = h.total;
+  return PCTC_OK;
+}
+
+pctc_status_t pruned_ctc_fwd_bwd_host(const pctc_problem_t* p, const void* hidden, const void* W, const void* bias,
+                                      const int32_t* targets, const int32_t* input_lengths,
+                                      const int32_t* target_lengths, float* loss, void* dH, void* dW, void* dbias,
+                                      int32_t* subset_out, int32_t* K_out, int32_t* relabeled_out,
+                                      int32_t* utt_flags, void* device_scratch, size_t scratch_bytes,
+                                      void* stream_v) {
+  HostLayout h;
+  pctc_status_t st = host_layout(p, input_lengths, target_lengths, bias != nullptr, &h);
+  if (st != PCTC_OK) return st;
+  if (!hidden || !W || !loss || !dH || !dW || !device_scratch) return PCTC_ERR_INVALID_ARG;
+  if (!targets && h.b_targets > 0) return PCTC_ERR_INVALID_ARG;
+  if ((size_t)device_scratch & (ALIGN - 1)) return PCTC_ERR_INVALID_ARG;
+  if (scratch_bytes < h.total) return PCTC_ERR_WORKSPACE_TOO_SMALL;
+  cudaStream_t stream = (cudaStream_t)stream_v;
+  char* d = (char*)device_scratch;
+  const bool want_db = bias && dbias;
+#define PCTC_CUDA(call)                              \
+  do {                                               \
+    if ((call) != cudaSuccess) return PCTC_ERR_CUDA; \
+  } while (0)
+  PCTC_CUDA(cudaMemcpyAsync(d + h.o_hidden, hidden, h.b_hidden, cudaMemcpyHostToDevice, stream));
+  PCTC_CUDA(cudaMemcpyAsync(d + h.o_W, W, h.b_W, cudaMemcpyHostToDevice, stream));
+  if (bias) PCTC_CUDA(cudaMemcpyAsync(d + h.o_bias, bias, h.b_bias, cudaMemcpyHostToDevice, stream));
+  if (h.b_targets) PCTC_CUDA(cudaMemcpyAsync(d + h.o_targets, targets, h.b_targets, cudaMemcpyHostToDevice, stream));
+  st = pruned_ctc_fwd_bwd(p, d + h.o_hidden, d + h.o_W, bias ? d + h.o_bias : nullptr,
+                          (const int32_t*)(d + h.o_targets), input_lengths, target_lengths, (float*)(d + h.o_loss),
+                          d + h.o_dH, d + h.o_dW, want_db ? d + h.o_dbias : nullptr, (int32_t*)(d + h.o_subset),
+                          (int32_t*)(d + h.o_K), (int32_t*)(d + h.o_rel), (int32_t*)(d + h.o_flags), d + h.o_ws,
+                          h.ws_bytes, stream_v);
+  if (st != PCTC_OK) return st;
+  PCTC_CUDA(cudaMemcpyAsync(loss, d + h.o_loss, (size_t)p->N * 4, cudaMemcpyDeviceToHost, stream));
+  PCTC_CUDA(cudaMemcpyAsync(dH, d + h.o_dH, h.b_hidden, cudaMemcpyDeviceToHost, stream));
+  PCTC_CUDA(cudaMemcpyAsync(dW, d + h.o_dW, h.b_W, cudaMemcpyDeviceToHost, stream));
+  if (want_db) PCTC_CUDA(cudaMemcpyAsync(dbias, d + h.o_dbias, h.b_bias, cudaMemcpyDeviceToHost, stream));
+  if (subset_out) PCTC_CUDA(cudaMemcpyAsync(subset_out, d + h.o_subset, h.b_subset, cudaMemcpyDeviceToHost, stream));
+  if (K_out) PCTC_CUDA(cudaMemcpyAsync(K_out, d + h.o_K, 4, cudaMemcpyDeviceToHost, stream));
+  if (relabeled_out && h.b_rel)
+    PCTC_CUDA(cudaMemcpyAsync(relabeled_out, d + h.o_rel, h.b_rel, cudaMemcpyDeviceToHost, stream));
+  if (utt_flags) PCTC_CUDA(cudaMemcpyAsync(utt_flags, d + h.o_flags, (size_t)p->N * 4, cudaMemcpyDeviceToHost, stream));
 #undef PCTC_CUDA
   return PCTC_OK;
 }

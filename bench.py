@@ -108,6 +108,29 @@ class ClockSampler:
                     samples=len(sm), reasons=sorted(reasons))
 
 
+def rank_seed(cfg, rank: int) -> int:
+    """Every rank draws its own utterances: same configuration, different seed."""
+    return cfg.seed + 7919 * rank
+
+
+def reduce_over_ranks(ms: float, frames: float, flops: float, device=None):
+    """Whole-job figures: time is the max over ranks, frames and FLOPs are summed.
+
+    Works on any initialised process group (NCCL on the GPU machine, gloo in the CPU tests); without
+    one it returns its arguments.
+    """
+    import torch
+    import torch.distributed as dist
+
+    if not (dist.is_available() and dist.is_initialized()) or dist.get_world_size() == 1:
+        return ms, frames, flops
+    t = torch.tensor([ms], dtype=torch.float64, device=device)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    s = torch.tensor([frames, flops], dtype=torch.float64, device=device)
+    dist.all_reduce(s, op=dist.ReduceOp.SUM)
+    return float(t[0].item()), float(s[0].item()), float(s[1].item())
+
+
 def oracle_sample(batch, frames: int):
     """The first `frames` frames of utterance 0 with a proportional prefix of its labels."""
     n = 0
@@ -211,7 +234,7 @@ def main():
     peaks = load_peaks()
 
     # ---- the batch: every rank its own utterances, same shape distribution ----
-    batch = wl.make_batch(cfg, seed=cfg.seed + 7919 * rank)
+    batch = wl.make_batch(cfg, seed=rank_seed(cfg, rank))
     tdt = torch.bfloat16 if cfg.dtype == "bf16" else torch.float32
     h_hidden = torch.from_numpy(batch.hidden).to(tdt).pin_memory()
     h_W = torch.from_numpy(batch.W).to(tdt).pin_memory()
@@ -260,18 +283,7 @@ def main():
     status = binding.workspace_status(res["workspace"])
     if status != 0:
         raise SystemExit(f"device status word {status}: a bounded wait gave up")
-    if world > 1:
-        t = torch.tensor([ms_total], device=dev, dtype=torch.float64)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        ms_total = float(t.item())
-        mt = torch.tensor([float(M)], device=dev, dtype=torch.float64)
-        dist.all_reduce(mt, op=dist.ReduceOp.SUM)
-        frames_all = float(mt.item())
-        fl = torch.tensor([flops_per_step], device=dev, dtype=torch.float64)
-        dist.all_reduce(fl, op=dist.ReduceOp.SUM)
-        flops_all = float(fl.item())
-    else:
-        frames_all, flops_all = float(M), flops_per_step
+    ms_total, frames_all, flops_all = reduce_over_ranks(ms_total, float(M), flops_per_step, dev)
     ms_per_step = ms_total / args.steps
     value = frames_all / (ms_per_step * 1e-3)
 
@@ -317,10 +329,7 @@ def main():
         e1.record()
         torch.cuda.synchronize()
         ms_e2e = e0.elapsed_time(e1) / args.e2e_steps
-        if world > 1:
-            t = torch.tensor([ms_e2e], device=dev, dtype=torch.float64)
-            dist.all_reduce(t, op=dist.ReduceOp.MAX)
-            ms_e2e = float(t.item())
+        ms_e2e, _, _ = reduce_over_ranks(ms_e2e, 0.0, 0.0, dev)
         h2d = h_hidden.numel() * h_hidden.element_size() + h_W.numel() * h_W.element_size() + h_targets.numel() * 4
         d2h = (N * 4 + h_hidden.numel() * h_hidden.element_size() + h_W.numel() * h_W.element_size()
                + (int(tl.sum()) + 1) * 4 + 4 + h_targets.numel() * 4 + N * 4)

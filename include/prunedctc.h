@@ -199,6 +199,41 @@ pctc_status_t pctc_gemm_bf16(const void* A, const void* B, float* C,
                              void* stream);
 
 /*
+ * Algorithm 1 lines 2-3 on their own, for callers that cannot allocate device
+ * memory.  (The paper has no counterpart: this is a packaging of the subset and
+ * relabelling step, not another method.)
+ *
+ * Who needs it: code that runs where cudaMalloc is off the table -- inside a
+ * framework's memory-pool callback, in a process whose device memory was handed
+ * out in full at start-up, or in a latency-critical loop that must not touch the
+ * allocator -- and that only wants U, K and the relabelled targets, e.g. to size
+ * its own buffers before the main call.  pruned_ctc_fwd_bwd takes its scratch
+ * from a caller-provided workspace; this entry point needs no workspace at all:
+ * its scratch (a V-bit set, its rank table and a class-to-index map) lives in a
+ * fixed device array inside the library, PCTC_NOALLOC_MAX_V classes large
+ * (about 1.1 MB, resident on every GPU that loads the library until exit).
+ *
+ *   targets [N, target_stride] int32 (device), target_lengths [N] int32 (DEVICE
+ *   here, unlike pruned_ctc_fwd_bwd), outputs as in pruned_ctc_fwd_bwd, all
+ *   device and all required: subset_out [1 + sum U_n] (entries past K are left
+ *   untouched), K_out [1], relabeled_out [N, target_stride], utt_flags [N]
+ *   (only PCTC_UTT_BAD_TARGET can be set).
+ *
+ * V > PCTC_NOALLOC_MAX_V returns PCTC_ERR_UNSUPPORTED and launches nothing.
+ * The call makes no cudaMalloc/cudaFree and uses no allocating library routine.
+ * The first call on each device looks up the address of the scratch array
+ * (with that device current); make that first call before any stream capture.
+ * All calls share the one array: calls whose kernels overlap on the GPU (two
+ * streams, two threads) race on it.  The array keeps the previous call's
+ * contents; each call clears what it reads before use.
+ */
+#define PCTC_NOALLOC_MAX_V 262144
+pctc_status_t pctc_subset_relabel_noalloc(const int32_t* targets, const int32_t* target_lengths,
+                                          int32_t N, int32_t target_stride, int64_t V, int32_t blank_id,
+                                          int32_t* subset_out, int32_t* K_out, int32_t* relabeled_out,
+                                          int32_t* utt_flags, void* stream);
+
+/*
  * Device-side status word.  Every wait inside a kernel (on an mbarrier) is
  * bounded; a wait that gives up stores a non-zero code and the kernel returns
  * cleanly instead of hanging.  pruned_ctc_fwd_bwd keeps the word at the start of

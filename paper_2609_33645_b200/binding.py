@@ -22,7 +22,8 @@ UTT_INFEASIBLE, UTT_NONFINITE, UTT_BAD_TARGET = 1, 2, 4
 
 EXPORTS = ("pctc_workspace_bytes", "pruned_ctc_fwd_bwd", "pruned_ctc_fwd_bwd_traced", "pctc_gemm_bf16",
            "pctc_workspace_status", "pctc_status_string", "pctc_host_call_scratch_bytes",
-           "pruned_ctc_fwd_bwd_host")
+           "pruned_ctc_fwd_bwd_host", "pctc_subset_relabel_noalloc")
+NOALLOC_MAX_V = 262144
 
 PHASES = ("prep", "lse", "subset_logp", "dp", "dlogits", "dh", "dw", "dbias", "finish")
 
@@ -99,6 +100,9 @@ def load() -> ctypes.CDLL:
     lib.pctc_host_call_scratch_bytes.restype = ctypes.c_int
     lib.pctc_host_call_scratch_bytes.argtypes = [ctypes.POINTER(Problem), i32p, i32p, ctypes.c_int32,
                                                  ctypes.POINTER(ctypes.c_size_t)]
+    lib.pctc_subset_relabel_noalloc.restype = ctypes.c_int
+    lib.pctc_subset_relabel_noalloc.argtypes = [vp, vp, ctypes.c_int32, ctypes.c_int32, ctypes.c_int64,
+                                                ctypes.c_int32, vp, vp, vp, vp, vp]
     lib.pctc_gemm_bf16.restype = ctypes.c_int
     lib.pctc_gemm_bf16.argtypes = [vp, vp, vp, ctypes.c_int32, ctypes.c_int32, ctypes.c_int32,
                                    ctypes.c_int32, ctypes.c_int32, ctypes.c_int32, vp, vp]
@@ -291,3 +295,24 @@ def pruned_ctc_fwd_bwd_host(hidden, W, bias, targets, input_lengths, target_leng
     if st != 0:
         raise PctcError(st, "pruned_ctc_fwd_bwd_host")
     return res
+
+
+def subset_relabel_noalloc(targets, target_lengths, V, blank_id, out):
+    """Algorithm 1 lines 2-3 through the entry point that allocates nothing.
+
+    For callers that may not allocate device memory: every buffer, including the
+    outputs in `out` (subset, K, relabeled, flags: int32 CUDA tensors), is the
+    caller's; the library's own scratch is a fixed array inside it, so V may be
+    at most NOALLOC_MAX_V.  targets [N,stride] and target_lengths [N] are int32
+    CUDA tensors.  Runs on the current stream; returns `out`.
+    """
+    import torch
+
+    N, stride = targets.shape
+    stream = ctypes.c_void_p(torch.cuda.current_stream(targets.device).cuda_stream)
+    st = load().pctc_subset_relabel_noalloc(_dptr(targets), _dptr(target_lengths), int(N), int(stride), int(V),
+                                            int(blank_id), _dptr(out["subset"]), _dptr(out["K"]),
+                                            _dptr(out["relabeled"]), _dptr(out["flags"]), stream)
+    if st != 0:
+        raise PctcError(st, "pctc_subset_relabel_noalloc")
+    return out

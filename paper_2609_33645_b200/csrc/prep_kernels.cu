@@ -1,9 +1,12 @@
 // Integer and copy steps of Algorithm 1: batch-union subset and relabelling
 // (lines 2-3), stacking of the valid frames (line 4), the gather of the selected
 // head rows (line 6), and the small reductions around the contractions.
+#include "../../include/prunedctc.h"
 #include "pctc_internal.h"
 
 #include <math_constants.h>
+
+#include <mutex>
 
 namespace pctc {
 
@@ -219,3 +222,63 @@ cudaError_t lse_combine(const float2* partial, int nsplit, int M, float* lambda,
 }
 
 }  // namespace pctc
+
+// ---------------------------------------------------------------------------------------------
+// Subset and relabelling without any allocation: the scratch of the kernels above lives in a
+// file-scope device array instead of a caller-provided workspace.
+// ---------------------------------------------------------------------------------------------
+namespace pctc {
+namespace {
+
+constexpr long long NOALLOC_MAX_V = PCTC_NOALLOC_MAX_V;
+constexpr size_t NOALLOC_WORDS = (size_t)(NOALLOC_MAX_V / 32);
+// layout: bitmap [words] | word_rank [words] | vmap [MAX_V]
+constexpr size_t NOALLOC_BYTES = NOALLOC_WORDS * 4 * 2 + (size_t)NOALLOC_MAX_V * 4;
+
+static __device__ __align__(256) unsigned char g_noalloc_scratch[NOALLOC_BYTES];
+
+constexpr int MAX_DEVICES = 64;
+std::mutex g_noalloc_mutex;
+unsigned char* g_noalloc_ptr[MAX_DEVICES] = {};
+
+// The array's name is only a host-side handle; the device address has to be asked for, once per
+// device, while that device is current.
+cudaError_t noalloc_scratch(unsigned char** out) {
+  int dev = 0;
+  cudaError_t e = cudaGetDevice(&dev);
+  if (e != cudaSuccess) return e;
+  if (dev < 0 || dev >= MAX_DEVICES) return cudaErrorInvalidDevice;
+  std::lock_guard<std::mutex> lock(g_noalloc_mutex);
+  if (!g_noalloc_ptr[dev]) {
+    void* p = nullptr;
+    e = cudaGetSymbolAddress(&p, g_noalloc_scratch);
+    if (e != cudaSuccess) return e;
+    g_noalloc_ptr[dev] = (unsigned char*)p;
+  }
+  *out = g_noalloc_ptr[dev];
+  return cudaSuccess;
+}
+
+}  // namespace
+}  // namespace pctc
+
+extern "C" pctc_status_t pctc_subset_relabel_noalloc(const int32_t* targets, const int32_t* target_lengths,
+                                                     int32_t N, int32_t target_stride, int64_t V,
+                                                     int32_t blank_id, int32_t* subset_out, int32_t* K_out,
+                                                     int32_t* relabeled_out, int32_t* utt_flags, void* stream) {
+  using namespace pctc;
+  if (N <= 0 || target_stride < 0 || V <= 0 || blank_id < 0 || (long long)blank_id >= V) return PCTC_ERR_INVALID_ARG;
+  if (!target_lengths || !subset_out || !K_out || !utt_flags) return PCTC_ERR_INVALID_ARG;
+  if (target_stride > 0 && (!targets || !relabeled_out)) return PCTC_ERR_INVALID_ARG;
+  if (V > NOALLOC_MAX_V) return PCTC_ERR_UNSUPPORTED;      // the fixed scratch holds PCTC_NOALLOC_MAX_V classes
+  unsigned char* base = nullptr;
+  if (noalloc_scratch(&base) != cudaSuccess) return PCTC_ERR_CUDA;
+  unsigned* bitmap = (unsigned*)base;
+  int* word_rank = (int*)(base + NOALLOC_WORDS * 4);
+  int* vmap = (int*)(base + NOALLOC_WORDS * 8);
+  // subset_and_relabel clears the bitmap, the class map and the flags itself: nothing of an
+  // earlier call survives into this one.
+  cudaError_t e = subset_and_relabel(targets, target_stride, target_lengths, N, V, blank_id, bitmap, word_rank, vmap,
+                                     subset_out, K_out, relabeled_out, utt_flags, (cudaStream_t)stream);
+  return e == cudaSuccess ? PCTC_OK : PCTC_ERR_CUDA;
+}

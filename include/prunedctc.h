@@ -6,9 +6,13 @@
  * the utterance losses with respect to the head input and the head, without
  * ever holding a frames-by-vocabulary array.
  *
- * All device work is enqueued on the caller's stream.  Every buffer is owned by
- * the caller; the library keeps no pointers and no state between calls and,
- * except where an entry point says otherwise, allocates nothing.
+ * All device work is ordered after what the caller enqueued on its stream, and
+ * the stream waits for all of it (the alignment DP runs on one auxiliary stream
+ * per device that the library creates at its first call and joins back before
+ * the call's later steps).  Every buffer is owned by the caller; the library
+ * keeps no pointers between calls and, except where an entry point says
+ * otherwise, allocates no device memory.  Calls on one device must not be issued
+ * from several host threads at once.
  * Functions return a status code and never throw or abort.
  */
 #ifndef PRUNEDCTC_H_
@@ -81,9 +85,12 @@ pctc_status_t pctc_workspace_bytes(const pctc_problem_t* problem,
  *             targets relabelled by their index in U               -> subset_out, K_out, relabeled_out
  *   line 4    the M = sum T_n valid frames are stacked             (workspace)
  *   line 5    lambda_m = log sum_v exp Z[m,v], online over vocabulary chunks (Eq. "lognorm")
- *   line 6    S = X W_U^T + 1 b_U^T - lambda 1^T                   (workspace, fp32)
- *   line 7-9  per utterance: loss = -log sum over (retained) alignments; loss of an
- *             infeasible, bad-target or non-finite utterance is 0  -> loss, utt_flags
+ *   line 6    Z_U = X W_U^T + 1 b_U^T  (workspace, fp32); the shift by lambda is applied to
+ *             the loss instead of to every entry (Eq. "ctc-factorization"): occupancies do
+ *             not depend on it, and the DP can run while line 5 is still computing
+ *   line 7-9  per utterance: loss = sum_t lambda_t - log sum over (retained) alignments of
+ *             exp(sum_t Z_U); loss of an infeasible, bad-target or non-finite utterance
+ *             is 0                                                  -> loss, utt_flags
  *   line 10   occupancies gamma (G = -gamma)                       (workspace, fp32)
  *   line 11-17 per vocabulary chunk: recompute Z, dZ = w_m (exp(Z - lambda) - scatter_U(gamma))
  *             (Eq. "vjp" with unit weights; w_m = 0 on frames of excluded utterances),
@@ -123,9 +130,11 @@ pctc_status_t pruned_ctc_fwd_bwd(const pctc_problem_t* problem,
  * The same call with a per-phase timeline, for measurement.  The caller creates
  * `capacity` CUDA events (timing enabled); the call records one at the start of
  * every phase and one at the end, on `stream`, without synchronising:
- * events[i], events[i+1] bracket a span of phase kinds[i], for i < used-1.
- * capacity must be at least 8 + 4 * (number of vocabulary chunks), i.e.
- * 8 + 4 * ceil(V / chunk); otherwise PCTC_ERR_INVALID_ARG and nothing is launched.
+ * events[i], events[i+1] bracket a span of phase kinds[i], for i < used-1;
+ * spans with a negative kind are gaps between streams and carry no meaning (the
+ * alignment DP runs on an auxiliary stream, concurrently with line 5).
+ * capacity must be at least 12 + 4 * (number of vocabulary chunks), i.e.
+ * 12 + 4 * ceil(V / chunk); otherwise PCTC_ERR_INVALID_ARG and nothing is launched.
  * trace == NULL makes the call identical to pruned_ctc_fwd_bwd.  No counterpart
  * in the paper (its Appendix C times whole steps with a device synchronise).
  */

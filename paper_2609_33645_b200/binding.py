@@ -66,7 +66,7 @@ class Trace:
 
     @staticmethod
     def capacity_for(V: int, chunk: int) -> int:
-        return 8 + 4 * ((V + chunk - 1) // chunk)
+        return 12 + 4 * ((V + chunk - 1) // chunk)
 
 
 class PctcError(RuntimeError):

@@ -349,9 +349,37 @@ __global__ void k_gamma(const float* __restrict__ alpha, const float* __restrict
   if (lane == 0) { grow[0] = gb; roww[m] = 1.f; }
 }
 
+// loss_n = sum_t lambda_t - log sum over alignments of exp(sum_t Z[t, pi_t])  (Eq. "ctc-factorization")
+__global__ void k_finalize_loss(const float* __restrict__ lambda, BatchMeta meta, float* loss, int* flags,
+                                float* roww) {
+  __shared__ double s_part[8];
+  __shared__ int s_bad;
+  const int n = blockIdx.x, tid = threadIdx.x;
+  const int r0 = meta.row0[n], T = meta.T_n[n];
+  if (flags[n] != 0) return;                 // excluded: loss is already 0, row weights already 0
+  double acc = 0.0;
+  for (int t = tid; t < T; t += blockDim.x) acc += (double)lambda[r0 + t];
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) acc += __shfl_xor_sync(0xffffffffu, acc, o);
+  if ((tid & 31) == 0) s_part[tid >> 5] = acc;
+  __syncthreads();
+  if (tid == 0) {
+    double tot = 0.0;
+    for (int w = 0; w < (int)(blockDim.x >> 5); ++w) tot += s_part[w];
+    const float l = (float)((double)loss[n] + tot);
+    const bool ok = isfinite(l);
+    loss[n] = ok ? l : 0.f;
+    if (!ok) atomicOr(&flags[n], 2);
+    s_bad = ok ? 0 : 1;
+  }
+  __syncthreads();
+  if (s_bad)
+    for (int t = tid; t < T; t += blockDim.x) roww[r0 + t] = 0.f;
+}
+
 template <int W, int SPL, int MODE>
 cudaError_t launch_sweep(const SweepArgs& a, int N, cudaStream_t stream) {
-  constexpr int DEPTH = (MODE == MODE_MASKED) ? (SPL >= 8 ? 3 : 4) : (SPL >= 8 ? 4 : 8);
+  constexpr int DEPTH = (MODE == MODE_MASKED) ? (SPL >= 8 ? 3 : 4) : 4;   // small enough to share an SM with a GEMM CTA
   constexpr int NE = (SPL == 1) ? 1 : 1 + SPL / 2;
   constexpr int NX = (MODE == MODE_MASKED) ? (2 * SPL + 2) : 0;
   const size_t smem = (size_t)DEPTH * (NE + NX) * W * 32 * sizeof(float);
@@ -380,6 +408,12 @@ cudaError_t dispatch_sweep(const SweepArgs& a, int N, int Lmax, cudaStream_t s) 
 }  // namespace
 
 int dp_max_states() { return 4096; }
+
+cudaError_t finalize_loss(const float* lambda, const BatchMeta& meta, int N, float* loss, int* utt_flags,
+                          float* roww, cudaStream_t stream) {
+  k_finalize_loss<<<N, 256, 0, stream>>>(lambda, meta, loss, utt_flags, roww);
+  return cudaGetLastError();
+}
 
 cudaError_t alignment_dp(const float* S, long long ldS, const int* relabeled, int target_stride,
                          const BatchMeta& meta, int N, int M, int Lmax, float beam,

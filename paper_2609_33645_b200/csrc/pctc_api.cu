@@ -5,6 +5,7 @@
 
 #include <cmath>
 #include <cstring>
+#include <mutex>
 #include <vector>
 
 namespace {
@@ -27,7 +28,7 @@ struct Plan {
   size_t meta_ints;  // T_n[N] | U_n[N] | row0[N+1] | row_utt[M]
 };
 
-int default_chunk(bool /*bf16*/) { return 4096; }
+int default_chunk(bool bf16) { return bf16 ? 8192 : 4096; }
 
 pctc_status_t make_plan(const pctc_problem_t* p, const int32_t* Tn, const int32_t* Un, Plan* pl) {
   if (!p || !Tn || !Un) return PCTC_ERR_INVALID_ARG;
@@ -100,6 +101,30 @@ pctc_status_t make_plan(const pctc_problem_t* p, const int32_t* Tn, const int32_
   pl->o_dHacc = take((size_t)pl->M * pl->D * 4);
   pl->total = o;
   return PCTC_OK;
+}
+
+// One auxiliary stream and a fork/join event pair per device, created at the first call on that
+// device and kept until exit.  Calls on one device are therefore not re-entrant across host threads.
+struct Aux {
+  cudaStream_t side = nullptr;
+  cudaEvent_t fork = nullptr, join = nullptr;
+};
+cudaError_t get_aux(Aux* out) {
+  static std::mutex mu;
+  static Aux table[64];
+  int dev = 0;
+  cudaError_t e = cudaGetDevice(&dev);
+  if (e != cudaSuccess) return e;
+  if (dev < 0 || dev >= 64) return cudaErrorInvalidDevice;
+  std::lock_guard<std::mutex> lock(mu);
+  Aux& a = table[dev];
+  if (!a.side) {
+    if ((e = cudaStreamCreateWithFlags(&a.side, cudaStreamNonBlocking)) != cudaSuccess) return e;
+    if ((e = cudaEventCreateWithFlags(&a.fork, cudaEventDisableTiming)) != cudaSuccess) return e;
+    if ((e = cudaEventCreateWithFlags(&a.join, cudaEventDisableTiming)) != cudaSuccess) return e;
+  }
+  *out = a;
+  return cudaSuccess;
 }
 
 struct GemmCall {
@@ -194,7 +219,7 @@ pctc_status_t pruned_ctc_fwd_bwd_traced(const pctc_problem_t* p, const void* hid
   pctc_status_t st = make_plan(p, input_lengths, target_lengths, &pl);
   if (st != PCTC_OK) return st;
   if (trace) {
-    if (!trace->events || !trace->kinds || trace->capacity < 8 + 4 * pl.nchunks) return PCTC_ERR_INVALID_ARG;
+    if (!trace->events || !trace->kinds || trace->capacity < 12 + 4 * pl.nchunks) return PCTC_ERR_INVALID_ARG;
     trace->used = 0;
   }
   if (!hidden || !W || !loss || !dH || !dW || !workspace) return PCTC_ERR_INVALID_ARG;
@@ -205,6 +230,8 @@ pctc_status_t pruned_ctc_fwd_bwd_traced(const pctc_problem_t* p, const void* hid
     return PCTC_ERR_INVALID_ARG;
   if (pl.use_umma && !umma_available()) return PCTC_ERR_CUDA;
   cudaStream_t stream = (cudaStream_t)stream_v;
+  Aux aux;
+  if (get_aux(&aux) != cudaSuccess) return PCTC_ERR_CUDA;
   char* ws = (char*)workspace;
   const int N = pl.N, M = pl.M, D = pl.D;
   const long long V = pl.V;
@@ -292,7 +319,39 @@ pctc_status_t pruned_ctc_fwd_bwd_traced(const pctc_problem_t* p, const void* hid
   // ---- line 4: stack the valid frames ----
   PCTC_CUDA(stack_frames(hidden, d_X, N, pl.T, D, pl.elem, bm.row_utt, bm.row0, M, stream));
 
-  // ---- line 5: normaliser, online over the vocabulary ----
+  // ---- line 6 first: logits of the selected classes, Z_U = X W_U^T + b_U ----
+  // The alignment sum of Eq. "ctc-factorization" needs no normaliser, so the DP runs on Z_U while
+  // the full-vocabulary normaliser is still being computed; lambda enters the loss at the end.
+  PCTC_MARK(PCTC_PHASE_SUBSET_LOGP);
+  {
+    PCTC_CUDA(gather_rows(W, d_WU, d_U, d_K, pl.Kcap, D, pl.elem, stream));
+    Epilogue e;
+    e.kind = EPI_SUBSET_LOGP;
+    e.out = d_S;
+    e.ld = (long long)pl.ldS;
+    e.lambda = nullptr;
+    e.bias = bias;
+    e.U = d_U;
+    e.Kdev = d_K;
+    GemmCall c{d_X, D, false, d_WU, D, false, M, pl.Kcap, D};
+    PCTC_CUDA(run_gemm(pl.use_umma, pl.bf16, c, e, d_status, stream));
+  }
+  // ---- lines 7-10 on the auxiliary stream: alignment DP, occupancies ----
+  PCTC_MARK(-2);
+  PCTC_CUDA(cudaEventRecord(aux.fork, stream));
+  PCTC_CUDA(cudaStreamWaitEvent(aux.side, aux.fork, 0));
+  {
+    cudaStream_t main_stream = stream;
+    stream = aux.side;
+    PCTC_MARK(PCTC_PHASE_DP);
+    PCTC_CUDA(alignment_dp(d_S, (long long)pl.ldS, d_rel, p->target_stride, bm, N, M, pl.Lmax,
+                           pl.beam ? p->beam : 0.f, dp, d_G, (long long)pl.ldS, d_K, loss, d_flags, stream));
+    PCTC_MARK(-2);
+    stream = main_stream;
+  }
+  PCTC_CUDA(cudaEventRecord(aux.join, aux.side));
+
+  // ---- line 5: normaliser, online over the vocabulary (concurrent with the DP) ----
   PCTC_MARK(PCTC_PHASE_LSE);
   {
     Epilogue e;
@@ -304,25 +363,8 @@ pctc_status_t pruned_ctc_fwd_bwd_traced(const pctc_problem_t* p, const void* hid
     PCTC_CUDA(run_gemm(pl.use_umma, pl.bf16, c, e, d_status, stream));
     PCTC_CUDA(lse_combine(d_partial, e.nsplit, M, d_lambda, stream));
   }
-  // ---- line 6: log-probabilities of the selected classes ----
-  PCTC_MARK(PCTC_PHASE_SUBSET_LOGP);
-  {
-    PCTC_CUDA(gather_rows(W, d_WU, d_U, d_K, pl.Kcap, D, pl.elem, stream));
-    Epilogue e;
-    e.kind = EPI_SUBSET_LOGP;
-    e.out = d_S;
-    e.ld = (long long)pl.ldS;
-    e.lambda = d_lambda;
-    e.bias = bias;
-    e.U = d_U;
-    e.Kdev = d_K;
-    GemmCall c{d_X, D, false, d_WU, D, false, M, pl.Kcap, D};
-    PCTC_CUDA(run_gemm(pl.use_umma, pl.bf16, c, e, d_status, stream));
-  }
-  // ---- lines 7-10: alignment DP, losses, occupancies ----
-  PCTC_MARK(PCTC_PHASE_DP);
-  PCTC_CUDA(alignment_dp(d_S, (long long)pl.ldS, d_rel, p->target_stride, bm, N, M, pl.Lmax,
-                         pl.beam ? p->beam : 0.f, dp, d_G, (long long)pl.ldS, d_K, loss, d_flags, stream));
+  PCTC_CUDA(cudaStreamWaitEvent(stream, aux.join, 0));
+  PCTC_CUDA(finalize_loss(d_lambda, bm, N, loss, d_flags, dp.roww, stream));
 
   // ---- lines 11-17: backward, one vocabulary chunk at a time ----
   for (int ci = 0; ci < pl.nchunks; ++ci) {

@@ -16,7 +16,7 @@ namespace pctc {
 enum EpiKind : int {
   EPI_STORE_F32 = 0,    // C[i*ld + j] = acc                                  (validation GEMM)
   EPI_LSE_PARTIAL = 1,  // running (max, sum exp) of z = acc + bias[j] over a column range
-  EPI_SUBSET_LOGP = 2,  // S[i*ld + j] = acc + bias[U[j]] - lambda[i],  j < K  (Algorithm 1 line 6)
+  EPI_SUBSET_LOGP = 2,  // S[i*ld + j] = acc + bias[U[j]] - lambda[i],  j < K  (Algorithm 1 line 6); lambda null: no shift
   EPI_DLOGITS = 3,      // chunk[i*ld + j] = w_i (exp(acc + bias[v0+j] - lambda[i]) - gamma[i, vmap[v0+j]])
   EPI_ACCUM_F32 = 4,    // acc_out[i*ld + j] (+)= acc                          (dH across chunks)
   EPI_STORE_OUT = 5     // out[i*ld + j] = T(acc)                              (rows of dW)
@@ -119,5 +119,11 @@ cudaError_t alignment_dp(const float* S, long long ldS, const int* relabeled, in
                          const BatchMeta& meta, int N, int M, int Lmax, float beam,
                          const DpBuffers& buf, float* gamma, long long ld_gamma, const int* Kdev,
                          float* loss, int* utt_flags, cudaStream_t stream);
+
+// loss[n] += sum of lambda over the frames of utterance n (Eq. "ctc-factorization"): the DP ran on
+// unnormalised selected logits.  Utterances already excluded keep loss 0; a non-finite result
+// flags the utterance, zeroes its loss and its row weights.
+cudaError_t finalize_loss(const float* lambda, const BatchMeta& meta, int N, float* loss, int* utt_flags,
+                          float* roww, cudaStream_t stream);
 
 }  // namespace pctc

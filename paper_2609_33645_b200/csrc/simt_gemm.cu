@@ -88,7 +88,7 @@ __global__ void __launch_bounds__(NT) k_simt_gemm(const T* __restrict__ A, const
       const int i = i0 + ty * 4 + r;
       if (i >= g.m) continue;
       float lam = 0.f, w = 0.f;
-      if (EPI == EPI_SUBSET_LOGP || EPI == EPI_DLOGITS) lam = e.lambda[i];
+      if (EPI == EPI_DLOGITS || (EPI == EPI_SUBSET_LOGP && e.lambda)) lam = e.lambda[i];
       if (EPI == EPI_DLOGITS) w = e.roww[i];
 #pragma unroll
       for (int c = 0; c < 4; ++c) {

@@ -313,7 +313,7 @@ k_umma_gemm(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
       const int i = mt * BM + r;
       const bool row_ok = i < a.m;
       float lam2 = 0.f, lam = 0.f, w = 0.f;
-      if ((EPI == EPI_SUBSET_LOGP || EPI == EPI_DLOGITS) && row_ok) { lam = a.e.lambda[i]; lam2 = lam * LOG2E; }
+      if ((EPI == EPI_DLOGITS || (EPI == EPI_SUBSET_LOGP && a.e.lambda)) && row_ok) { lam = a.e.lambda[i]; lam2 = lam * LOG2E; }
       if (EPI == EPI_DLOGITS && row_ok) w = a.e.roww[i];
       float run_max2 = -CUDART_INF_F, run_sum = 0.f;     // EPI_LSE_PARTIAL, base-2 domain
 

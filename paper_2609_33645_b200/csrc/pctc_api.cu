@@ -17,13 +17,13 @@ inline size_t up(size_t x, size_t a = ALIGN) { return (x + a - 1) / a * a; }
 
 struct Plan {
   int N, T, D, M, Usum, Kcap, Lmax, chunk, nsplit, nchunks;
-  long long V, cells;
+  long long V, cells, mcells;
   size_t ldS;
   int elem;          // bytes per element of hidden/W
   bool bf16, use_umma, beam;
   // byte offsets into the workspace
   size_t o_status, o_meta_i, o_cell0, o_bitmap, o_wrank, o_vmap, o_U, o_K, o_rel, o_flags, o_X, o_lambda,
-      o_partial, o_WU, o_S, o_G, o_roww, o_alpha, o_beta, o_va, o_vb, o_offa, o_offb, o_best, o_chunk, o_dHacc;
+      o_partial, o_WU, o_S, o_G, o_roww, o_alpha, o_beta, o_va, o_vb, o_offa, o_offb, o_best, o_maskf, o_maskb, o_mcell0, o_chunk, o_dHacc;
   size_t total;
   size_t meta_ints;  // T_n[N] | U_n[N] | row0[N+1] | row_utt[M]
 };
@@ -39,7 +39,7 @@ pctc_status_t make_plan(const pctc_problem_t* p, const int32_t* Tn, const int32_
   if (p->gemm_path != PCTC_GEMM_AUTO && p->gemm_path != PCTC_GEMM_SIMT) return PCTC_ERR_INVALID_ARG;
   if (p->chunk < 0) return PCTC_ERR_INVALID_ARG;
   if (std::isnan(p->beam)) return PCTC_ERR_INVALID_ARG;
-  long long M = 0, Usum = 0, cells = 0;
+  long long M = 0, Usum = 0, cells = 0, mcells = 0;
   int Umax = 0;
   for (int n = 0; n < p->N; ++n) {
     if (Tn[n] < 1 || Tn[n] > p->T) return PCTC_ERR_INVALID_ARG;
@@ -47,11 +47,12 @@ pctc_status_t make_plan(const pctc_problem_t* p, const int32_t* Tn, const int32_
     M += Tn[n];
     Usum += Un[n];
     cells += (long long)Tn[n] * (2LL * Un[n] + 1);
+    mcells += (long long)Tn[n] * ((2LL * Un[n] + 1 + 3) / 4 * 4);
     if (Un[n] > Umax) Umax = Un[n];
   }
   if (M > 0x7fffffffLL / 2 || Usum > 0x3fffffffLL) return PCTC_ERR_UNSUPPORTED;
   pl->N = p->N; pl->T = p->T; pl->D = p->D; pl->V = p->V;
-  pl->M = (int)M; pl->Usum = (int)Usum; pl->Kcap = (int)Usum + 1; pl->cells = cells;
+  pl->M = (int)M; pl->Usum = (int)Usum; pl->Kcap = (int)Usum + 1; pl->cells = cells; pl->mcells = mcells;
   pl->Lmax = 2 * Umax + 1;
   if (pl->Lmax > dp_max_states()) return PCTC_ERR_UNSUPPORTED;
   pl->bf16 = (p->dtype == PCTC_BF16);
@@ -89,13 +90,16 @@ pctc_status_t make_plan(const pctc_problem_t* p, const int32_t* Tn, const int32_
   pl->o_roww = take((size_t)pl->M * 4);
   pl->o_alpha = take((size_t)cells * 4);
   pl->o_beta = take((size_t)cells * 4);
-  pl->o_va = pl->o_vb = pl->o_offa = pl->o_offb = pl->o_best = 0;
+  pl->o_va = pl->o_vb = pl->o_offa = pl->o_offb = pl->o_best = pl->o_maskf = pl->o_maskb = pl->o_mcell0 = 0;
   if (pl->beam) {
     pl->o_va = take((size_t)cells * 4);
     pl->o_vb = take((size_t)cells * 4);
     pl->o_offa = take((size_t)pl->M * 8);
     pl->o_offb = take((size_t)pl->M * 8);
     pl->o_best = take((size_t)pl->N * 8);
+    pl->o_maskf = take((size_t)mcells);
+    pl->o_maskb = take((size_t)mcells);
+    pl->o_mcell0 = take((size_t)pl->N * 8);
   }
   pl->o_chunk = take((size_t)pl->M * pl->chunk * pl->elem);
   pl->o_dHacc = take((size_t)pl->M * pl->D * 4);
@@ -253,19 +257,21 @@ pctc_status_t pruned_ctc_fwd_bwd_traced(const pctc_problem_t* p, const void* hid
   PCTC_MARK(PCTC_PHASE_PREP);
   // ---- batch description: lengths, first stacked row, first trellis cell, row -> utterance ----
   std::vector<int> meta(pl.meta_ints);
-  std::vector<long long> cell0(N);
+  std::vector<long long> cell0(N), mcell0(N);
   {
     int* Tn = meta.data();
     int* Un = Tn + N;
     int* row0 = Un + N;
     int* row_utt = row0 + N + 1;
-    long long cells = 0;
+    long long cells = 0, mcells = 0;
     int r = 0;
     for (int n = 0; n < N; ++n) {
       Tn[n] = input_lengths[n];
       Un[n] = target_lengths[n];
       row0[n] = r;
       cell0[n] = cells;
+      mcell0[n] = mcells;
+      mcells += (long long)Tn[n] * ((2LL * Un[n] + 1 + 3) / 4 * 4);
       for (int t = 0; t < Tn[n]; ++t) row_utt[r + t] = n;
       r += Tn[n];
       cells += (long long)Tn[n] * (2LL * Un[n] + 1);
@@ -276,6 +282,8 @@ pctc_status_t pruned_ctc_fwd_bwd_traced(const pctc_problem_t* p, const void* hid
   long long* d_cell0 = (long long*)(ws + pl.o_cell0);
   PCTC_CUDA(cudaMemcpyAsync(d_meta, meta.data(), pl.meta_ints * 4, cudaMemcpyHostToDevice, stream));
   PCTC_CUDA(cudaMemcpyAsync(d_cell0, cell0.data(), (size_t)N * 8, cudaMemcpyHostToDevice, stream));
+  if (pl.beam)
+    PCTC_CUDA(cudaMemcpyAsync(ws + pl.o_mcell0, mcell0.data(), (size_t)N * 8, cudaMemcpyHostToDevice, stream));
   PCTC_CUDA(cudaMemsetAsync(ws + pl.o_status, 0, 256, stream));
   BatchMeta bm;
   bm.T_n = d_meta;
@@ -310,6 +318,9 @@ pctc_status_t pruned_ctc_fwd_bwd_traced(const pctc_problem_t* p, const void* hid
     dp.off_a = (double*)(ws + pl.o_offa);
     dp.off_b = (double*)(ws + pl.o_offb);
     dp.best = (double*)(ws + pl.o_best);
+    dp.mask_f = (unsigned char*)(ws + pl.o_maskf);
+    dp.mask_b = (unsigned char*)(ws + pl.o_maskb);
+    dp.mcell0 = (const long long*)(ws + pl.o_mcell0);
   }
 
   // ---- Algorithm 1 lines 2-3: subset and relabelling ----

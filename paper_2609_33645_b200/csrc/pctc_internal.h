@@ -109,6 +109,9 @@ struct DpBuffers {
   double* off_a;       // [M] per-frame offsets of va   (beam only)
   double* off_b;       // [M]
   double* best;        // [N] best alignment score (beam only)
+  unsigned char* mask_f;      // [sum T_n * roundup4(L_n)] arc flags, forward sweep coordinates (beam only)
+  unsigned char* mask_b;      // same, backward sweep coordinates
+  const long long* mcell0;    // [N] first flag byte of each utterance
   float* roww;         // [M]
 };
 

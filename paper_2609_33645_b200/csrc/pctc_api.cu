@@ -50,7 +50,7 @@ pctc_status_t make_plan(const pctc_problem_t* p, const int32_t* Tn, const int32_
     mcells += (long long)Tn[n] * ((2LL * Un[n] + 1 + 3) / 4 * 4);
     if (Un[n] > Umax) Umax = Un[n];
   }
-  if (M > 0x7fffffffLL / 2 || Usum > 0x3fffffffLL) return PCTC_ERR_UNSUPPORTED;
+  if (M > 0x7fffffffLL / 2 || Usum >= (1LL << 23) - 1) return PCTC_ERR_UNSUPPORTED;   // index in U packs into 23 bits
   pl->N = p->N; pl->T = p->T; pl->D = p->D; pl->V = p->V;
   pl->M = (int)M; pl->Usum = (int)Usum; pl->Kcap = (int)Usum + 1; pl->cells = cells; pl->mcells = mcells;
   pl->Lmax = 2 * Umax + 1;

@@ -25,6 +25,17 @@ namespace pctc {
 
 namespace {
 
+// Tunables (overridable at compile time for experiments)
+#ifndef PCTC_DBG_SKIP_STORE
+#define PCTC_DBG_SKIP_STORE 0     // timing experiments only: drop the epilogue's global stores
+#endif
+#ifndef PCTC_DBG_SKIP_MATH
+#define PCTC_DBG_SKIP_MATH 0      // timing experiments only: drop the exponentials of the dlogits epilogue
+#endif
+#ifndef PCTC_TUNE_N_FASTEST
+#define PCTC_TUNE_N_FASTEST 1     // dX / dW kernels walk column tiles first
+#endif
+
 constexpr int BM = 128, BN = 256, BK = 64, STAGES = 4;
 constexpr int A_STAGE_BYTES = BM * BK * 2;
 constexpr int B_STAGE_BYTES = BN * BK * 2;
@@ -39,11 +50,12 @@ struct UmmaArgs {
   int m, n, k;
   int a_mn, b_mn;
   int nsplit;          // EPI_LSE_PARTIAL: column splits per row tile
+  int n_fastest;       // tile order: consecutive CTAs walk the column tiles of one row tile first
   int* status;
   Epilogue e;
 };
 
-struct SharedTail {   // after the operand ring
+struct SharedTail {   // barriers and flags
   unsigned long long full[STAGES];
   unsigned long long empty[STAGES];
   unsigned long long tmem_full[2];
@@ -51,11 +63,23 @@ struct SharedTail {   // after the operand ring
   unsigned long long done;
   unsigned tmem_base;
   int abort;
-  float bias[4][BN];       // per epilogue warp: bias of the tile's columns
-  int2 list[4][BN];        // per epilogue warp: (column, index in U) of the selected classes
 };
 
-constexpr size_t SMEM_BYTES = 1024 + (size_t)STAGES * (A_STAGE_BYTES + B_STAGE_BYTES) + sizeof(SharedTail);
+// Dynamic shared memory after the operand ring, by epilogue kind:
+//   store staging  4 warps x 4 KB, 128-byte-swizzled boxes for the TMA stores (dlogits, dX, dW)
+//   SharedTail
+//   bias           4 warps x BN floats (lse, subset, dlogits)
+//   list           4 warps x BN packed (index in U << 8 | column) of the tile's selected classes (dlogits)
+constexpr int STAGE_BOX_BYTES = 4096;
+constexpr bool epi_uses_tma_store(int epi) { return epi == EPI_DLOGITS || epi == EPI_ACCUM_F32 || epi == EPI_STORE_OUT; }
+constexpr bool epi_uses_bias(int epi) { return epi == EPI_LSE_PARTIAL || epi == EPI_SUBSET_LOGP || epi == EPI_DLOGITS; }
+constexpr size_t RING_BYTES = (size_t)STAGES * (A_STAGE_BYTES + B_STAGE_BYTES);
+constexpr size_t off_stage() { return RING_BYTES; }
+constexpr size_t off_tail(int epi) { return RING_BYTES + (epi_uses_tma_store(epi) ? 4 * STAGE_BOX_BYTES : 0); }
+constexpr size_t off_bias(int epi) { return off_tail(epi) + 128; }
+constexpr size_t off_list(int epi) { return off_bias(epi) + (epi_uses_bias(epi) ? 4 * BN * 4 : 0); }
+constexpr size_t smem_bytes(int epi) { return 1024 + off_list(epi) + (epi == EPI_DLOGITS ? 4 * BN * 4 : 0); }
+static_assert(sizeof(SharedTail) <= 128, "tail layout");
 
 // ---------------------------------------------------------------------------------------------
 // PTX wrappers
@@ -107,6 +131,22 @@ __device__ __forceinline__ void tma_load_2d(void* smem_dst, const CUtensorMap* m
       ::"r"(smem_u32(smem_dst)), "l"(map), "r"(c0), "r"(c1), "r"(smem_u32(bar))
       : "memory");
 }
+
+// Store (or fp32 add-reduce) of one staged box; the tensor map clips rows and columns past the extents.
+__device__ __forceinline__ void tma_store_2d(const CUtensorMap* map, const void* smem_src, int c0, int c1) {
+  asm volatile("cp.async.bulk.tensor.2d.global.shared::cta.tile.bulk_group [%0, {%1, %2}], [%3];"
+               ::"l"(map), "r"(c0), "r"(c1), "r"(smem_u32(smem_src))
+               : "memory");
+}
+__device__ __forceinline__ void tma_reduce_add_2d(const CUtensorMap* map, const void* smem_src, int c0, int c1) {
+  asm volatile("cp.reduce.async.bulk.tensor.2d.global.shared::cta.add.tile.bulk_group [%0, {%1, %2}], [%3];"
+               ::"l"(map), "r"(c0), "r"(c1), "r"(smem_u32(smem_src))
+               : "memory");
+}
+__device__ __forceinline__ void bulk_commit() { asm volatile("cp.async.bulk.commit_group;" ::: "memory"); }
+__device__ __forceinline__ void bulk_wait_read0() { asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory"); }
+__device__ __forceinline__ void bulk_wait0() { asm volatile("cp.async.bulk.wait_group 0;" ::: "memory"); }
+__device__ __forceinline__ void fence_async_smem() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
 
 __device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
 __device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
@@ -176,17 +216,28 @@ __device__ __forceinline__ void split_range(int n_tiles, int splits, int sp, int
   start = sp * base + min(sp, rem);
 }
 
+// Unit u -> (row tile, first column tile, number of column tiles).  The order decides which operand
+// streams through L2 once and which stays resident while a wave of CTAs runs: row tile fastest
+// keeps A (all row tiles) resident and streams B; column tile fastest does the opposite.
+__device__ __forceinline__ void decode_unit(int u, int m_tiles, int n_tiles, int splits, bool n_fastest,
+                                            int& mt, int& sp, int& nt0, int& cnt) {
+  if (n_fastest) { sp = u % splits; mt = u / splits; }
+  else { mt = u % m_tiles; sp = u / m_tiles; }
+  split_range(n_tiles, splits, sp, nt0, cnt);
+}
+
 // ---------------------------------------------------------------------------------------------
 // The kernel
 // ---------------------------------------------------------------------------------------------
 template <int EPI>
 __global__ void __launch_bounds__(NUM_THREADS, 1)
-k_umma_gemm(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB, UmmaArgs a) {
+k_umma_gemm(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
+            const __grid_constant__ CUtensorMap tmC, UmmaArgs a) {
   extern __shared__ unsigned char smem_raw[];
   unsigned char* smem = (unsigned char*)(((size_t)smem_raw + 1023) & ~(size_t)1023);
   unsigned char* sA = smem;
   unsigned char* sB = smem + (size_t)STAGES * A_STAGE_BYTES;
-  SharedTail* st = (SharedTail*)(smem + (size_t)STAGES * (A_STAGE_BYTES + B_STAGE_BYTES));
+  SharedTail* st = (SharedTail*)(smem + off_tail(EPI));
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
 
@@ -225,9 +276,8 @@ k_umma_gemm(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
       unsigned g = 0;
       bool ok = true;
       for (int u = blockIdx.x; u < units && ok; u += gridDim.x) {
-        const int mt = u % m_tiles, sp = u / m_tiles;
-        int nt0, cnt;
-        split_range(n_tiles, splits, sp, nt0, cnt);
+        int mt, sp, nt0, cnt;
+        decode_unit(u, m_tiles, n_tiles, splits, a.n_fastest != 0, mt, sp, nt0, cnt);
         for (int nt = nt0; nt < nt0 + cnt && ok; ++nt) {
           for (int kb = 0; kb < k_blocks; ++kb, ++g) {
             const int s = g % STAGES;
@@ -269,9 +319,9 @@ k_umma_gemm(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
       unsigned g = 0, it = 0;
       bool ok = true;
       for (int u = blockIdx.x; u < units && ok; u += gridDim.x) {
-        const int sp = u / m_tiles;
-        int nt0, cnt;
-        split_range(n_tiles, splits, sp, nt0, cnt);
+        int mt, sp, nt0, cnt;
+        decode_unit(u, m_tiles, n_tiles, splits, a.n_fastest != 0, mt, sp, nt0, cnt);
+        (void)mt;
         for (int nt = nt0; nt < nt0 + cnt && ok; ++nt, ++it) {
           const unsigned acc = it & 1u, aph = (it >> 1) & 1u;
           if (!mbar_wait(&st->tmem_empty[acc], aph ^ 1u, abort_flag, a.status, 2)) { ok = false; break; }
@@ -302,14 +352,15 @@ k_umma_gemm(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
     const int ew = warp - 2;                 // private staging slot
     const int q = warp & 3;                  // tensor-memory lane quarter this warp may read
     const int r = q * 32 + lane;             // accumulator row of this thread
-    float* sb = st->bias[ew];
-    int2* sl = st->list[ew];
+    float* sb = (float*)(smem + off_bias(EPI)) + ew * BN;
+    unsigned* sl = (unsigned*)(smem + off_list(EPI)) + ew * BN;
+    unsigned char* stage = smem + off_stage() + ew * STAGE_BOX_BYTES;   // this warp's store staging box
+    const unsigned swz = (unsigned)(lane & 7);                           // 128-byte swizzle of the staged row
     unsigned it = 0;
     bool ok = true;
     for (int u = blockIdx.x; u < units && ok; u += gridDim.x) {
-      const int mt = u % m_tiles, sp = u / m_tiles;
-      int nt0, cnt;
-      split_range(n_tiles, splits, sp, nt0, cnt);
+      int mt, sp, nt0, cnt;
+      decode_unit(u, m_tiles, n_tiles, splits, a.n_fastest != 0, mt, sp, nt0, cnt);
       const int i = mt * BM + r;
       const bool row_ok = i < a.m;
       float lam2 = 0.f, lam = 0.f, w = 0.f;
@@ -340,7 +391,7 @@ k_umma_gemm(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
             const int j = n0 + c0 + lane;
             const int jj = (j < n_eff) ? a.e.vmap[a.e.v0 + j] : -1;
             const unsigned mask = __ballot_sync(0xffffffffu, jj >= 0);
-            if (jj >= 0) sl[nsel + __popc(mask & ((1u << lane) - 1u))] = make_int2(c0 + lane, jj);
+            if (jj >= 0) sl[nsel + __popc(mask & ((1u << lane) - 1u))] = ((unsigned)jj << 8) | (unsigned)(c0 + lane);
             nsel += __popc(mask);
           }
         }
@@ -353,8 +404,75 @@ k_umma_gemm(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
         tc_fence_after();
         const unsigned taddr = tmem_base + ((unsigned)(q * 32) << 16) + acc * BN;
 
+        if (epi_uses_tma_store(EPI)) {
+          // ---- staged epilogues: the warp's 32 rows go out as 128-byte-wide boxes through TMA ----
+          constexpr int BOX_COLS = (EPI == EPI_ACCUM_F32) ? 32 : 64;   // fp32 : bf16
+          int e_idx = 0;
 #pragma unroll 1
-        for (int cg = 0; cg < BN / 32; ++cg) {
+          for (int cb = 0; cb < BN / BOX_COLS; ++cb) {
+            const int j0 = n0 + cb * BOX_COLS;
+            if (j0 >= n_eff) break;                   // warp-uniform
+            if (lane == 0) bulk_wait_read0();          // the previous box has been read out of the staging buffer
+            __syncwarp();
+            unsigned char* row = stage + lane * 128;
+            if (EPI == EPI_ACCUM_F32) {
+              float v[32];
+              tmem_ld32(taddr + cb * 32, v);
+#pragma unroll
+              for (int c4 = 0; c4 < 8; ++c4)
+                *reinterpret_cast<float4*>(row + (((unsigned)c4 ^ swz) << 4)) =
+                    make_float4(v[c4 * 4], v[c4 * 4 + 1], v[c4 * 4 + 2], v[c4 * 4 + 3]);
+            } else {
+#pragma unroll
+              for (int half = 0; half < 2; ++half) {
+                float v[32];
+                tmem_ld32(taddr + cb * 64 + half * 32, v);
+                if (EPI == EPI_DLOGITS && !PCTC_DBG_SKIP_MATH) {
+#pragma unroll
+                  for (int c = 0; c < 32; ++c)
+                    v[c] = w * ex2(fmaf(v[c] + sb[cb * 64 + half * 32 + c], LOG2E, -lam2));
+                }
+#pragma unroll
+                for (int c8 = 0; c8 < 4; ++c8) {
+                  uint4 o;
+                  __nv_bfloat162 p0 = __floats2bfloat162_rn(v[c8 * 8 + 0], v[c8 * 8 + 1]);
+                  __nv_bfloat162 p1 = __floats2bfloat162_rn(v[c8 * 8 + 2], v[c8 * 8 + 3]);
+                  __nv_bfloat162 p2 = __floats2bfloat162_rn(v[c8 * 8 + 4], v[c8 * 8 + 5]);
+                  __nv_bfloat162 p3 = __floats2bfloat162_rn(v[c8 * 8 + 6], v[c8 * 8 + 7]);
+                  o.x = *(unsigned*)&p0; o.y = *(unsigned*)&p1; o.z = *(unsigned*)&p2; o.w = *(unsigned*)&p3;
+                  *reinterpret_cast<uint4*>(row + (((unsigned)(half * 4 + c8) ^ swz) << 4)) = o;
+                }
+              }
+              if (EPI == EPI_DLOGITS) {
+                // selected classes of this box: subtract the occupancy in fp32, before the rounding to bf16
+                while (e_idx < nsel) {
+                  const unsigned ent = sl[e_idx];
+                  const int col = (int)(ent & 0xffu);
+                  if (col >= cb * 64 + 64) break;       // warp-uniform: the list is in ascending column order
+                  ++e_idx;
+                  const float z = tmem_ld1(taddr + col);
+                  if (row_ok) {
+                    const float pz = ex2(fmaf(z + sb[col], LOG2E, -lam2));
+                    const float g = a.e.gamma[(long long)i * a.e.ld_gamma + (int)(ent >> 8)];
+                    const unsigned cbx = (unsigned)(col - cb * 64) * 2u;    // byte offset inside the 128-byte row
+                    *reinterpret_cast<__nv_bfloat16*>(row + ((((cbx >> 4) ^ swz) << 4) | (cbx & 15u))) =
+                        __float2bfloat16_rn(w * (pz - g));
+                  }
+                }
+              }
+            }
+            fence_async_smem();                        // staged data visible to the TMA engine
+            __syncwarp();
+            if (lane == 0 && !PCTC_DBG_SKIP_STORE) {
+              if (EPI == EPI_ACCUM_F32 && a.e.accumulate) tma_reduce_add_2d(&tmC, stage, j0, mt * BM + q * 32);
+              else tma_store_2d(&tmC, stage, j0, mt * BM + q * 32);
+              bulk_commit();
+            }
+          }
+        }
+
+#pragma unroll 1
+        for (int cg = 0; cg < BN / 32 && !epi_uses_tma_store(EPI); ++cg) {
           if (n0 + cg * 32 >= n_eff) break;          // warp-uniform
           float v[32];
           tmem_ld32(taddr + cg * 32, v);
@@ -365,42 +483,6 @@ k_umma_gemm(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
 #pragma unroll
               for (int c = 0; c < 32; ++c)
                 if (j0 + c < n_eff) dst[c] = v[c];
-            }
-          } else if (EPI == EPI_ACCUM_F32) {
-            if (row_ok) {
-              float4* dst = (float4*)((float*)a.e.out + (long long)i * a.e.ld + j0);
-#pragma unroll
-              for (int c4 = 0; c4 < 8; ++c4) {
-                if (j0 + c4 * 4 < n_eff) {
-                  float4 o = make_float4(v[c4 * 4], v[c4 * 4 + 1], v[c4 * 4 + 2], v[c4 * 4 + 3]);
-                  if (a.e.accumulate) {
-                    const float4 old = dst[c4];
-                    o.x += old.x; o.y += old.y; o.z += old.z; o.w += old.w;
-                  }
-                  dst[c4] = o;
-                }
-              }
-            }
-          } else if (EPI == EPI_STORE_OUT || EPI == EPI_DLOGITS) {
-            if (EPI == EPI_DLOGITS) {
-#pragma unroll
-              for (int c = 0; c < 32; ++c)
-                v[c] = w * ex2(fmaf(v[c] + sb[cg * 32 + c], LOG2E, -lam2));
-            }
-            if (row_ok) {
-              uint4* dst = (uint4*)((__nv_bfloat16*)a.e.out + (long long)i * a.e.ld + j0);
-#pragma unroll
-              for (int c8 = 0; c8 < 4; ++c8) {
-                if (j0 + c8 * 8 < n_eff) {
-                  uint4 o;
-                  __nv_bfloat162 p0 = __floats2bfloat162_rn(v[c8 * 8 + 0], v[c8 * 8 + 1]);
-                  __nv_bfloat162 p1 = __floats2bfloat162_rn(v[c8 * 8 + 2], v[c8 * 8 + 3]);
-                  __nv_bfloat162 p2 = __floats2bfloat162_rn(v[c8 * 8 + 4], v[c8 * 8 + 5]);
-                  __nv_bfloat162 p3 = __floats2bfloat162_rn(v[c8 * 8 + 6], v[c8 * 8 + 7]);
-                  o.x = *(unsigned*)&p0; o.y = *(unsigned*)&p1; o.z = *(unsigned*)&p2; o.w = *(unsigned*)&p3;
-                  dst[c8] = o;
-                }
-              }
             }
           } else if (EPI == EPI_SUBSET_LOGP) {
             if (row_ok) {
@@ -428,19 +510,6 @@ k_umma_gemm(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
           }
         }
 
-        if (EPI == EPI_DLOGITS) {
-          // selected classes: subtract the occupancy in fp32, before the rounding to bf16
-          for (int e = 0; e < nsel; ++e) {
-            const int2 cj = sl[e];
-            const float z = tmem_ld1(taddr + cj.x);
-            if (row_ok) {
-              const float p = ex2(fmaf(z + sb[cj.x], LOG2E, -lam2));
-              const float g = a.e.gamma[(long long)i * a.e.ld_gamma + cj.y];
-              ((__nv_bfloat16*)a.e.out)[(long long)i * a.e.ld + n0 + cj.x] = __float2bfloat16_rn(w * (p - g));
-            }
-          }
-        }
-
         tc_fence_before();
         __syncwarp();
         if (lane == 0) mbar_arrive(&st->tmem_empty[acc]);
@@ -449,6 +518,7 @@ k_umma_gemm(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
       if (EPI == EPI_LSE_PARTIAL && ok && row_ok)
         a.e.partial[(long long)i * a.nsplit + sp] = make_float2(run_max2 * LN2, run_sum);
     }
+    if (epi_uses_tma_store(EPI) && lane == 0) bulk_wait0();   // this warp's stores have completed
   }
 
   tc_fence_before();
@@ -480,14 +550,15 @@ EncodeTiledFn encode_fn() {
 
 // 2-D bf16 tensor map: `inner` contiguous elements per row, `rows` rows of pitch `ld` elements.
 bool make_map(CUtensorMap* map, const void* base, unsigned long long inner, unsigned long long rows,
-              unsigned long long ld, unsigned box_inner, unsigned box_rows) {
+              unsigned long long ld, unsigned box_inner, unsigned box_rows, bool fp32 = false) {
   EncodeTiledFn fn = encode_fn();
   if (!fn) return false;
   cuuint64_t dims[2] = {inner, rows};
-  cuuint64_t strides[1] = {ld * 2};
+  cuuint64_t strides[1] = {ld * (fp32 ? 4 : 2)};
   cuuint32_t box[2] = {box_inner, box_rows};
   cuuint32_t estr[2] = {1, 1};
-  return fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(base), dims, strides, box, estr,
+  return fn(map, fp32 ? CU_TENSOR_MAP_DATA_TYPE_FLOAT32 : CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2,
+            const_cast<void*>(base), dims, strides, box, estr,
             CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
             CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
@@ -503,14 +574,17 @@ int sm_count() {
 }
 
 template <int EPI>
-cudaError_t launch(const CUtensorMap& tmA, const CUtensorMap& tmB, const UmmaArgs& a, int grid, cudaStream_t stream) {
+cudaError_t launch(const CUtensorMap& tmA, const CUtensorMap& tmB, const CUtensorMap& tmC, const UmmaArgs& a,
+                   int grid, cudaStream_t stream) {
   static bool configured = false;
+  constexpr size_t SMEM = smem_bytes(EPI);
+  static_assert(SMEM <= 227 * 1024, "shared memory budget");
   if (!configured) {
-    cudaError_t e = cudaFuncSetAttribute(k_umma_gemm<EPI>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)SMEM_BYTES);
+    cudaError_t e = cudaFuncSetAttribute(k_umma_gemm<EPI>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)SMEM);
     if (e != cudaSuccess) return e;
     configured = true;
   }
-  k_umma_gemm<EPI><<<grid, NUM_THREADS, SMEM_BYTES, stream>>>(tmA, tmB, a);
+  k_umma_gemm<EPI><<<grid, NUM_THREADS, SMEM, stream>>>(tmA, tmB, tmC, a);
   return cudaGetLastError();
 }
 
@@ -539,8 +613,17 @@ cudaError_t umma_gemm(const __nv_bfloat16* A, long long lda, bool a_mn_major,
                       int m, int n, int k, const Epilogue& e, int* status, cudaStream_t stream) {
   if (m <= 0 || n <= 0 || k <= 0) return cudaSuccess;
   if ((lda % 8) || (ldb % 8) || ((size_t)A & 15) || ((size_t)B & 15)) return cudaErrorInvalidValue;
-  alignas(64) CUtensorMap tmA, tmB;
+  alignas(64) CUtensorMap tmA, tmB, tmC;
   bool ok = true;
+  tmC = CUtensorMap{};
+  // output boxes of the staged epilogues: 32 rows x 128 bytes, clipped to the [m, n] extent
+  if (e.kind == EPI_ACCUM_F32) {
+    if ((e.ld % 4) || ((size_t)e.out & 15)) return cudaErrorInvalidValue;
+    ok = ok && make_map(&tmC, e.out, (unsigned long long)n, (unsigned long long)m, (unsigned long long)e.ld, 32, 32, true);
+  } else if (e.kind == EPI_DLOGITS || e.kind == EPI_STORE_OUT) {
+    if ((e.ld % 8) || ((size_t)e.out & 15)) return cudaErrorInvalidValue;
+    ok = ok && make_map(&tmC, e.out, (unsigned long long)n, (unsigned long long)m, (unsigned long long)e.ld, 64, 32);
+  }
   if (!a_mn_major) ok = ok && make_map(&tmA, A, (unsigned long long)k, (unsigned long long)m, lda, BK, BM);
   else ok = ok && make_map(&tmA, A, (unsigned long long)m, (unsigned long long)k, lda, 64, BK);
   if (!b_mn_major) ok = ok && make_map(&tmB, B, (unsigned long long)k, (unsigned long long)n, ldb, BK, BN);
@@ -552,6 +635,8 @@ cudaError_t umma_gemm(const __nv_bfloat16* A, long long lda, bool a_mn_major,
   a.a_mn = a_mn_major ? 1 : 0;
   a.b_mn = b_mn_major ? 1 : 0;
   a.nsplit = e.nsplit;
+  // dX += dZ W and dW = dZ^T X read a large A (the dZ chunk) against a smaller B: keep B resident
+  a.n_fastest = (PCTC_TUNE_N_FASTEST && (e.kind == EPI_ACCUM_F32 || e.kind == EPI_STORE_OUT)) ? 1 : 0;
   a.status = status;
   a.e = e;
   const int m_tiles = (m + BM - 1) / BM, n_tiles = (n + BN - 1) / BN;
@@ -559,12 +644,12 @@ cudaError_t umma_gemm(const __nv_bfloat16* A, long long lda, bool a_mn_major,
   if (e.kind == EPI_LSE_PARTIAL && (e.nsplit < 1 || e.nsplit > n_tiles)) return cudaErrorInvalidValue;
   const int grid = (int)(units < sm_count() ? units : sm_count());
   switch (e.kind) {
-    case EPI_STORE_F32: return launch<EPI_STORE_F32>(tmA, tmB, a, grid, stream);
-    case EPI_LSE_PARTIAL: return launch<EPI_LSE_PARTIAL>(tmA, tmB, a, grid, stream);
-    case EPI_SUBSET_LOGP: return launch<EPI_SUBSET_LOGP>(tmA, tmB, a, grid, stream);
-    case EPI_DLOGITS: return launch<EPI_DLOGITS>(tmA, tmB, a, grid, stream);
-    case EPI_ACCUM_F32: return launch<EPI_ACCUM_F32>(tmA, tmB, a, grid, stream);
-    case EPI_STORE_OUT: return launch<EPI_STORE_OUT>(tmA, tmB, a, grid, stream);
+    case EPI_STORE_F32: return launch<EPI_STORE_F32>(tmA, tmB, tmC, a, grid, stream);
+    case EPI_LSE_PARTIAL: return launch<EPI_LSE_PARTIAL>(tmA, tmB, tmC, a, grid, stream);
+    case EPI_SUBSET_LOGP: return launch<EPI_SUBSET_LOGP>(tmA, tmB, tmC, a, grid, stream);
+    case EPI_DLOGITS: return launch<EPI_DLOGITS>(tmA, tmB, tmC, a, grid, stream);
+    case EPI_ACCUM_F32: return launch<EPI_ACCUM_F32>(tmA, tmB, tmC, a, grid, stream);
+    case EPI_STORE_OUT: return launch<EPI_STORE_OUT>(tmA, tmB, tmC, a, grid, stream);
   }
   return cudaErrorInvalidValue;
 }

@@ -298,14 +298,16 @@ def utterance_fwd_bwd(Hn, W, b, y, blank, beam=None, bad=False):
 
 
 def pruned_ctc_reference(hidden, W, bias, targets, input_lengths, target_lengths, blank,
-                         beam=None, want_dW=True, dW_rows=None):
+                         beam=None, want_dW=True, dW_rows=None, dH_for=None):
     """Full-vocabulary CTC loss and gradients of the sum of utterance losses.
 
     hidden [N,T,D], W [V,D], bias [V] or None, targets [N,stride] int,
     input_lengths [N], target_lengths [N].  Returns a dict with
     loss [N], dH [N,T,D] (padded frames zero), dW [V,D] (or only the rows in
     `dW_rows`), db [V], U, K, relabeled, flags [N], exact_loss [N],
-    lam (list of per-utterance normalisers).
+    lam (list of per-utterance normalisers).  `dH_for`, if given, lists the
+    utterances whose dH is wanted (the others are left zero): sampled checks at
+    full size skip the products they do not look at.
     """
     hidden = np.asarray(hidden, dtype=np.float64)
     W64 = np.asarray(W, dtype=np.float64)
@@ -333,7 +335,8 @@ def pruned_ctc_reference(hidden, W, bias, targets, input_lengths, target_lengths
         loss[n], flags[n], exact[n] = l, f, ex
         if dZ is None:
             continue
-        dH[n, :Tn] = dZ @ W64
+        if dH_for is None or n in dH_for:
+            dH[n, :Tn] = dZ @ W64
         if want_dW:
             if rows is None:
                 dW += dZ.T @ Hn

@@ -169,7 +169,7 @@ def run_reference(args, cfg):
     budget = 150.0 / max(1, total_steps)
     dt8, _ = time_oracle(batch, W64, 8)          # calibration (also the first touch of the BLAS)
     frames = 8
-    for cand in (16, 32, 64, 128, 256):
+    for cand in (16, 32, 64, 128, 256, 512, 1024, 2048):
         # the per-call cost is a fixed O(V D) part plus a part linear in the frames
         if dt8 * (0.6 + 0.4 * cand / 8.0) <= budget:
             frames = cand
@@ -206,7 +206,7 @@ def main():
     ap.add_argument("--chunk", type=int, default=0)
     ap.add_argument("--e2e-steps", type=int, default=3)
     ap.add_argument("--no-cpu-baseline", action="store_true")
-    ap.add_argument("--cpu-frames", type=int, default=128)
+    ap.add_argument("--cpu-frames", type=int, default=1024)
     args = ap.parse_args()
     cfg = wl.CONFIGS[args.config]
 

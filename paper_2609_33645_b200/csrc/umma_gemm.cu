@@ -2,6 +2,12 @@
 // Algorithm 1:  acc(i,j) = sum_k A(i,k) B(j,k), bf16 operands, fp32 accumulators
 // in tensor memory.
 //
+// With CTAS == 2 (the default) two CTAs on neighbouring SMs form a cluster and share one
+// 256x256 tile: each loads its own 128 rows of A and its own 128 columns of B, the leader issues
+// tcgen05.mma.cta_group::2 for both, each keeps the accumulator of its 128 rows in its own tensor
+// memory and runs its own epilogue.  B then crosses L2 -> shared memory once per pair instead of
+// once per CTA, and the freed shared memory deepens the ring to six stages.
+//
 // One persistent CTA per SM, 192 threads in three roles:
 //   warp 0      TMA producer: 128-byte-swizzled operand tiles into a 4-stage ring
 //   warp 1      MMA issuer: tcgen05.mma 128x256x16 from shared-memory descriptors
@@ -36,9 +42,15 @@ namespace {
 #define PCTC_TUNE_N_FASTEST 1     // dX / dW kernels walk column tiles first
 #endif
 
-constexpr int BM = 128, BN = 256, BK = 64, STAGES = 4;
+#ifndef PCTC_TUNE_CTAS
+#define PCTC_TUNE_CTAS 2          // CTAs per tile: 2 = tcgen05 cta_group::2 pairs, 1 = independent CTAs
+#endif
+
+constexpr int BM = 128, BN = 256, BK = 64;
+constexpr int MAX_STAGES = 6;
+constexpr int stages_of(int ctas) { return ctas == 2 ? 6 : 4; }
 constexpr int A_STAGE_BYTES = BM * BK * 2;
-constexpr int B_STAGE_BYTES = BN * BK * 2;
+constexpr int b_stage_bytes(int ctas) { return (BN / ctas) * BK * 2; }   // each CTA of a pair holds half of B
 constexpr int NUM_THREADS = 192;
 constexpr int TMEM_COLS = 512;
 constexpr int MN_GROUP_BYTES = 64 * BK * 2;          // one 64-wide MN group of an MN-major tile
@@ -56,8 +68,8 @@ struct UmmaArgs {
 };
 
 struct SharedTail {   // barriers and flags
-  unsigned long long full[STAGES];
-  unsigned long long empty[STAGES];
+  unsigned long long full[MAX_STAGES];
+  unsigned long long empty[MAX_STAGES];
   unsigned long long tmem_full[2];
   unsigned long long tmem_empty[2];
   unsigned long long done;
@@ -73,13 +85,15 @@ struct SharedTail {   // barriers and flags
 constexpr int STAGE_BOX_BYTES = 4096;
 constexpr bool epi_uses_tma_store(int epi) { return epi == EPI_DLOGITS || epi == EPI_ACCUM_F32 || epi == EPI_STORE_OUT; }
 constexpr bool epi_uses_bias(int epi) { return epi == EPI_LSE_PARTIAL || epi == EPI_SUBSET_LOGP || epi == EPI_DLOGITS; }
-constexpr size_t RING_BYTES = (size_t)STAGES * (A_STAGE_BYTES + B_STAGE_BYTES);
+constexpr size_t ring_bytes(int ctas) { return (size_t)stages_of(ctas) * (A_STAGE_BYTES + b_stage_bytes(ctas)); }
+static_assert(ring_bytes(1) == ring_bytes(2), "both tile modes use the same operand ring size");
+constexpr size_t RING_BYTES = ring_bytes(1);
 constexpr size_t off_stage() { return RING_BYTES; }
 constexpr size_t off_tail(int epi) { return RING_BYTES + (epi_uses_tma_store(epi) ? 4 * STAGE_BOX_BYTES : 0); }
-constexpr size_t off_bias(int epi) { return off_tail(epi) + 128; }
+constexpr size_t off_bias(int epi) { return off_tail(epi) + 256; }
 constexpr size_t off_list(int epi) { return off_bias(epi) + (epi_uses_bias(epi) ? 4 * BN * 4 : 0); }
 constexpr size_t smem_bytes(int epi) { return 1024 + off_list(epi) + (epi == EPI_DLOGITS ? 4 * BN * 4 : 0); }
-static_assert(sizeof(SharedTail) <= 128, "tail layout");
+static_assert(sizeof(SharedTail) <= 256, "tail layout");
 
 // ---------------------------------------------------------------------------------------------
 // PTX wrappers
@@ -147,6 +161,47 @@ __device__ __forceinline__ void bulk_commit() { asm volatile("cp.async.bulk.comm
 __device__ __forceinline__ void bulk_wait_read0() { asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory"); }
 __device__ __forceinline__ void bulk_wait0() { asm volatile("cp.async.bulk.wait_group 0;" ::: "memory"); }
 __device__ __forceinline__ void fence_async_smem() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
+
+// --- two-CTA (cluster) forms ---
+constexpr unsigned PEER_MASK = 0xFEFFFFFFu;   // shared::cluster address of the same offset in the pair's CTA 0
+__device__ __forceinline__ unsigned cluster_ctarank() {
+  unsigned r;
+  asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(r));
+  return r;
+}
+__device__ __forceinline__ void cluster_sync_all() {
+  asm volatile("barrier.cluster.arrive.release.aligned;\n\tbarrier.cluster.wait.acquire.aligned;" ::: "memory");
+}
+// TMA load issued by either CTA of a pair into its own shared memory; the bytes are counted on the
+// leader's barrier (no multicast: every CTA fetches its own box).
+__device__ __forceinline__ void tma_load_2d_pair(void* smem_dst, const CUtensorMap* map, int c0, int c1,
+                                                 unsigned long long* bar) {
+  asm volatile(
+      "cp.async.bulk.tensor.2d.cta_group::2.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
+      ::"r"(smem_u32(smem_dst)), "l"(map), "r"(c0), "r"(c1), "r"(smem_u32(bar) & PEER_MASK)
+      : "memory");
+}
+__device__ __forceinline__ void mbar_arrive_leader(unsigned long long* bar) {
+  asm volatile("mbarrier.arrive.shared::cluster.b64 _, [%0];" ::"r"(smem_u32(bar) & PEER_MASK) : "memory");
+}
+__device__ __forceinline__ void tc_commit_pair(unsigned long long* bar) {       // arrives in both CTAs
+  asm volatile("tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.multicast::cluster.b64 [%0], %1;"
+               ::"r"(smem_u32(bar)), "h"((unsigned short)3)
+               : "memory");
+}
+__device__ __forceinline__ void tc_commit_pair_local(unsigned long long* bar) { // arrives in the issuing CTA only
+  asm volatile("tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(smem_u32(bar))
+               : "memory");
+}
+__device__ __forceinline__ void tc_mma_bf16_pair(unsigned tmem_d, unsigned long long adesc, unsigned long long bdesc,
+                                                 unsigned idesc, unsigned accumulate) {
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "setp.ne.b32 p, %4, 0;\n\t"
+      "tcgen05.mma.cta_group::2.kind::f16 [%0], %1, %2, %3, p;\n\t}"
+      ::"r"(tmem_d), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate)
+      : "memory");
+}
 
 __device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
 __device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
@@ -229,10 +284,13 @@ __device__ __forceinline__ void decode_unit(int u, int m_tiles, int n_tiles, int
 // ---------------------------------------------------------------------------------------------
 // The kernel
 // ---------------------------------------------------------------------------------------------
-template <int EPI>
+template <int EPI, int CTAS>
 __global__ void __launch_bounds__(NUM_THREADS, 1)
 k_umma_gemm(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
             const __grid_constant__ CUtensorMap tmC, UmmaArgs a) {
+  constexpr int STAGES = stages_of(CTAS);
+  constexpr int B_STAGE_BYTES = b_stage_bytes(CTAS);
+  constexpr int TILE_M = BM * CTAS;            // rows of the tile a CTA (pair) works on
   extern __shared__ unsigned char smem_raw[];
   unsigned char* smem = (unsigned char*)(((size_t)smem_raw + 1023) & ~(size_t)1023);
   unsigned char* sA = smem;
@@ -240,11 +298,13 @@ k_umma_gemm(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
   SharedTail* st = (SharedTail*)(smem + off_tail(EPI));
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int rank = (CTAS == 2) ? (int)cluster_ctarank() : 0;     // position inside the pair
+  const int group = blockIdx.x / CTAS, ngroups = gridDim.x / CTAS;
 
   // problem decomposition, identical in every role
   int n_eff = a.n;
   if (EPI == EPI_SUBSET_LOGP) n_eff = min(a.n, *a.e.Kdev);
-  const int m_tiles = (a.m + BM - 1) / BM;
+  const int m_tiles = (a.m + TILE_M - 1) / TILE_M;
   const int n_tiles = (n_eff + BN - 1) / BN;
   const int splits = (EPI == EPI_LSE_PARTIAL) ? a.nsplit : n_tiles;
   const int units = m_tiles * splits;
@@ -252,20 +312,28 @@ k_umma_gemm(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
 
   if (threadIdx.x == 0) {
     for (int s = 0; s < STAGES; ++s) { mbar_init(&st->full[s], 1); mbar_init(&st->empty[s], 1); }
-    for (int s = 0; s < 2; ++s) { mbar_init(&st->tmem_full[s], 1); mbar_init(&st->tmem_empty[s], 4); }
+    for (int s = 0; s < 2; ++s) { mbar_init(&st->tmem_full[s], 1); mbar_init(&st->tmem_empty[s], 4 * CTAS); }
     mbar_init(&st->done, 1);
     st->abort = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
   }
   if (warp == 1) {
-    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&st->tmem_base)),
-                 "r"(TMEM_COLS)
-                 : "memory");
-    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+    if (CTAS == 2) {
+      asm volatile("tcgen05.alloc.cta_group::2.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&st->tmem_base)),
+                   "r"(TMEM_COLS)
+                   : "memory");
+      asm volatile("tcgen05.relinquish_alloc_permit.cta_group::2.sync.aligned;" ::: "memory");
+    } else {
+      asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&st->tmem_base)),
+                   "r"(TMEM_COLS)
+                   : "memory");
+      asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+    }
   }
   tc_fence_before();
   __syncthreads();
+  if (CTAS == 2) cluster_sync_all();     // the peer's barriers exist before anything signals them
   tc_fence_after();
   const unsigned tmem_base = st->tmem_base;
   volatile int* abort_flag = &st->abort;
@@ -275,50 +343,60 @@ k_umma_gemm(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
     if (lane == 0) {
       unsigned g = 0;
       bool ok = true;
-      for (int u = blockIdx.x; u < units && ok; u += gridDim.x) {
+      auto load = [&](void* dst, const CUtensorMap* map, int c0, int c1, unsigned long long* bar) {
+        if (CTAS == 2) tma_load_2d_pair(dst, map, c0, c1, bar);
+        else tma_load_2d(dst, map, c0, c1, bar);
+      };
+      for (int u = group; u < units && ok; u += ngroups) {
         int mt, sp, nt0, cnt;
         decode_unit(u, m_tiles, n_tiles, splits, a.n_fastest != 0, mt, sp, nt0, cnt);
+        const int row_a = mt * TILE_M + rank * BM;               // this CTA's rows of A
         for (int nt = nt0; nt < nt0 + cnt && ok; ++nt) {
+          const int row_b = nt * BN + rank * (BN / CTAS);        // this CTA's columns of the tile (rows of B)
           for (int kb = 0; kb < k_blocks; ++kb, ++g) {
             const int s = g % STAGES;
             const unsigned ph = (g / STAGES) & 1u;
             if (!mbar_wait(&st->empty[s], ph ^ 1u, abort_flag, a.status, 1)) { ok = false; break; }
-            mbar_expect_tx(&st->full[s], A_STAGE_BYTES + B_STAGE_BYTES);
+            // the leader's barrier counts the bytes of both CTAs
+            if (rank == 0) mbar_expect_tx(&st->full[s], CTAS * (A_STAGE_BYTES + B_STAGE_BYTES));
             unsigned char* dA = sA + (size_t)s * A_STAGE_BYTES;
             unsigned char* dB = sB + (size_t)s * B_STAGE_BYTES;
             if (!a.a_mn) {
-              tma_load_2d(dA, &tmA, kb * BK, mt * BM, &st->full[s]);
+              load(dA, &tmA, kb * BK, row_a, &st->full[s]);
             } else {
 #pragma unroll
               for (int q = 0; q < BM / 64; ++q)
-                tma_load_2d(dA + q * MN_GROUP_BYTES, &tmA, mt * BM + q * 64, kb * BK, &st->full[s]);
+                load(dA + q * MN_GROUP_BYTES, &tmA, row_a + q * 64, kb * BK, &st->full[s]);
             }
             if (!a.b_mn) {
-              tma_load_2d(dB, &tmB, kb * BK, nt * BN, &st->full[s]);
+              load(dB, &tmB, kb * BK, row_b, &st->full[s]);
             } else {
 #pragma unroll
-              for (int q = 0; q < BN / 64; ++q)
-                tma_load_2d(dB + q * MN_GROUP_BYTES, &tmB, nt * BN + q * 64, kb * BK, &st->full[s]);
+              for (int q = 0; q < BN / CTAS / 64; ++q)
+                load(dB + q * MN_GROUP_BYTES, &tmB, row_b + q * 64, kb * BK, &st->full[s]);
             }
           }
         }
       }
-      // drain: every copy this thread issued has landed before the CTA may exit
-      const unsigned issued = g;
-      for (unsigned j = (issued > STAGES ? issued - STAGES : 0); j < issued; ++j)
-        mbar_wait(&st->full[j % STAGES], (j / STAGES) & 1u, abort_flag, nullptr, 0, 200000000LL);
+      // drain: every copy issued has landed before the CTA may exit.  The leader's barriers count
+      // the peer's bytes too; the peer itself stays alive until the closing cluster barrier.
+      if (rank == 0) {
+        const unsigned issued = g;
+        for (unsigned j = (issued > STAGES ? issued - STAGES : 0); j < issued; ++j)
+          mbar_wait(&st->full[j % STAGES], (j / STAGES) & 1u, abort_flag, nullptr, 0, 200000000LL);
+      }
     }
   } else if (warp == 1) {
     // ===================== MMA issuer =====================
-    if (lane == 0) {
+    if (lane == 0 && rank == 0) {        // the leader issues the MMAs of the pair
       const unsigned idesc = (1u << 4) | (1u << 7) | (1u << 10) | ((unsigned)(a.a_mn ? 1 : 0) << 15) |
                              ((unsigned)(a.b_mn ? 1 : 0) << 16) | ((unsigned)(BN >> 3) << 17) |
-                             ((unsigned)(BM >> 4) << 24);
+                             ((unsigned)(TILE_M >> 4) << 24);
       const unsigned a_step = a.a_mn ? (2048u >> 4) : (32u >> 4);   // descriptor advance per 16 k
       const unsigned b_step = a.b_mn ? (2048u >> 4) : (32u >> 4);
       unsigned g = 0, it = 0;
       bool ok = true;
-      for (int u = blockIdx.x; u < units && ok; u += gridDim.x) {
+      for (int u = group; u < units && ok; u += ngroups) {
         int mt, sp, nt0, cnt;
         decode_unit(u, m_tiles, n_tiles, splits, a.n_fastest != 0, mt, sp, nt0, cnt);
         (void)mt;
@@ -335,16 +413,20 @@ k_umma_gemm(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
             const unsigned long long adesc = make_smem_desc(smem_u32(sA + (size_t)s * A_STAGE_BYTES), a.a_mn);
             const unsigned long long bdesc = make_smem_desc(smem_u32(sB + (size_t)s * B_STAGE_BYTES), a.b_mn);
 #pragma unroll
-            for (int kk = 0; kk < BK / 16; ++kk)
-              tc_mma_bf16(d_tmem, adesc + (unsigned long long)(kk * a_step), bdesc + (unsigned long long)(kk * b_step),
-                          idesc, (kb | kk) != 0 ? 1u : 0u);
-            tc_commit(&st->empty[s]);        // frees the stage once these MMAs have read it
+            for (int kk = 0; kk < BK / 16; ++kk) {
+              const unsigned long long ad = adesc + (unsigned long long)(kk * a_step);
+              const unsigned long long bd = bdesc + (unsigned long long)(kk * b_step);
+              if (CTAS == 2) tc_mma_bf16_pair(d_tmem, ad, bd, idesc, (kb | kk) != 0 ? 1u : 0u);
+              else tc_mma_bf16(d_tmem, ad, bd, idesc, (kb | kk) != 0 ? 1u : 0u);
+            }
+            // frees the stage (in both CTAs) once these MMAs have read it
+            if (CTAS == 2) tc_commit_pair(&st->empty[s]); else tc_commit(&st->empty[s]);
           }
-          if (ok) tc_commit(&st->tmem_full[acc]);
+          if (ok) { if (CTAS == 2) tc_commit_pair(&st->tmem_full[acc]); else tc_commit(&st->tmem_full[acc]); }
         }
       }
       // all MMAs issued by this thread have completed before tensor memory is freed
-      tc_commit(&st->done);
+      if (CTAS == 2) tc_commit_pair_local(&st->done); else tc_commit(&st->done);
       mbar_wait(&st->done, 0, abort_flag, nullptr, 0, 200000000LL);
     }
   } else {
@@ -358,10 +440,11 @@ k_umma_gemm(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
     const unsigned swz = (unsigned)(lane & 7);                           // 128-byte swizzle of the staged row
     unsigned it = 0;
     bool ok = true;
-    for (int u = blockIdx.x; u < units && ok; u += gridDim.x) {
+    for (int u = group; u < units && ok; u += ngroups) {
       int mt, sp, nt0, cnt;
       decode_unit(u, m_tiles, n_tiles, splits, a.n_fastest != 0, mt, sp, nt0, cnt);
-      const int i = mt * BM + r;
+      const int row0_cta = mt * TILE_M + rank * BM;      // first row of this CTA's half of the tile
+      const int i = row0_cta + r;
       const bool row_ok = i < a.m;
       float lam2 = 0.f, lam = 0.f, w = 0.f;
       if ((EPI == EPI_DLOGITS || (EPI == EPI_SUBSET_LOGP && a.e.lambda)) && row_ok) { lam = a.e.lambda[i]; lam2 = lam * LOG2E; }
@@ -464,8 +547,8 @@ k_umma_gemm(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
             fence_async_smem();                        // staged data visible to the TMA engine
             __syncwarp();
             if (lane == 0 && !PCTC_DBG_SKIP_STORE) {
-              if (EPI == EPI_ACCUM_F32 && a.e.accumulate) tma_reduce_add_2d(&tmC, stage, j0, mt * BM + q * 32);
-              else tma_store_2d(&tmC, stage, j0, mt * BM + q * 32);
+              if (EPI == EPI_ACCUM_F32 && a.e.accumulate) tma_reduce_add_2d(&tmC, stage, j0, row0_cta + q * 32);
+              else tma_store_2d(&tmC, stage, j0, row0_cta + q * 32);
               bulk_commit();
             }
           }
@@ -512,7 +595,7 @@ k_umma_gemm(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
 
         tc_fence_before();
         __syncwarp();
-        if (lane == 0) mbar_arrive(&st->tmem_empty[acc]);
+        if (lane == 0) { if (CTAS == 2) mbar_arrive_leader(&st->tmem_empty[acc]); else mbar_arrive(&st->tmem_empty[acc]); }
       }
 
       if (EPI == EPI_LSE_PARTIAL && ok && row_ok)
@@ -523,9 +606,13 @@ k_umma_gemm(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
 
   tc_fence_before();
   __syncthreads();
+  if (CTAS == 2) cluster_sync_all();     // no CTA of a pair leaves while the other may still signal it
   if (warp == 1) {
     tc_fence_after();
-    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(TMEM_COLS) : "memory");
+    if (CTAS == 2)
+      asm volatile("tcgen05.dealloc.cta_group::2.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(TMEM_COLS) : "memory");
+    else
+      asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(TMEM_COLS) : "memory");
   }
 }
 
@@ -573,19 +660,51 @@ int sm_count() {
   return n;
 }
 
+constexpr int CTAS_DEFAULT = PCTC_TUNE_CTAS;
+
 template <int EPI>
 cudaError_t launch(const CUtensorMap& tmA, const CUtensorMap& tmB, const CUtensorMap& tmC, const UmmaArgs& a,
                    int grid, cudaStream_t stream) {
   static bool configured = false;
   constexpr size_t SMEM = smem_bytes(EPI);
   static_assert(SMEM <= 227 * 1024, "shared memory budget");
+  auto kern = k_umma_gemm<EPI, CTAS_DEFAULT>;
   if (!configured) {
-    cudaError_t e = cudaFuncSetAttribute(k_umma_gemm<EPI>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)SMEM);
+    cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)SMEM);
     if (e != cudaSuccess) return e;
     configured = true;
   }
-  k_umma_gemm<EPI><<<grid, NUM_THREADS, SMEM, stream>>>(tmA, tmB, tmC, a);
-  return cudaGetLastError();
+  cudaLaunchConfig_t cfg = {};
+  static int max_groups = 0;        // CTA groups (clusters) that can be resident at once
+  if (max_groups == 0) {
+    cudaLaunchConfig_t q = {};
+    q.gridDim = dim3((unsigned)(sm_count() / CTAS_DEFAULT * CTAS_DEFAULT));
+    q.blockDim = dim3(NUM_THREADS);
+    q.dynamicSmemBytes = SMEM;
+    cudaLaunchAttribute qa[1];
+    qa[0].id = cudaLaunchAttributeClusterDimension;
+    qa[0].val.clusterDim.x = CTAS_DEFAULT;
+    qa[0].val.clusterDim.y = 1;
+    qa[0].val.clusterDim.z = 1;
+    q.attrs = qa;
+    q.numAttrs = 1;
+    int n = 0;
+    if (cudaOccupancyMaxActiveClusters(&n, kern, &q) != cudaSuccess || n <= 0) n = sm_count() / CTAS_DEFAULT;
+    max_groups = n;
+  }
+  if (grid > max_groups * CTAS_DEFAULT) grid = max_groups * CTAS_DEFAULT;
+  cfg.gridDim = dim3((unsigned)grid);
+  cfg.blockDim = dim3(NUM_THREADS);
+  cfg.dynamicSmemBytes = SMEM;
+  cfg.stream = stream;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeClusterDimension;
+  attr[0].val.clusterDim.x = CTAS_DEFAULT;
+  attr[0].val.clusterDim.y = 1;
+  attr[0].val.clusterDim.z = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = 1;
+  return cudaLaunchKernelEx(&cfg, kern, tmA, tmB, tmC, a);
 }
 
 }  // namespace
@@ -594,8 +713,8 @@ bool umma_available() { return encode_fn() != nullptr; }
 
 int umma_lse_splits(int m, int n) {
   // column splits per row tile such that the (row tile, split) units fill whole waves of CTAs
-  const int sms = sm_count();
-  const int m_tiles = (m + BM - 1) / BM, n_tiles = (n + BN - 1) / BN;
+  const int sms = sm_count() / CTAS_DEFAULT;       // CTA groups that run at once
+  const int m_tiles = (m + BM * CTAS_DEFAULT - 1) / (BM * CTAS_DEFAULT), n_tiles = (n + BN - 1) / BN;
   int best = 1;
   double best_cost = 1e30;
   for (int s = 1; s <= 64 && s <= n_tiles; ++s) {
@@ -626,7 +745,7 @@ cudaError_t umma_gemm(const __nv_bfloat16* A, long long lda, bool a_mn_major,
   }
   if (!a_mn_major) ok = ok && make_map(&tmA, A, (unsigned long long)k, (unsigned long long)m, lda, BK, BM);
   else ok = ok && make_map(&tmA, A, (unsigned long long)m, (unsigned long long)k, lda, 64, BK);
-  if (!b_mn_major) ok = ok && make_map(&tmB, B, (unsigned long long)k, (unsigned long long)n, ldb, BK, BN);
+  if (!b_mn_major) ok = ok && make_map(&tmB, B, (unsigned long long)k, (unsigned long long)n, ldb, BK, BN / CTAS_DEFAULT);
   else ok = ok && make_map(&tmB, B, (unsigned long long)n, (unsigned long long)k, ldb, 64, BK);
   if (!ok) return cudaErrorInvalidValue;
 
@@ -639,10 +758,11 @@ cudaError_t umma_gemm(const __nv_bfloat16* A, long long lda, bool a_mn_major,
   a.n_fastest = (PCTC_TUNE_N_FASTEST && (e.kind == EPI_ACCUM_F32 || e.kind == EPI_STORE_OUT)) ? 1 : 0;
   a.status = status;
   a.e = e;
-  const int m_tiles = (m + BM - 1) / BM, n_tiles = (n + BN - 1) / BN;
+  const int m_tiles = (m + BM * CTAS_DEFAULT - 1) / (BM * CTAS_DEFAULT), n_tiles = (n + BN - 1) / BN;
   long long units = (long long)m_tiles * (e.kind == EPI_LSE_PARTIAL ? e.nsplit : n_tiles);
   if (e.kind == EPI_LSE_PARTIAL && (e.nsplit < 1 || e.nsplit > n_tiles)) return cudaErrorInvalidValue;
-  const int grid = (int)(units < sm_count() ? units : sm_count());
+  const int groups = sm_count() / CTAS_DEFAULT;
+  const int grid = (int)(units < groups ? units : groups) * CTAS_DEFAULT;
   switch (e.kind) {
     case EPI_STORE_F32: return launch<EPI_STORE_F32>(tmA, tmB, tmC, a, grid, stream);
     case EPI_LSE_PARTIAL: return launch<EPI_LSE_PARTIAL>(tmA, tmB, tmC, a, grid, stream);

@@ -38,6 +38,9 @@ namespace {
 #ifndef PCTC_DBG_SKIP_MATH
 #define PCTC_DBG_SKIP_MATH 0      // timing experiments only: drop the exponentials of the dlogits epilogue
 #endif
+#ifndef PCTC_DBG_NO_STAGE_WAIT
+#define PCTC_DBG_NO_STAGE_WAIT 0  // timing experiments only (races): do not wait for the staging buffer
+#endif
 #ifndef PCTC_TUNE_N_FASTEST
 #define PCTC_TUNE_N_FASTEST 1     // dX / dW kernels walk column tiles first
 #endif
@@ -495,7 +498,7 @@ k_umma_gemm(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
           for (int cb = 0; cb < BN / BOX_COLS; ++cb) {
             const int j0 = n0 + cb * BOX_COLS;
             if (j0 >= n_eff) break;                   // warp-uniform
-            if (lane == 0) bulk_wait_read0();          // the previous box has been read out of the staging buffer
+            if (lane == 0 && !PCTC_DBG_NO_STAGE_WAIT) bulk_wait_read0();   // the previous box has left the staging buffer
             __syncwarp();
             unsigned char* row = stage + lane * 128;
             if (EPI == EPI_ACCUM_F32) {

@@ -32,15 +32,6 @@ namespace pctc {
 namespace {
 
 // Tunables (overridable at compile time for experiments)
-#ifndef PCTC_DBG_SKIP_STORE
-#define PCTC_DBG_SKIP_STORE 0     // timing experiments only: drop the epilogue's global stores
-#endif
-#ifndef PCTC_DBG_SKIP_MATH
-#define PCTC_DBG_SKIP_MATH 0      // timing experiments only: drop the exponentials of the dlogits epilogue
-#endif
-#ifndef PCTC_DBG_NO_STAGE_WAIT
-#define PCTC_DBG_NO_STAGE_WAIT 0  // timing experiments only (races): do not wait for the staging buffer
-#endif
 #ifndef PCTC_TUNE_N_FASTEST
 #define PCTC_TUNE_N_FASTEST 1     // dX / dW kernels walk column tiles first
 #endif
@@ -498,7 +489,7 @@ k_umma_gemm(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
           for (int cb = 0; cb < BN / BOX_COLS; ++cb) {
             const int j0 = n0 + cb * BOX_COLS;
             if (j0 >= n_eff) break;                   // warp-uniform
-            if (lane == 0 && !PCTC_DBG_NO_STAGE_WAIT) bulk_wait_read0();   // the previous box has left the staging buffer
+            if (lane == 0) bulk_wait_read0();   // the previous box has left the staging buffer
             __syncwarp();
             unsigned char* row = stage + lane * 128;
             if (EPI == EPI_ACCUM_F32) {
@@ -513,7 +504,7 @@ k_umma_gemm(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
               for (int half = 0; half < 2; ++half) {
                 float v[32];
                 tmem_ld32(taddr + cb * 64 + half * 32, v);
-                if (EPI == EPI_DLOGITS && !PCTC_DBG_SKIP_MATH) {
+                if (EPI == EPI_DLOGITS) {
 #pragma unroll
                   for (int c = 0; c < 32; ++c)
                     v[c] = w * ex2(fmaf(v[c] + sb[cb * 64 + half * 32 + c], LOG2E, -lam2));
@@ -549,7 +540,7 @@ k_umma_gemm(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
             }
             fence_async_smem();                        // staged data visible to the TMA engine
             __syncwarp();
-            if (lane == 0 && !PCTC_DBG_SKIP_STORE) {
+            if (lane == 0) {
               if (EPI == EPI_ACCUM_F32 && a.e.accumulate) tma_reduce_add_2d(&tmC, stage, j0, row0_cta + q * 32);
               else tma_store_2d(&tmC, stage, j0, row0_cta + q * 32);
               bulk_commit();

@@ -204,6 +204,8 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--beam", type=float, default=0.0)
     ap.add_argument("--chunk", type=int, default=0)
+    ap.add_argument("--frozen-head", action="store_true",
+                    help="skip dW (the LLM-CTC setting): 6 M D V FLOPs per step instead of 8")
     ap.add_argument("--e2e-steps", type=int, default=3)
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--cpu-frames", type=int, default=1024)
@@ -244,7 +246,7 @@ def main():
     targets = h_targets.to(dev, non_blocking=True)
     il, tl = batch.input_lengths, batch.target_lengths
     M, D, V, N = batch.M, cfg.D, cfg.V, cfg.N
-    flops_per_step = 8.0 * M * D * V
+    flops_per_step = (6.0 if args.frozen_head else 8.0) * M * D * V
 
     chunk = args.chunk or DEFAULT_CHUNK
     prob = binding.make_problem(N, batch.T, D, V, binding.PCTC_BF16 if cfg.dtype == "bf16" else binding.PCTC_FP32,
@@ -253,12 +255,13 @@ def main():
     chunk = args.chunk or DEFAULT_CHUNK
     nchunks = (V + chunk - 1) // chunk
     call = dict(beam=args.beam, chunk=chunk)
+    dev_call = dict(call, skip_dW=args.frozen_head)
 
-    res = binding.pruned_ctc_fwd_bwd(hidden, W, None, targets, il, tl, batch.blank, check_status=True, **call)
+    res = binding.pruned_ctc_fwd_bwd(hidden, W, None, targets, il, tl, batch.blank, check_status=True, **dev_call)
     torch.cuda.synchronize()
     for _ in range(max(0, args.warmup - 1)):
         res = binding.pruned_ctc_fwd_bwd(hidden, W, None, targets, il, tl, batch.blank,
-                                         workspace=res["workspace"], out=res, **call)
+                                         workspace=res["workspace"], out=res, **dev_call)
     torch.cuda.synchronize()
 
     traces = [binding.Trace(binding.Trace.capacity_for(V, chunk)) for _ in range(args.steps)]
@@ -273,7 +276,7 @@ def main():
     ev0.record()
     for s in range(args.steps):
         binding.pruned_ctc_fwd_bwd(hidden, W, None, targets, il, tl, batch.blank, workspace=res["workspace"],
-                                   out=res, trace=traces[s], **call)
+                                   out=res, trace=traces[s], **dev_call)
     ev1.record()
     torch.cuda.synchronize()
     if world > 1:
@@ -305,18 +308,22 @@ def main():
     peak = peaks["bf16_tflops_sustained"]
     per_kernel = {}
     split_flops = dict(lse=2.0 * M * D * V, dlogits=2.0 * M * D * V, dh=2.0 * M * D * V, dw=2.0 * M * D * V)
+    if args.frozen_head:
+        gemm_phases = ("lse", "dlogits", "dh")
+        gemm_ms = sum(phase_ms[k] for k in gemm_phases)
+        achieved_tflops = flops_per_step / (gemm_ms * 1e-3) / 1e12
     for k in gemm_phases:
         per_kernel[k] = dict(ms=round(phase_ms[k], 4), launches=phase_cnt[k] // args.steps,
                              tflops=round(split_flops[k] / (phase_ms[k] * 1e-3) / 1e12, 2))
 
     # kernels launched by the library inside the timed region
     dp_launches = 3 if args.beam > 0 else 2
-    launches_per_step = 3 + 1 + 2 + 2 + dp_launches + 1 + 3 * nchunks + 1
+    launches_per_step = 3 + 1 + 2 + 2 + dp_launches + 1 + (2 if args.frozen_head else 3) * nchunks + 1
     gpu_launches = launches_per_step * args.steps
 
     # ---- end to end through the host-buffer entry point ----
     e2e = None
-    if args.e2e_steps > 0:
+    if args.e2e_steps > 0 and not args.frozen_head:
         h_res = binding.pruned_ctc_fwd_bwd_host(h_hidden, h_W, None, h_targets, il, tl, batch.blank,
                                                 device=dev, **call)
         torch.cuda.synchronize()
@@ -345,7 +352,8 @@ def main():
         return 0
 
     # ---- peak head-and-loss bytes; the workspace does not depend on M*V ----
-    out_bytes = (N * 4 + hidden.numel() * hidden.element_size() + W.numel() * W.element_size())
+    out_bytes = (N * 4 + hidden.numel() * hidden.element_size()
+                 + (0 if args.frozen_head else W.numel() * W.element_size()))
     prob_half = binding.make_problem(N, batch.T, D, V // 2 // 8 * 8, prob.dtype, batch.blank, args.beam, chunk,
                                      batch.targets.shape[1])
     ws_half = binding.workspace_bytes(prob_half, il, tl)
@@ -364,7 +372,7 @@ def main():
         ms_per_step=ms_per_step, higher_is_better=True, scaling="weak", vs_baseline=None,
         dtype=cfg.dtype, data="synthetic",
         config=dict(workload=cfg.name, N=N, T_range=[cfg.T_lo, cfg.T_hi], D=D, V=V, M_frames=M,
-                    K_selected=int(res["K"].item()), beam=args.beam, chunk=chunk,
+                    K_selected=int(res["K"].item()), beam=args.beam, chunk=chunk, frozen_head=args.frozen_head,
                     l2="inputs larger than L2 (W and dW are %.2f GB each)" % (W.numel() * 2 / 1e9),
                     parallelism="independent utterance batches per GPU, no collective"),
         tflops=flops_all / (ms_per_step * 1e-3) / 1e12,

@@ -64,6 +64,14 @@ typedef struct {
   int32_t chunk;         /* vocabulary chunk width C (Algorithm 1); 0: library default        */
   int32_t target_stride; /* row pitch of targets and relabeled_out                            */
   int32_t gemm_path;     /* pctc_gemm_path_t                                                  */
+  int32_t skip_dW;       /* 1: frozen head (the LLM-CTC setting, Section 4.2): dW is neither
+                            computed nor touched (dW may be NULL); dH and dbias still are        */
+  int32_t accumulate_dW; /* 1: dW and dbias are added to (gradient accumulation over
+                            micro-batches) instead of overwritten                              */
+  const float* utt_weights; /* device [N] or NULL: upstream gradient c_n of each utterance loss
+                            (loss scaling, token-count normalisation; Appendix B.1, "row sums of
+                            G"): gradients are those of sum_n c_n L_n; the returned losses stay
+                            unweighted.  NULL means c_n = 1                                    */
 } pctc_problem_t;
 
 /*
@@ -93,7 +101,7 @@ pctc_status_t pctc_workspace_bytes(const pctc_problem_t* problem,
  *             is 0                                                  -> loss, utt_flags
  *   line 10   occupancies gamma (G = -gamma)                       (workspace, fp32)
  *   line 11-17 per vocabulary chunk: recompute Z, dZ = w_m (exp(Z - lambda) - scatter_U(gamma))
- *             (Eq. "vjp" with unit weights; w_m = 0 on frames of excluded utterances),
+ *             (Eq. "vjp"; w_m = c_n on frames of utterance n, 0 on frames of excluded utterances),
  *             dH += dZ W_c, dW_c = dZ^T X, db_c = dZ^T 1           -> dH, dW, dbias
  *
  * Pointers (device unless marked HOST; all contiguous, row-major):
@@ -175,7 +183,8 @@ pctc_status_t pruned_ctc_fwd_bwd_traced(const pctc_problem_t* problem,
  * 1; device-to-host copies of loss, dH, dW, dbias and the optional integer
  * outputs.  The call does not synchronise: the host outputs are valid once
  * `stream` has been synchronised, and the host inputs must stay unchanged until
- * then.  Same return codes as pruned_ctc_fwd_bwd.
+ * then.  Same return codes as pruned_ctc_fwd_bwd.  skip_dW, accumulate_dW and utt_weights
+ * belong to the device entry point only: here they return PCTC_ERR_UNSUPPORTED.
  */
 pctc_status_t pctc_host_call_scratch_bytes(const pctc_problem_t* problem,
                                            const int32_t* input_lengths_host,

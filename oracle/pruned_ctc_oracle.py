@@ -298,7 +298,7 @@ def utterance_fwd_bwd(Hn, W, b, y, blank, beam=None, bad=False):
 
 
 def pruned_ctc_reference(hidden, W, bias, targets, input_lengths, target_lengths, blank,
-                         beam=None, want_dW=True, dW_rows=None, dH_for=None):
+                         beam=None, want_dW=True, dW_rows=None, dH_for=None, utt_weights=None):
     """Full-vocabulary CTC loss and gradients of the sum of utterance losses.
 
     hidden [N,T,D], W [V,D], bias [V] or None, targets [N,stride] int,
@@ -307,7 +307,10 @@ def pruned_ctc_reference(hidden, W, bias, targets, input_lengths, target_lengths
     `dW_rows`), db [V], U, K, relabeled, flags [N], exact_loss [N],
     lam (list of per-utterance normalisers).  `dH_for`, if given, lists the
     utterances whose dH is wanted (the others are left zero): sampled checks at
-    full size skip the products they do not look at.
+    full size skip the products they do not look at.  `utt_weights` [N] are
+    upstream gradients c_n of the utterance losses (Appendix B.1: the row sums of
+    G account for loss scaling): gradients are then those of sum_n c_n L_n, the
+    returned losses stay unweighted.
     """
     hidden = np.asarray(hidden, dtype=np.float64)
     W64 = np.asarray(W, dtype=np.float64)
@@ -335,6 +338,8 @@ def pruned_ctc_reference(hidden, W, bias, targets, input_lengths, target_lengths
         loss[n], flags[n], exact[n] = l, f, ex
         if dZ is None:
             continue
+        if utt_weights is not None:
+            dZ = dZ * float(utt_weights[n])
         if dH_for is None or n in dH_for:
             dH[n, :Tn] = dZ @ W64
         if want_dW:

@@ -35,6 +35,8 @@ class Problem(ctypes.Structure):
         ("dtype", ctypes.c_int32), ("blank_id", ctypes.c_int32),
         ("beam", ctypes.c_float),
         ("chunk", ctypes.c_int32), ("target_stride", ctypes.c_int32), ("gemm_path", ctypes.c_int32),
+        ("skip_dW", ctypes.c_int32), ("accumulate_dW", ctypes.c_int32),
+        ("utt_weights", ctypes.c_void_p),
     ]
 
 
@@ -126,9 +128,11 @@ def _ptr_i32(a: np.ndarray):
     return a.ctypes.data_as(ctypes.POINTER(ctypes.c_int32))
 
 
-def make_problem(N, T, D, V, dtype, blank_id, beam=0.0, chunk=0, target_stride=0, gemm_path=GEMM_AUTO) -> Problem:
+def make_problem(N, T, D, V, dtype, blank_id, beam=0.0, chunk=0, target_stride=0, gemm_path=GEMM_AUTO,
+                 skip_dW=False, accumulate_dW=False, utt_weights_ptr=None) -> Problem:
     return Problem(int(N), int(T), int(D), int(V), int(dtype), int(blank_id), float(beam), int(chunk),
-                   int(target_stride), int(gemm_path))
+                   int(target_stride), int(gemm_path), int(bool(skip_dW)), int(bool(accumulate_dW)),
+                   utt_weights_ptr)
 
 
 def workspace_bytes(problem: Problem, input_lengths, target_lengths) -> int:
@@ -146,7 +150,7 @@ def _dptr(t) -> Optional[int]:
 
 def pruned_ctc_fwd_bwd(hidden, W, bias, targets, input_lengths, target_lengths, blank_id, *, beam=0.0,
                        chunk=0, gemm_path=GEMM_AUTO, workspace=None, out=None, check_status=False,
-                       trace: Optional[Trace] = None):
+                       trace: Optional[Trace] = None, skip_dW=False, accumulate_dW=False, utt_weights=None):
     """Algorithm 1 on CUDA tensors.
 
     hidden [N,T,D], W [V,D], bias [V] or None (bf16 or fp32, same dtype), targets
@@ -155,6 +159,8 @@ def pruned_ctc_fwd_bwd(hidden, W, bias, targets, input_lengths, target_lengths, 
     dbias (or None), subset [1+sum U], K [1], relabeled [N,stride], flags [N],
     plus "workspace" (reusable) and "workspace_bytes".  `out` may carry
     preallocated tensors from an earlier call with the same shapes.
+    skip_dW: frozen head, dW is None.  accumulate_dW: add into out["dW"] / out["dbias"].
+    utt_weights: fp32 CUDA tensor [N] of upstream gradients of the utterance losses.
     """
     import torch
 
@@ -172,7 +178,10 @@ def pruned_ctc_fwd_bwd(hidden, W, bias, targets, input_lengths, target_lengths, 
     if targets.dtype != torch.int32 or not targets.is_contiguous():
         raise ValueError("targets must be a contiguous int32 CUDA tensor")
     stride = targets.shape[1]
-    prob = make_problem(N, T, D, V, dt, blank_id, beam, chunk, stride, gemm_path)
+    if utt_weights is not None and (utt_weights.dtype != torch.float32 or tuple(utt_weights.shape) != (N,)):
+        raise ValueError("utt_weights must be an fp32 CUDA tensor of shape [N]")
+    prob = make_problem(N, T, D, V, dt, blank_id, beam, chunk, stride, gemm_path, skip_dW, accumulate_dW,
+                        None if utt_weights is None else utt_weights.data_ptr())
     need = workspace_bytes(prob, il, tl)
     dev = hidden.device
     if workspace is None or workspace.numel() < need:
@@ -189,7 +198,7 @@ def pruned_ctc_fwd_bwd(hidden, W, bias, targets, input_lengths, target_lengths, 
     res = dict(
         loss=buf("loss", (N,), torch.float32),
         dH=buf("dH", (N, T, D), hidden.dtype),
-        dW=buf("dW", (V, D), hidden.dtype),
+        dW=None if skip_dW else buf("dW", (V, D), hidden.dtype),
         dbias=buf("dbias", (V,), hidden.dtype) if bias is not None else None,
         subset=buf("subset", (ksum,), torch.int32),
         K=buf("K", (1,), torch.int32),

@@ -386,7 +386,8 @@ __global__ void k_arc_flags(const float* __restrict__ va, const float* __restric
 __global__ void k_gamma(const float* __restrict__ alpha, const float* __restrict__ beta,
                         const float* __restrict__ S, long long ldS, const int* __restrict__ rel_all, int stride,
                         BatchMeta meta, int M, const int* __restrict__ flags,
-                        float* __restrict__ gamma, long long ldg, float* __restrict__ roww) {
+                        float* __restrict__ gamma, long long ldg, float* __restrict__ roww,
+                        const float* __restrict__ utt_weights) {
   const int m = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
   const int lane = threadIdx.x & 31;
   if (m >= M) return;
@@ -427,7 +428,7 @@ __global__ void k_gamma(const float* __restrict__ alpha, const float* __restrict
   }
 #pragma unroll
   for (int o = 16; o > 0; o >>= 1) gb += __shfl_xor_sync(0xffffffffu, gb, o);
-  if (lane == 0) { grow[0] = gb; roww[m] = 1.f; }
+  if (lane == 0) { grow[0] = gb; roww[m] = utt_weights ? utt_weights[n] : 1.f; }
 }
 
 // loss_n = sum_t lambda_t - log sum over alignments of exp(sum_t Z[t, pi_t])  (Eq. "ctc-factorization")
@@ -527,7 +528,7 @@ cudaError_t alignment_dp(const float* S, long long ldS, const int* relabeled, in
   const int warps = 8;
   k_gamma<<<(M + warps - 1) / warps, warps * 32, 0, stream>>>(buf.alpha, buf.beta, S, ldS, relabeled,
                                                                 target_stride, meta, M, utt_flags, gamma,
-                                                                ld_gamma, buf.roww);
+                                                                ld_gamma, buf.roww, buf.utt_weights);
   return cudaGetLastError();
 }
 

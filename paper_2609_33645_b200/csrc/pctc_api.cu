@@ -38,6 +38,7 @@ pctc_status_t make_plan(const pctc_problem_t* p, const int32_t* Tn, const int32_
   if (p->dtype != PCTC_BF16 && p->dtype != PCTC_FP32) return PCTC_ERR_UNSUPPORTED;
   if (p->gemm_path != PCTC_GEMM_AUTO && p->gemm_path != PCTC_GEMM_SIMT) return PCTC_ERR_INVALID_ARG;
   if (p->chunk < 0) return PCTC_ERR_INVALID_ARG;
+  if ((p->skip_dW | p->accumulate_dW) & ~1) return PCTC_ERR_INVALID_ARG;
   if (std::isnan(p->beam)) return PCTC_ERR_INVALID_ARG;
   long long M = 0, Usum = 0, cells = 0, mcells = 0;
   int Umax = 0;
@@ -226,7 +227,7 @@ pctc_status_t pruned_ctc_fwd_bwd_traced(const pctc_problem_t* p, const void* hid
     if (!trace->events || !trace->kinds || trace->capacity < 12 + 4 * pl.nchunks) return PCTC_ERR_INVALID_ARG;
     trace->used = 0;
   }
-  if (!hidden || !W || !loss || !dH || !dW || !workspace) return PCTC_ERR_INVALID_ARG;
+  if (!hidden || !W || !loss || !dH || (!dW && !p->skip_dW) || !workspace) return PCTC_ERR_INVALID_ARG;
   if (!targets && pl.Usum > 0) return PCTC_ERR_INVALID_ARG;
   if (workspace_bytes < pl.total) return PCTC_ERR_WORKSPACE_TOO_SMALL;
   if (((size_t)workspace & (ALIGN - 1)) || ((size_t)hidden & 15) || ((size_t)W & 15) || ((size_t)dH & 15) ||
@@ -312,6 +313,7 @@ pctc_status_t pruned_ctc_fwd_bwd_traced(const pctc_problem_t* p, const void* hid
   dp.alpha = (float*)(ws + pl.o_alpha);
   dp.beta = (float*)(ws + pl.o_beta);
   dp.roww = (float*)(ws + pl.o_roww);
+  dp.utt_weights = p->utt_weights;
   if (pl.beam) {
     dp.va = (float*)(ws + pl.o_va);
     dp.vb = (float*)(ws + pl.o_vb);
@@ -410,18 +412,19 @@ pctc_status_t pruned_ctc_fwd_bwd_traced(const pctc_problem_t* p, const void* hid
       PCTC_CUDA(run_gemm(pl.use_umma, pl.bf16, c, e, d_status, stream));
     }
     PCTC_MARK(PCTC_PHASE_DW);
-    {
+    if (!p->skip_dW) {
       Epilogue e;                      // rows of dW: dZ_c^T X
       e.kind = EPI_STORE_OUT;
       e.out = (char*)dW + (size_t)v0 * D * pl.elem;
       e.ld = D;
       e.out_is_bf16 = pl.bf16;
+      e.accumulate = p->accumulate_dW;
       GemmCall c{d_chunk, pl.chunk, true, d_X, D, true, Cc, D, M};
       PCTC_CUDA(run_gemm(pl.use_umma, pl.bf16, c, e, d_status, stream));
     }
     if (bias && dbias) {
       PCTC_MARK(PCTC_PHASE_DBIAS);
-      PCTC_CUDA(column_sums(d_chunk, pl.bf16, pl.chunk, M, Cc, dbias, pl.bf16, v0, stream));
+      PCTC_CUDA(column_sums(d_chunk, pl.bf16, pl.chunk, M, Cc, dbias, pl.bf16, v0, p->accumulate_dW != 0, stream));
     }
   }
   PCTC_MARK(PCTC_PHASE_FINISH);
@@ -499,6 +502,7 @@ pctc_status_t pruned_ctc_fwd_bwd_host(const pctc_problem_t* p, const void* hidde
   pctc_status_t st = host_layout(p, input_lengths, target_lengths, bias != nullptr, &h);
   if (st != PCTC_OK) return st;
   if (!hidden || !W || !loss || !dH || !dW || !device_scratch) return PCTC_ERR_INVALID_ARG;
+  if (p->skip_dW || p->accumulate_dW || p->utt_weights) return PCTC_ERR_UNSUPPORTED;   // device entry point only
   if (!targets && h.b_targets > 0) return PCTC_ERR_INVALID_ARG;
   if ((size_t)device_scratch & (ALIGN - 1)) return PCTC_ERR_INVALID_ARG;
   if (scratch_bytes < h.total) return PCTC_ERR_WORKSPACE_TOO_SMALL;

@@ -37,7 +37,7 @@ struct Epilogue {
   const int* Kdev = nullptr;    // device scalar K
   float2* partial = nullptr;    // [M, nsplit] (max, sum)
   int nsplit = 1;
-  int accumulate = 0;           // EPI_ACCUM_F32: add to the destination instead of overwriting
+  int accumulate = 0;           // EPI_ACCUM_F32 / EPI_STORE_OUT: add to the destination instead of overwriting
   int out_is_bf16 = 0;          // EPI_DLOGITS / EPI_STORE_OUT destination type
 };
 
@@ -95,7 +95,7 @@ cudaError_t gather_rows(const void* W, void* W_U, const int* U, const int* Kdev,
 
 // db[v0 + j] = sum_i chunk[i*ld + j]
 cudaError_t column_sums(const void* chunk, bool chunk_bf16, long long ld, int M, int cols,
-                        void* db, bool db_bf16, long long v0, cudaStream_t stream);
+                        void* db, bool db_bf16, long long v0, bool accumulate, cudaStream_t stream);
 
 // ---------------------------------------------------------------------------
 // Alignment dynamic program (Algorithm 1 lines 7-10; Section 3.3 for the beam)
@@ -113,6 +113,7 @@ struct DpBuffers {
   unsigned char* mask_b;      // same, backward sweep coordinates
   const long long* mcell0;    // [N] first flag byte of each utterance
   float* roww;         // [M]
+  const float* utt_weights;   // [N] upstream gradient of each utterance loss, or null (all 1)
 };
 
 // Largest trellis width the DP kernels cover.

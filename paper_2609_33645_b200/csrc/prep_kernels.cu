@@ -132,7 +132,7 @@ __global__ void k_gather_rows(const char* __restrict__ W, char* __restrict__ W_U
 // --- db_c = dZ_c^T 1 (Algorithm 1 line 16): fixed summation order, no atomics -------------------
 template <typename TIn, typename TOut>
 __global__ void k_column_sums(const TIn* __restrict__ chunk, long long ld, int M, int cols,
-                              TOut* __restrict__ db, long long v0) {
+                              TOut* __restrict__ db, long long v0, bool accumulate) {
   __shared__ float s_part[32][33];
   const int cx = threadIdx.x, ry = threadIdx.y;
   const int j = blockIdx.x * 32 + cx;
@@ -144,6 +144,7 @@ __global__ void k_column_sums(const TIn* __restrict__ chunk, long long ld, int M
   if (ry == 0 && j < cols) {
     float tot = 0.f;
     for (int r = 0; r < 32; ++r) tot += s_part[r][cx];
+    if (accumulate) tot += float(db[v0 + j]);
     db[v0 + j] = TOut(tot);
   }
 }
@@ -205,12 +206,12 @@ cudaError_t gather_rows(const void* W, void* W_U, const int* U, const int* Kdev,
 }
 
 cudaError_t column_sums(const void* chunk, bool chunk_bf16, long long ld, int M, int cols,
-                        void* db, bool db_bf16, long long v0, cudaStream_t stream) {
+                        void* db, bool db_bf16, long long v0, bool accumulate, cudaStream_t stream) {
   dim3 block(32, 32), grid((cols + 31) / 32);
   if (chunk_bf16 && db_bf16)
-    k_column_sums<<<grid, block, 0, stream>>>((const __nv_bfloat16*)chunk, ld, M, cols, (__nv_bfloat16*)db, v0);
+    k_column_sums<<<grid, block, 0, stream>>>((const __nv_bfloat16*)chunk, ld, M, cols, (__nv_bfloat16*)db, v0, accumulate);
   else if (!chunk_bf16 && !db_bf16)
-    k_column_sums<<<grid, block, 0, stream>>>((const float*)chunk, ld, M, cols, (float*)db, v0);
+    k_column_sums<<<grid, block, 0, stream>>>((const float*)chunk, ld, M, cols, (float*)db, v0, accumulate);
   else
     return cudaErrorInvalidValue;
   return cudaGetLastError();

@@ -118,7 +118,8 @@ __global__ void __launch_bounds__(NT) k_simt_gemm(const T* __restrict__ A, const
           float* dst = reinterpret_cast<float*>(e.out) + (long long)i * e.ld + j;
           *dst = e.accumulate ? (*dst + a) : a;
         } else if (EPI == EPI_STORE_OUT) {
-          reinterpret_cast<T*>(e.out)[(long long)i * e.ld + j] = T(a);
+          T* dst = reinterpret_cast<T*>(e.out) + (long long)i * e.ld + j;
+          *dst = e.accumulate ? T(float(*dst) + a) : T(a);
         }
       }
     }

@@ -541,7 +541,8 @@ k_umma_gemm(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
             fence_async_smem();                        // staged data visible to the TMA engine
             __syncwarp();
             if (lane == 0) {
-              if (EPI == EPI_ACCUM_F32 && a.e.accumulate) tma_reduce_add_2d(&tmC, stage, j0, row0_cta + q * 32);
+              if ((EPI == EPI_ACCUM_F32 || EPI == EPI_STORE_OUT) && a.e.accumulate)
+                tma_reduce_add_2d(&tmC, stage, j0, row0_cta + q * 32);
               else tma_store_2d(&tmC, stage, j0, row0_cta + q * 32);
               bulk_commit();
             }

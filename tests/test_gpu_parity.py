@@ -136,6 +136,39 @@ def test_two_calls_are_bitwise_identical_and_workspace_is_reusable(lib):
     torch.cuda.synchronize()
 
 
+@pytest.mark.parametrize("path", [SIMT, AUTO])
+def test_frozen_head_utterance_weights_and_accumulation(lib, path):
+    import torch
+    cfg = small("c3", V=8192 + 384, D=256, N=4, T_div=4, U_div=2)
+    batch = wl.make_batch(cfg, with_bias=True, permute_ids=True)
+    c = np.array([0.25, 1.0, 2.0, 0.5], dtype=np.float32)
+    ref = H.run_oracle(batch, utt_weights=c)
+    # weighted gradients, full outputs
+    full = H.run_gpu(lib, batch, gemm_path=path, utt_weights=c, chunk=2048)
+    H.assert_parity(full, ref, batch)
+    # frozen head: dH and dbias as before, dW not produced
+    frozen = H.run_gpu(lib, batch, gemm_path=path, utt_weights=c, chunk=2048, skip_dW=True)
+    assert frozen["dW"] is None
+    np.testing.assert_array_equal(frozen["dH"], full["dH"])
+    np.testing.assert_array_equal(frozen["dbias"], full["dbias"])
+    np.testing.assert_array_equal(frozen["loss"], full["loss"])
+    # accumulation over two micro-batches: the second call adds to dW / dbias of the first
+    dev = torch.device("cuda:0")
+    hidden = torch.from_numpy(batch.hidden).to(dev).to(torch.bfloat16)
+    W = torch.from_numpy(batch.W).to(dev).to(torch.bfloat16)
+    bias = torch.from_numpy(batch.bias).to(dev).to(torch.bfloat16)
+    targets = torch.from_numpy(batch.targets).to(dev)
+    cw = torch.from_numpy(c).to(dev)
+    args = (hidden, W, bias, targets, batch.input_lengths, batch.target_lengths, batch.blank)
+    out = lib.pruned_ctc_fwd_bwd(*args, gemm_path=path, chunk=2048, utt_weights=cw)
+    out = lib.pruned_ctc_fwd_bwd(*args, gemm_path=path, chunk=2048, utt_weights=cw, accumulate_dW=True,
+                                 workspace=out["workspace"], out=out)
+    torch.cuda.synchronize()
+    assert H.rel_fro(out["dW"].float().cpu().numpy(), 2.0 * ref["dW"]) <= 1e-2
+    assert H.rel_fro(out["dbias"].float().cpu().numpy(), 2.0 * ref["db"]) <= 1e-2
+    np.testing.assert_array_equal(out["dH"].float().cpu().numpy(), full["dH"])   # dH is never accumulated
+
+
 @pytest.mark.parametrize("a_mn", [False, True])
 @pytest.mark.parametrize("b_mn", [False, True])
 @pytest.mark.parametrize("m,n,k", [(128, 256, 64), (200, 264, 328), (1000, 520, 1032), (72, 8, 4096)])

@@ -163,6 +163,28 @@ def test_gradients_match_finite_differences():
             assert grad[idx] == pytest.approx(fd, rel=2e-6, abs=2e-8)
 
 
+def test_utterance_weights_are_upstream_gradients():
+    # gradients of sum_n c_n L_n by central differences; losses stay unweighted
+    rng = np.random.default_rng(6)
+    H, W, b, targets, Tn, tl = _small_batch(rng, N=3, T=8, D=4, V=9, blank=0)
+    c = np.array([0.5, -1.25, 3.0])
+    out = O.pruned_ctc_reference(H, W, b, targets, Tn, tl, 0, utt_weights=c)
+    plain = O.pruned_ctc_reference(H, W, b, targets, Tn, tl, 0)
+    np.testing.assert_array_equal(out["loss"], plain["loss"])
+
+    def total(Wx):
+        return float(np.dot(c, O.pruned_ctc_reference(H, Wx, b, targets, Tn, tl, 0, want_dW=False)["loss"]))
+
+    h = 1e-6
+    for idx in [(0, 0), (3, 2), (8, 1), (5, 3)]:
+        p, m = W.copy(), W.copy()
+        p[idx] += h
+        m[idx] -= h
+        assert out["dW"][idx] == pytest.approx((total(p) - total(m)) / (2 * h), rel=2e-6, abs=2e-8)
+    for n in range(3):
+        np.testing.assert_allclose(out["dH"][n], c[n] * plain["dH"][n], rtol=1e-13, atol=1e-15)
+
+
 def test_invariants_and_exclusions():
     rng = np.random.default_rng(9)
     H, W, b, targets, Tn, tl = _small_batch(rng, N=3, T=9, D=5, V=11)

@@ -204,6 +204,10 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--beam", type=float, default=0.0)
     ap.add_argument("--chunk", type=int, default=0)
+    ap.add_argument("--vocab", type=int, default=0, help="override V of the configuration (vocabulary sweep)")
+    ap.add_argument("--promise-k", action="store_true",
+                    help="pass max_K = the number of selected classes, counted on the host as a data loader "
+                         "would (default for the g* grid workloads)")
     ap.add_argument("--frozen-head", action="store_true",
                     help="skip dW (the LLM-CTC setting): 6 M D V FLOPs per step instead of 8")
     ap.add_argument("--e2e-steps", type=int, default=3)
@@ -211,6 +215,10 @@ def main():
     ap.add_argument("--cpu-frames", type=int, default=1024)
     args = ap.parse_args()
     cfg = wl.CONFIGS[args.config]
+    if args.vocab:
+        cfg = wl.reduced(cfg, V=args.vocab, name=f"{cfg.name}-V{args.vocab}")
+    if cfg.name.startswith("g"):
+        args.promise_k = True
 
     if args.impl == "reference":
         return run_reference(args, cfg)
@@ -249,13 +257,20 @@ def main():
     flops_per_step = (6.0 if args.frozen_head else 8.0) * M * D * V
 
     chunk = args.chunk or DEFAULT_CHUNK
+    max_K_pre = 0
+    if args.promise_k:
+        max_K_pre = 1 + int(np.unique(np.concatenate([batch.targets[n, : tl[n]] for n in range(N)])).size)
     prob = binding.make_problem(N, batch.T, D, V, binding.PCTC_BF16 if cfg.dtype == "bf16" else binding.PCTC_FP32,
-                                batch.blank, args.beam, chunk, batch.targets.shape[1])
+                                batch.blank, args.beam, chunk, batch.targets.shape[1], max_K=max_K_pre)
     ws_bytes = binding.workspace_bytes(prob, il, tl)
     chunk = args.chunk or DEFAULT_CHUNK
     nchunks = (V + chunk - 1) // chunk
     call = dict(beam=args.beam, chunk=chunk)
-    dev_call = dict(call, skip_dW=args.frozen_head)
+    max_K = 0
+    if args.promise_k:
+        toks = np.concatenate([batch.targets[n, : tl[n]] for n in range(N)])
+        max_K = 1 + int(np.unique(toks).size)
+    dev_call = dict(call, skip_dW=args.frozen_head, max_K=max_K)
 
     res = binding.pruned_ctc_fwd_bwd(hidden, W, None, targets, il, tl, batch.blank, check_status=True, **dev_call)
     torch.cuda.synchronize()
@@ -355,7 +370,7 @@ def main():
     out_bytes = (N * 4 + hidden.numel() * hidden.element_size()
                  + (0 if args.frozen_head else W.numel() * W.element_size()))
     prob_half = binding.make_problem(N, batch.T, D, V // 2 // 8 * 8, prob.dtype, batch.blank, args.beam, chunk,
-                                     batch.targets.shape[1])
+                                     batch.targets.shape[1], max_K=max_K_pre)
     ws_half = binding.workspace_bytes(prob_half, il, tl)
 
     # ---- the oracle on the host cores, on a bounded sample ----
@@ -372,7 +387,7 @@ def main():
         ms_per_step=ms_per_step, higher_is_better=True, scaling="weak", vs_baseline=None,
         dtype=cfg.dtype, data="synthetic",
         config=dict(workload=cfg.name, N=N, T_range=[cfg.T_lo, cfg.T_hi], D=D, V=V, M_frames=M,
-                    K_selected=int(res["K"].item()), beam=args.beam, chunk=chunk, frozen_head=args.frozen_head,
+                    K_selected=int(res["K"].item()), beam=args.beam, chunk=chunk, frozen_head=args.frozen_head, max_K=max_K,
                     l2="inputs larger than L2 (W and dW are %.2f GB each)" % (W.numel() * 2 / 1e9),
                     parallelism="independent utterance batches per GPU, no collective"),
         tflops=flops_all / (ms_per_step * 1e-3) / 1e12,

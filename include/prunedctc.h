@@ -46,6 +46,7 @@ typedef enum { PCTC_GEMM_AUTO = 0, PCTC_GEMM_SIMT = 1 } pctc_gemm_path_t;
 #define PCTC_UTT_INFEASIBLE 1 /* T_n < |y_n| + (adjacent equal pairs): no alignment exists  */
 #define PCTC_UTT_NONFINITE 2  /* loss not finite (NaN/Inf input, or empty retained lattice)  */
 #define PCTC_UTT_BAD_TARGET 4 /* a token equals blank_id or lies outside [0, V)              */
+#define PCTC_UTT_SUBSET_OVERFLOW 8 /* the batch has more selected classes than problem.max_K  */
 
 /*
  * The problem of Section 3.1 / Algorithm 1, line 1.
@@ -68,6 +69,12 @@ typedef struct {
                             computed nor touched (dW may be NULL); dH and dbias still are        */
   int32_t accumulate_dW; /* 1: dW and dbias are added to (gradient accumulation over
                             micro-batches) instead of overwritten                              */
+  int32_t max_K;         /* 0, or a promise K <= max_K (K = |U| is only known on the device; a
+                            data loader that holds the targets on the host knows it).  Sizes the
+                            [M, K] buffers by max_K instead of the bound 1 + sum U_n.  If the
+                            batch breaks the promise, nothing faults: every utterance is flagged
+                            PCTC_UTT_SUBSET_OVERFLOW, losses and gradients are zero, and the
+                            status word reads non-zero                                          */
   const float* utt_weights; /* device [N] or NULL: upstream gradient c_n of each utterance loss
                             (loss scaling, token-count normalisation; Appendix B.1, "row sums of
                             G"): gradients are those of sum_n c_n L_n; the returned losses stay

@@ -18,7 +18,7 @@ LIB_PATH = os.path.join(HERE, "libprunedctc.so")
 
 PCTC_BF16, PCTC_FP32 = 0, 1
 GEMM_AUTO, GEMM_SIMT = 0, 1
-UTT_INFEASIBLE, UTT_NONFINITE, UTT_BAD_TARGET = 1, 2, 4
+UTT_INFEASIBLE, UTT_NONFINITE, UTT_BAD_TARGET, UTT_SUBSET_OVERFLOW = 1, 2, 4, 8
 
 EXPORTS = ("pctc_workspace_bytes", "pruned_ctc_fwd_bwd", "pruned_ctc_fwd_bwd_traced", "pctc_gemm_bf16",
            "pctc_workspace_status", "pctc_status_string", "pctc_host_call_scratch_bytes",
@@ -35,7 +35,7 @@ class Problem(ctypes.Structure):
         ("dtype", ctypes.c_int32), ("blank_id", ctypes.c_int32),
         ("beam", ctypes.c_float),
         ("chunk", ctypes.c_int32), ("target_stride", ctypes.c_int32), ("gemm_path", ctypes.c_int32),
-        ("skip_dW", ctypes.c_int32), ("accumulate_dW", ctypes.c_int32),
+        ("skip_dW", ctypes.c_int32), ("accumulate_dW", ctypes.c_int32), ("max_K", ctypes.c_int32),
         ("utt_weights", ctypes.c_void_p),
     ]
 
@@ -129,10 +129,10 @@ def _ptr_i32(a: np.ndarray):
 
 
 def make_problem(N, T, D, V, dtype, blank_id, beam=0.0, chunk=0, target_stride=0, gemm_path=GEMM_AUTO,
-                 skip_dW=False, accumulate_dW=False, utt_weights_ptr=None) -> Problem:
+                 skip_dW=False, accumulate_dW=False, utt_weights_ptr=None, max_K=0) -> Problem:
     return Problem(int(N), int(T), int(D), int(V), int(dtype), int(blank_id), float(beam), int(chunk),
                    int(target_stride), int(gemm_path), int(bool(skip_dW)), int(bool(accumulate_dW)),
-                   utt_weights_ptr)
+                   int(max_K), utt_weights_ptr)
 
 
 def workspace_bytes(problem: Problem, input_lengths, target_lengths) -> int:
@@ -150,7 +150,8 @@ def _dptr(t) -> Optional[int]:
 
 def pruned_ctc_fwd_bwd(hidden, W, bias, targets, input_lengths, target_lengths, blank_id, *, beam=0.0,
                        chunk=0, gemm_path=GEMM_AUTO, workspace=None, out=None, check_status=False,
-                       trace: Optional[Trace] = None, skip_dW=False, accumulate_dW=False, utt_weights=None):
+                       trace: Optional[Trace] = None, skip_dW=False, accumulate_dW=False, utt_weights=None,
+                       max_K=0):
     """Algorithm 1 on CUDA tensors.
 
     hidden [N,T,D], W [V,D], bias [V] or None (bf16 or fp32, same dtype), targets
@@ -181,7 +182,7 @@ def pruned_ctc_fwd_bwd(hidden, W, bias, targets, input_lengths, target_lengths, 
     if utt_weights is not None and (utt_weights.dtype != torch.float32 or tuple(utt_weights.shape) != (N,)):
         raise ValueError("utt_weights must be an fp32 CUDA tensor of shape [N]")
     prob = make_problem(N, T, D, V, dt, blank_id, beam, chunk, stride, gemm_path, skip_dW, accumulate_dW,
-                        None if utt_weights is None else utt_weights.data_ptr())
+                        None if utt_weights is None else utt_weights.data_ptr(), max_K)
     need = workspace_bytes(prob, il, tl)
     dev = hidden.device
     if workspace is None or workspace.numel() < need:
@@ -195,6 +196,8 @@ def pruned_ctc_fwd_bwd(hidden, W, bias, targets, input_lengths, target_lengths, 
         return t
 
     ksum = int(tl.sum()) + 1
+    if max_K:
+        ksum = min(ksum, int(max_K))
     res = dict(
         loss=buf("loss", (N,), torch.float32),
         dH=buf("dH", (N, T, D), hidden.dtype),

@@ -93,7 +93,7 @@ __global__ void __launch_bounds__(W * 32) k_ctc_sweep(SweepArgs a) {
   if (tid == 0) { s_rep = 0; s_fin[0] = NEG_INF; s_fin[1] = NEG_INF; }
   if (tid < 2 * (W < 4 ? 4 : W)) (&s_wmax[0][0])[tid] = NEG_INF;
   __syncthreads();
-  if (a.flags[n] & 4) {                                            // bad target: excluded
+  if (a.flags[n] & (4 | 8)) {                                      // bad target or subset overflow: excluded
     if (dir == 0 && tid == 0 && MODE != MODE_MAX) a.loss[n] = 0.f;
     return;
   }

@@ -39,6 +39,7 @@ pctc_status_t make_plan(const pctc_problem_t* p, const int32_t* Tn, const int32_
   if (p->gemm_path != PCTC_GEMM_AUTO && p->gemm_path != PCTC_GEMM_SIMT) return PCTC_ERR_INVALID_ARG;
   if (p->chunk < 0) return PCTC_ERR_INVALID_ARG;
   if ((p->skip_dW | p->accumulate_dW) & ~1) return PCTC_ERR_INVALID_ARG;
+  if (p->max_K < 0) return PCTC_ERR_INVALID_ARG;
   if (std::isnan(p->beam)) return PCTC_ERR_INVALID_ARG;
   long long M = 0, Usum = 0, cells = 0, mcells = 0;
   int Umax = 0;
@@ -54,6 +55,8 @@ pctc_status_t make_plan(const pctc_problem_t* p, const int32_t* Tn, const int32_
   if (M > 0x7fffffffLL / 2 || Usum >= (1LL << 23) - 1) return PCTC_ERR_UNSUPPORTED;   // index in U packs into 23 bits
   pl->N = p->N; pl->T = p->T; pl->D = p->D; pl->V = p->V;
   pl->M = (int)M; pl->Usum = (int)Usum; pl->Kcap = (int)Usum + 1; pl->cells = cells; pl->mcells = mcells;
+  if ((long long)pl->Kcap > p->V) pl->Kcap = (int)p->V;                 // K <= V always
+  if (p->max_K > 0 && p->max_K < pl->Kcap) pl->Kcap = p->max_K;        // the caller's promise
   pl->Lmax = 2 * Umax + 1;
   if (pl->Lmax > dp_max_states()) return PCTC_ERR_UNSUPPORTED;
   pl->bf16 = (p->dtype == PCTC_BF16);
@@ -328,7 +331,7 @@ pctc_status_t pruned_ctc_fwd_bwd_traced(const pctc_problem_t* p, const void* hid
   // ---- Algorithm 1 lines 2-3: subset and relabelling ----
   PCTC_CUDA(cudaMemsetAsync(d_U, 0xFF, (size_t)pl.Kcap * 4, stream));   // entries past K read -1
   PCTC_CUDA(subset_and_relabel(targets, p->target_stride, bm.U_n, N, V, p->blank_id, d_bitmap, d_wrank, d_vmap,
-                               d_U, d_K, d_rel, d_flags, stream));
+                               d_U, d_K, d_rel, d_flags, pl.Kcap, d_status, stream));
   // ---- line 4: stack the valid frames ----
   PCTC_CUDA(stack_frames(hidden, d_X, N, pl.T, D, pl.elem, bm.row_utt, bm.row0, M, stream));
 

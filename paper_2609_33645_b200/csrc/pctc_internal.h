@@ -79,7 +79,7 @@ struct BatchMeta {              // device arrays describing the batch
 cudaError_t subset_and_relabel(const int* targets, int target_stride, const int* U_n_dev, int N,
                                long long V, int blank, unsigned* bitmap, int* word_rank,
                                int* vmap, int* U_out, int* K_out, int* relabeled, int* utt_flags,
-                               cudaStream_t stream);
+                               int cap, int* status, cudaStream_t stream);   // cap: capacity of U_out
 
 // Algorithm 1 line 4: X[row0[n] + t] = hidden[n, t], t < T_n.
 cudaError_t stack_frames(const void* hidden, void* X, int N, int T, int D, int elem_bytes,

@@ -30,8 +30,9 @@ __global__ void k_mark_targets(const int* __restrict__ targets, int stride, cons
 // --- rank the set bits: U = blank, then ascending ids; vmap[id] = position in U ----------------
 // One CTA: each thread owns a contiguous run of bitmap words, a block-wide exclusive scan of the
 // per-thread popcounts gives every run its first rank.
+// Ranks past `cap` are dropped (their classes stay unmapped): the caller then flags the batch.
 __global__ void k_rank_subset(const unsigned* __restrict__ bitmap, int nwords, int blank, int* word_rank,
-                              int* vmap, int* U_out, int* K_out) {
+                              int* vmap, int* U_out, int* K_out, int cap, int* utt_flags, int N, int* status) {
   __shared__ int s_scan[1024];
   const int tid = threadIdx.x, nt = blockDim.x;
   const int per = (nwords + nt - 1) / nt;
@@ -54,16 +55,22 @@ __global__ void k_rank_subset(const unsigned* __restrict__ bitmap, int nwords, i
       int b = __ffs(bits) - 1;
       bits &= bits - 1;
       int id = (w << 5) + b;
-      U_out[1 + rank] = id;
-      vmap[id] = 1 + rank;
+      if (1 + rank < cap) {
+        U_out[1 + rank] = id;
+        vmap[id] = 1 + rank;
+      }
       ++rank;
     }
   }
+  const int K = 1 + s_scan[nt - 1];
   if (tid == nt - 1) {
-    *K_out = 1 + s_scan[tid];
+    *K_out = min(K, cap);
     U_out[0] = blank;
     vmap[blank] = 0;
+    if (K > cap && status) atomicCAS(status, 0, 0x100);
   }
+  if (K > cap)                                   // more selected classes than the buffers hold
+    for (int n = tid; n < N; n += nt) atomicOr(&utt_flags[n], 8);
 }
 
 // --- Algorithm 1 line 3: relabel ----------------------------------------------------------------
@@ -167,7 +174,7 @@ __global__ void k_lse_combine(const float2* __restrict__ partial, int nsplit, in
 cudaError_t subset_and_relabel(const int* targets, int target_stride, const int* U_n_dev, int N,
                                long long V, int blank, unsigned* bitmap, int* word_rank,
                                int* vmap, int* U_out, int* K_out, int* relabeled, int* utt_flags,
-                               cudaStream_t stream) {
+                               int cap, int* status, cudaStream_t stream) {
   const int nwords = (int)((V + 31) / 32);
   cudaError_t e;
   if ((e = cudaMemsetAsync(bitmap, 0, (size_t)nwords * 4, stream)) != cudaSuccess) return e;
@@ -177,7 +184,8 @@ cudaError_t subset_and_relabel(const int* targets, int target_stride, const int*
   const int blocks = (total + 255) / 256;
   if (total > 0)
     k_mark_targets<<<blocks, 256, 0, stream>>>(targets, target_stride, U_n_dev, N, V, blank, bitmap, utt_flags);
-  k_rank_subset<<<1, 1024, 0, stream>>>(bitmap, nwords, blank, word_rank, vmap, U_out, K_out);
+  k_rank_subset<<<1, 1024, 0, stream>>>(bitmap, nwords, blank, word_rank, vmap, U_out, K_out, cap, utt_flags, N,
+                                        status);
   if (total > 0)
     k_relabel<<<blocks, 256, 0, stream>>>(targets, target_stride, U_n_dev, N, V, blank, vmap, relabeled);
   return cudaGetLastError();
@@ -280,6 +288,7 @@ extern "C" pctc_status_t pctc_subset_relabel_noalloc(const int32_t* targets, con
   // subset_and_relabel clears the bitmap, the class map and the flags itself: nothing of an
   // earlier call survives into this one.
   cudaError_t e = subset_and_relabel(targets, target_stride, target_lengths, N, V, blank_id, bitmap, word_rank, vmap,
-                                     subset_out, K_out, relabeled_out, utt_flags, (cudaStream_t)stream);
+                                     subset_out, K_out, relabeled_out, utt_flags, 0x7fffffff, nullptr,
+                                     (cudaStream_t)stream);
   return e == cudaSuccess ? PCTC_OK : PCTC_ERR_CUDA;
 }

@@ -72,21 +72,24 @@ struct SharedTail {   // barriers and flags
 };
 
 // Dynamic shared memory after the operand ring, by epilogue kind:
-//   store staging  4 warps x 4 KB, 128-byte-swizzled boxes for the TMA stores (dlogits, dX, dW)
+//   store staging  4 warps x 2 buffers: 32 rows x 64 B boxes (bf16: dlogits, dW) or 32 rows x 128 B
+//                  boxes (fp32: dX), swizzled, written out by TMA stores while the other buffer fills
 //   SharedTail
 //   bias           4 warps x BN floats (lse, subset, dlogits)
-//   list           4 warps x BN packed (index in U << 8 | column) of the tile's selected classes (dlogits)
-constexpr int STAGE_BOX_BYTES = 4096;
+//   list           4 warps x (BN indices in U, -1 if the column's class is not selected, + 8 group masks) (dlogits)
+constexpr int stage_box_bytes(int epi) { return epi == EPI_ACCUM_F32 ? 4096 : 2048; }   // one staged box
+constexpr int stage_warp_bytes(int epi) { return 2 * stage_box_bytes(epi); }              // double-buffered
 constexpr bool epi_uses_tma_store(int epi) { return epi == EPI_DLOGITS || epi == EPI_ACCUM_F32 || epi == EPI_STORE_OUT; }
 constexpr bool epi_uses_bias(int epi) { return epi == EPI_LSE_PARTIAL || epi == EPI_SUBSET_LOGP || epi == EPI_DLOGITS; }
 constexpr size_t ring_bytes(int ctas) { return (size_t)stages_of(ctas) * (A_STAGE_BYTES + b_stage_bytes(ctas)); }
 static_assert(ring_bytes(1) == ring_bytes(2), "both tile modes use the same operand ring size");
 constexpr size_t RING_BYTES = ring_bytes(1);
 constexpr size_t off_stage() { return RING_BYTES; }
-constexpr size_t off_tail(int epi) { return RING_BYTES + (epi_uses_tma_store(epi) ? 4 * STAGE_BOX_BYTES : 0); }
+constexpr size_t off_tail(int epi) { return RING_BYTES + (epi_uses_tma_store(epi) ? 4 * stage_warp_bytes(epi) : 0); }
 constexpr size_t off_bias(int epi) { return off_tail(epi) + 256; }
 constexpr size_t off_list(int epi) { return off_bias(epi) + (epi_uses_bias(epi) ? 4 * BN * 4 : 0); }
-constexpr size_t smem_bytes(int epi) { return 1024 + off_list(epi) + (epi == EPI_DLOGITS ? 4 * BN * 4 : 0); }
+constexpr int LIST_WORDS = BN + 32;
+constexpr size_t smem_bytes(int epi) { return 1024 + off_list(epi) + (epi == EPI_DLOGITS ? 4 * LIST_WORDS * 4 : 0); }
 static_assert(sizeof(SharedTail) <= 256, "tail layout");
 
 // ---------------------------------------------------------------------------------------------
@@ -152,7 +155,7 @@ __device__ __forceinline__ void tma_reduce_add_2d(const CUtensorMap* map, const 
                : "memory");
 }
 __device__ __forceinline__ void bulk_commit() { asm volatile("cp.async.bulk.commit_group;" ::: "memory"); }
-__device__ __forceinline__ void bulk_wait_read0() { asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory"); }
+__device__ __forceinline__ void bulk_wait_read1() { asm volatile("cp.async.bulk.wait_group.read 1;" ::: "memory"); }
 __device__ __forceinline__ void bulk_wait0() { asm volatile("cp.async.bulk.wait_group 0;" ::: "memory"); }
 __device__ __forceinline__ void fence_async_smem() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
 
@@ -232,13 +235,25 @@ __device__ __forceinline__ void tmem_ld32(unsigned taddr, float* v) {
 #pragma unroll
   for (int i = 0; i < 32; ++i) v[i] = __uint_as_float(r[i]);
 }
-__device__ __forceinline__ float tmem_ld1(unsigned taddr) {
-  unsigned r;
-  asm volatile("tcgen05.ld.sync.aligned.32x32b.x1.b32 {%0}, [%1];" : "=r"(r) : "r"(taddr) : "memory");
-  asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
-  return __uint_as_float(r);
+// The same load without the wait: the registers are valid only after tmem_wait_ld() and must be
+// read through tmem_regs_to_float() (volatile moves that stay behind the wait).
+__device__ __forceinline__ void tmem_ld32_issue(unsigned taddr, unsigned* r) {
+  asm volatile(
+      "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
+      "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
+      "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];"
+      : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]),
+        "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]),
+        "=r"(r[16]), "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]),
+        "=r"(r[24]), "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
+      : "r"(taddr)
+      : "memory");
 }
-
+__device__ __forceinline__ void tmem_wait_ld() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
+__device__ __forceinline__ void tmem_regs_to_float(const unsigned* r, float* v) {
+#pragma unroll
+  for (int i = 0; i < 32; ++i) asm volatile("mov.b32 %0, %1;" : "=f"(v[i]) : "r"(r[i]));
+}
 __device__ __forceinline__ float ex2(float x) {
   float y;
   asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
@@ -429,9 +444,12 @@ k_umma_gemm(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
     const int q = warp & 3;                  // tensor-memory lane quarter this warp may read
     const int r = q * 32 + lane;             // accumulator row of this thread
     float* sb = (float*)(smem + off_bias(EPI)) + ew * BN;
-    unsigned* sl = (unsigned*)(smem + off_list(EPI)) + ew * BN;
-    unsigned char* stage = smem + off_stage() + ew * STAGE_BOX_BYTES;   // this warp's store staging box
-    const unsigned swz = (unsigned)(lane & 7);                           // 128-byte swizzle of the staged row
+    int* sj = (int*)(smem + off_list(EPI)) + ew * LIST_WORDS;            // index in U of each tile column, or -1
+    unsigned* sg = (unsigned*)sj + BN;                                    // one mask of selected columns per 32
+    unsigned char* stage = smem + off_stage() + ew * stage_warp_bytes(EPI);   // this warp's two staging boxes
+    const unsigned swz = (unsigned)(lane & 7);          // 128-byte swizzle of a staged 128-byte row (fp32 boxes)
+    const unsigned swz64 = (unsigned)((lane >> 1) & 3); // 64-byte swizzle of a staged 64-byte row (bf16 boxes)
+    unsigned nbox = 0;                                  // boxes stored so far by this warp (buffer parity)
     unsigned it = 0;
     bool ok = true;
     for (int u = group; u < units && ok; u += ngroups) {
@@ -448,9 +466,9 @@ k_umma_gemm(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
       for (int nt = nt0; nt < nt0 + cnt && ok; ++nt, ++it) {
         const unsigned acc = it & 1u, aph = (it >> 1) & 1u;
         const int n0 = nt * BN;
-        int nsel = 0;
         // ---- warp-private staging of per-column data (overlaps the MMAs of this tile) ----
-        if (EPI == EPI_LSE_PARTIAL || EPI == EPI_DLOGITS || EPI == EPI_SUBSET_LOGP) {
+        const bool has_bias = a.e.bias != nullptr;        // without a bias the staged zeros are never read
+        if ((EPI == EPI_LSE_PARTIAL || EPI == EPI_DLOGITS || EPI == EPI_SUBSET_LOGP) && has_bias) {
           const __nv_bfloat16* bias = (const __nv_bfloat16*)a.e.bias;
 #pragma unroll
           for (int c = lane; c < BN; c += 32) {
@@ -464,12 +482,13 @@ k_umma_gemm(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
           }
         }
         if (EPI == EPI_DLOGITS) {
+#pragma unroll
           for (int c0 = 0; c0 < BN; c0 += 32) {
             const int j = n0 + c0 + lane;
             const int jj = (j < n_eff) ? a.e.vmap[a.e.v0 + j] : -1;
             const unsigned mask = __ballot_sync(0xffffffffu, jj >= 0);
-            if (jj >= 0) sl[nsel + __popc(mask & ((1u << lane) - 1u))] = ((unsigned)jj << 8) | (unsigned)(c0 + lane);
-            nsel += __popc(mask);
+            sj[c0 + lane] = jj;
+            if (lane == 0) sg[c0 >> 5] = mask;
           }
         }
         __syncwarp();
@@ -483,31 +502,53 @@ k_umma_gemm(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
 
         if (epi_uses_tma_store(EPI)) {
           // ---- staged epilogues: the warp's 32 rows go out as 128-byte-wide boxes through TMA ----
-          constexpr int BOX_COLS = (EPI == EPI_ACCUM_F32) ? 32 : 64;   // fp32 : bf16
-          int e_idx = 0;
+          // One box per 32 accumulator columns: 32 rows x 128 B (fp32) or 32 rows x 64 B (bf16).  Two
+          // buffers alternate, so a box is filled while the TMA engine still reads the previous one.
+          unsigned ra[32], rb[32];                    // the 32-column groups, loaded one group ahead
+          tmem_ld32_issue(taddr, ra);
 #pragma unroll 1
-          for (int cb = 0; cb < BN / BOX_COLS; ++cb) {
-            const int j0 = n0 + cb * BOX_COLS;
-            if (j0 >= n_eff) break;                   // warp-uniform
-            if (lane == 0) bulk_wait_read0();   // the previous box has left the staging buffer
-            __syncwarp();
-            unsigned char* row = stage + lane * 128;
-            if (EPI == EPI_ACCUM_F32) {
+          for (int cg = 0; cg < BN / 32; cg += 2) {
+#pragma unroll
+            for (int half = 0; half < 2; ++half) {
+              const int g0 = (cg + half) * 32;        // first tile column of this group
+              const int j0 = n0 + g0;
+              if (j0 >= n_eff) break;                 // warp-uniform
+              tmem_wait_ld();
               float v[32];
-              tmem_ld32(taddr + cb * 32, v);
+              tmem_regs_to_float(half ? rb : ra, v);
+              if (g0 + 32 < BN && j0 + 32 < n_eff)    // next group: the load flies while this one is processed
+                tmem_ld32_issue(taddr + g0 + 32, half ? ra : rb);
+              if (lane == 0) bulk_wait_read1();        // the box stored two groups ago has left its buffer
+              __syncwarp();
+              unsigned char* row = stage + (nbox & 1u) * stage_box_bytes(EPI) + lane * (EPI == EPI_ACCUM_F32 ? 128 : 64);
+              if (EPI == EPI_ACCUM_F32) {
 #pragma unroll
-              for (int c4 = 0; c4 < 8; ++c4)
-                *reinterpret_cast<float4*>(row + (((unsigned)c4 ^ swz) << 4)) =
-                    make_float4(v[c4 * 4], v[c4 * 4 + 1], v[c4 * 4 + 2], v[c4 * 4 + 3]);
-            } else {
-#pragma unroll
-              for (int half = 0; half < 2; ++half) {
-                float v[32];
-                tmem_ld32(taddr + cb * 64 + half * 32, v);
+                for (int c4 = 0; c4 < 8; ++c4)
+                  *reinterpret_cast<float4*>(row + (((unsigned)c4 ^ swz) << 4)) =
+                      make_float4(v[c4 * 4], v[c4 * 4 + 1], v[c4 * 4 + 2], v[c4 * 4 + 3]);
+              } else {
                 if (EPI == EPI_DLOGITS) {
+                  if (has_bias) {
 #pragma unroll
-                  for (int c = 0; c < 32; ++c)
-                    v[c] = w * ex2(fmaf(v[c] + sb[cb * 64 + half * 32 + c], LOG2E, -lam2));
+                    for (int c = 0; c < 32; ++c) v[c] += sb[g0 + c];
+                  }
+#pragma unroll
+                  for (int c = 0; c < 32; ++c) v[c] = ex2(fmaf(v[c], LOG2E, -lam2));     // p = exp(z - lambda)
+                  if (sg[g0 >> 5] != 0u) {
+                    // the group holds selected classes: subtract their occupancy in fp32, before the
+                    // rounding to bf16; the loads are issued together, the unselected ones predicated off
+                    float g[32];
+#pragma unroll
+                    for (int c = 0; c < 32; ++c) {
+                      const int jj = sj[g0 + c];
+                      g[c] = (jj >= 0 && row_ok) ? a.e.gamma[(long long)i * a.e.ld_gamma + jj] : 0.f;
+                    }
+#pragma unroll
+                    for (int c = 0; c < 32; ++c) v[c] = w * (v[c] - g[c]);
+                  } else {
+#pragma unroll
+                    for (int c = 0; c < 32; ++c) v[c] *= w;
+                  }
                 }
 #pragma unroll
                 for (int c8 = 0; c8 < 4; ++c8) {
@@ -517,36 +558,22 @@ k_umma_gemm(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
                   __nv_bfloat162 p2 = __floats2bfloat162_rn(v[c8 * 8 + 4], v[c8 * 8 + 5]);
                   __nv_bfloat162 p3 = __floats2bfloat162_rn(v[c8 * 8 + 6], v[c8 * 8 + 7]);
                   o.x = *(unsigned*)&p0; o.y = *(unsigned*)&p1; o.z = *(unsigned*)&p2; o.w = *(unsigned*)&p3;
-                  *reinterpret_cast<uint4*>(row + (((unsigned)(half * 4 + c8) ^ swz) << 4)) = o;
+                  *reinterpret_cast<uint4*>(row + (((unsigned)c8 ^ swz64) << 4)) = o;
                 }
               }
-              if (EPI == EPI_DLOGITS) {
-                // selected classes of this box: subtract the occupancy in fp32, before the rounding to bf16
-                while (e_idx < nsel) {
-                  const unsigned ent = sl[e_idx];
-                  const int col = (int)(ent & 0xffu);
-                  if (col >= cb * 64 + 64) break;       // warp-uniform: the list is in ascending column order
-                  ++e_idx;
-                  const float z = tmem_ld1(taddr + col);
-                  if (row_ok) {
-                    const float pz = ex2(fmaf(z + sb[col], LOG2E, -lam2));
-                    const float g = a.e.gamma[(long long)i * a.e.ld_gamma + (int)(ent >> 8)];
-                    const unsigned cbx = (unsigned)(col - cb * 64) * 2u;    // byte offset inside the 128-byte row
-                    *reinterpret_cast<__nv_bfloat16*>(row + ((((cbx >> 4) ^ swz) << 4) | (cbx & 15u))) =
-                        __float2bfloat16_rn(w * (pz - g));
-                  }
-                }
+              fence_async_smem();                      // staged data visible to the TMA engine
+              __syncwarp();
+              if (lane == 0) {
+                const void* box = stage + (nbox & 1u) * stage_box_bytes(EPI);
+                if ((EPI == EPI_ACCUM_F32 || EPI == EPI_STORE_OUT) && a.e.accumulate)
+                  tma_reduce_add_2d(&tmC, box, j0, row0_cta + q * 32);
+                else tma_store_2d(&tmC, box, j0, row0_cta + q * 32);
+                bulk_commit();
               }
-            }
-            fence_async_smem();                        // staged data visible to the TMA engine
-            __syncwarp();
-            if (lane == 0) {
-              if ((EPI == EPI_ACCUM_F32 || EPI == EPI_STORE_OUT) && a.e.accumulate)
-                tma_reduce_add_2d(&tmC, stage, j0, row0_cta + q * 32);
-              else tma_store_2d(&tmC, stage, j0, row0_cta + q * 32);
-              bulk_commit();
+              ++nbox;
             }
           }
+          tmem_wait_ld();     // nothing of this tile is in flight when the accumulator is released
         }
 
 #pragma unroll 1
@@ -567,13 +594,13 @@ k_umma_gemm(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
               float* dst = (float*)a.e.out + (long long)i * a.e.ld + j0;
 #pragma unroll
               for (int c = 0; c < 32; ++c)
-                if (j0 + c < n_eff) dst[c] = v[c] + sb[cg * 32 + c] - lam;
+                if (j0 + c < n_eff) dst[c] = v[c] + (has_bias ? sb[cg * 32 + c] : 0.f) - lam;
             }
           } else if (EPI == EPI_LSE_PARTIAL) {
             float gmax = -CUDART_INF_F;
 #pragma unroll
             for (int c = 0; c < 32; ++c) {
-              v[c] = (j0 + c < n_eff) ? (v[c] + sb[cg * 32 + c]) * LOG2E : -CUDART_INF_F;
+              v[c] = (j0 + c < n_eff) ? (has_bias ? v[c] + sb[cg * 32 + c] : v[c]) * LOG2E : -CUDART_INF_F;
               gmax = fmaxf(gmax, v[c]);
             }
             if (gmax > run_max2) {
@@ -639,9 +666,11 @@ bool make_map(CUtensorMap* map, const void* base, unsigned long long inner, unsi
   cuuint64_t strides[1] = {ld * (fp32 ? 4 : 2)};
   cuuint32_t box[2] = {box_inner, box_rows};
   cuuint32_t estr[2] = {1, 1};
+  const CUtensorMapSwizzle swizzle =
+      (box_inner * (fp32 ? 4u : 2u) == 64u) ? CU_TENSOR_MAP_SWIZZLE_64B : CU_TENSOR_MAP_SWIZZLE_128B;
   return fn(map, fp32 ? CU_TENSOR_MAP_DATA_TYPE_FLOAT32 : CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2,
             const_cast<void*>(base), dims, strides, box, estr,
-            CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+            CU_TENSOR_MAP_INTERLEAVE_NONE, swizzle, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
             CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
@@ -730,13 +759,13 @@ cudaError_t umma_gemm(const __nv_bfloat16* A, long long lda, bool a_mn_major,
   alignas(64) CUtensorMap tmA, tmB, tmC;
   bool ok = true;
   tmC = CUtensorMap{};
-  // output boxes of the staged epilogues: 32 rows x 128 bytes, clipped to the [m, n] extent
+  // output boxes of the staged epilogues: 32 rows x 32 columns, clipped to the [m, n] extent
   if (e.kind == EPI_ACCUM_F32) {
     if ((e.ld % 4) || ((size_t)e.out & 15)) return cudaErrorInvalidValue;
     ok = ok && make_map(&tmC, e.out, (unsigned long long)n, (unsigned long long)m, (unsigned long long)e.ld, 32, 32, true);
   } else if (e.kind == EPI_DLOGITS || e.kind == EPI_STORE_OUT) {
     if ((e.ld % 8) || ((size_t)e.out & 15)) return cudaErrorInvalidValue;
-    ok = ok && make_map(&tmC, e.out, (unsigned long long)n, (unsigned long long)m, (unsigned long long)e.ld, 64, 32);
+    ok = ok && make_map(&tmC, e.out, (unsigned long long)n, (unsigned long long)m, (unsigned long long)e.ld, 32, 32);
   }
   if (!a_mn_major) ok = ok && make_map(&tmA, A, (unsigned long long)k, (unsigned long long)m, lda, BK, BM);
   else ok = ok && make_map(&tmA, A, (unsigned long long)m, (unsigned long long)k, lda, 64, BK);

@@ -56,6 +56,16 @@ CONFIGS = {
                  U_lo=100, U_hi=300, zipf_s=1.1, rms_norm=True, seed=1004),
     "c5": Config("c5", N=4, T_lo=1500, T_hi=3000, D=5120, V=151936, dtype="bf16",
                  U_lo=300, U_hi=600, zipf_s=1.0, rms_norm=True, seed=1005),
+    # The paper's own resource benchmark (Appendix C.2): utterances of exactly 100 encoder frames,
+    # 160 / 320 / 640 of them (16k / 32k / 64k frames), Zipformer-M head width, vocabulary swept
+    # from 500 to 180,000 (use `reduced(cfg, V=...)` for the sweep).  Transcript lengths are not
+    # stated; 10-30 tokens is about four seconds of speech at the usual subword rates.
+    "g16k": Config("g16k", N=160, T_lo=100, T_hi=100, D=512, V=180000, dtype="bf16",
+                   U_lo=10, U_hi=30, zipf_s=1.1, seed=1016),
+    "g32k": Config("g32k", N=320, T_lo=100, T_hi=100, D=512, V=180000, dtype="bf16",
+                   U_lo=10, U_hi=30, zipf_s=1.1, seed=1032),
+    "g64k": Config("g64k", N=640, T_lo=100, T_hi=100, D=512, V=180000, dtype="bf16",
+                   U_lo=10, U_hi=30, zipf_s=1.1, seed=1064),
 }
 
 

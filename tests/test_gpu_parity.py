@@ -186,3 +186,26 @@ def test_tensor_core_contraction_all_operand_layouts(lib, a_mn, b_mn, m, n, k):
         C = lib.gemm_bf16(Ad, Bd, m, n, k, a_mn, b_mn, gemm_path=path).cpu().double()
         err = (C - ref).abs().max().item()
         assert err <= 2e-3 * (k ** 0.5), (path, err)
+
+
+def test_max_K_promise_kept_and_broken(lib):
+    cfg = small("c2", V=4096, D=64, N=6, T_div=10, U_div=4)
+    batch = wl.make_batch(cfg, permute_ids=True)
+    ref = H.run_oracle(batch)
+    K = ref["K"]
+    kept = H.run_gpu(lib, batch, max_K=K)                 # exact promise: same result, smaller buffers
+    H.assert_parity(kept, ref, batch)
+    assert kept["workspace_bytes"] < H.run_gpu(lib, batch)["workspace_bytes"]
+    broken = H.run_gpu(lib, batch, max_K=K - 3, check_status=False)   # promise broken: flagged, nothing faults
+    assert np.all(broken["flags"] & 8)
+    assert np.all(broken["loss"] == 0) and np.all(broken["dH"] == 0) and np.all(broken["dW"] == 0)
+    assert int(broken["K"][0]) == K - 3
+    np.testing.assert_array_equal(broken["subset"][: K - 3], ref["U"][: K - 3])
+
+
+def test_paper_grid_shape_many_short_utterances(lib):
+    # the paper's benchmark grid: every utterance exactly 100 frames, many utterances, D = 512
+    cfg = wl.reduced(wl.CONFIGS["g16k"], V=8192, N=24, name="g-small")
+    batch = wl.make_batch(cfg, permute_ids=True)
+    gpu = H.run_gpu(lib, batch)
+    H.assert_parity(gpu, H.run_oracle(batch), batch)

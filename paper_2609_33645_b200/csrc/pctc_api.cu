@@ -377,7 +377,8 @@ pctc_status_t pruned_ctc_fwd_bwd_traced(const pctc_problem_t* p, const void* hid
     e.nsplit = pl.use_umma ? umma_lse_splits(M, (int)V) : 32;
     GemmCall c{d_X, D, false, W, D, false, M, (int)V, D};
     PCTC_CUDA(run_gemm(pl.use_umma, pl.bf16, c, e, d_status, stream));
-    PCTC_CUDA(lse_combine(d_partial, e.nsplit, M, d_lambda, stream));
+    PCTC_CUDA(lse_combine(d_partial, pl.use_umma ? umma_lse_partials_per_split(D) * e.nsplit : e.nsplit, M, d_lambda,
+                          stream));
   }
   PCTC_CUDA(cudaStreamWaitEvent(stream, aux.join, 0));
   PCTC_CUDA(finalize_loss(d_lambda, bm, N, loss, d_flags, dp.roww, stream));

@@ -58,7 +58,9 @@ cudaError_t umma_gemm(const __nv_bfloat16* A, long long lda, bool a_mn_major,
                       const __nv_bfloat16* B, long long ldb, bool b_mn_major,
                       int m, int n, int k, const Epilogue& e, int* status, cudaStream_t stream);
 bool umma_available();   // the driver entry point for tensor maps could be resolved
-int umma_lse_splits(int m, int n);   // column splits (<= 64) for EPI_LSE_PARTIAL on this device
+int umma_lse_splits(int m, int n);   // column splits (<= 32) for EPI_LSE_PARTIAL on this device
+int umma_lse_partials_per_split(int k);   // the kernel writes this many partials per split (1 or 2):
+                                          // partial[(i*nsplit + sp)*pps + h]
 
 // Combine LSE partials: lambda[i] = log sum over splits.
 cudaError_t lse_combine(const float2* partial, int nsplit, int M, float* lambda, cudaStream_t stream);

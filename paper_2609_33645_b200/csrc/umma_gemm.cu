@@ -8,12 +8,13 @@
 // memory and runs its own epilogue.  B then crosses L2 -> shared memory once per pair instead of
 // once per CTA, and the freed shared memory deepens the ring to six stages.
 //
-// One persistent CTA per SM, 192 threads in three roles:
+// One persistent CTA per SM, 320 threads in three roles:
 //   warp 0      TMA producer: 128-byte-swizzled operand tiles into a 4-stage ring
 //   warp 1      MMA issuer: tcgen05.mma 128x256x16 from shared-memory descriptors
 //               into one of two 256-column accumulators in tensor memory
-//   warps 2..5  epilogue: tcgen05.ld (one accumulator row per thread), the fused
-//               arithmetic, global stores; runs while the next tile's MMAs issue
+//   warps 2..9  epilogue: tcgen05.ld (one accumulator row per thread; two warps per
+//               tensor-memory lane quarter, 128 columns each), the fused arithmetic,
+//               stores; runs while the next tile's MMAs issue
 // Operands may be K-major (k contiguous) or MN-major (the transposed storage),
 // chosen at run time through the descriptors, so that dX += dZ W and
 // dW = dZ^T X need no transposed copies.
@@ -42,10 +43,17 @@ namespace {
 
 constexpr int BM = 128, BN = 256, BK = 64;
 constexpr int MAX_STAGES = 6;
-constexpr int stages_of(int ctas) { return ctas == 2 ? 6 : 4; }
+#ifndef PCTC_TUNE_EPI_WARPS
+#define PCTC_TUNE_EPI_WARPS 0     // 0: by the contraction depth; 4 or 8: forced
+#endif
+// Epilogue warps per CTA (template parameter EW): 4 = one per tensor-memory lane quarter, 256
+// columns each; 8 = two per quarter, 128 columns each.  Eight hide the latency of a math-heavy
+// epilogue when the main loop of a tile is short (narrow heads); four leave the ring one stage
+// deeper and the SM cooler when the main loop is long.
+constexpr int warp_cols(int ew) { return BN / (ew / 4); }   // accumulator columns per epilogue warp
 constexpr int A_STAGE_BYTES = BM * BK * 2;
 constexpr int b_stage_bytes(int ctas) { return (BN / ctas) * BK * 2; }   // each CTA of a pair holds half of B
-constexpr int NUM_THREADS = 192;
+constexpr int num_threads(int ew) { return 64 + ew * 32; }
 constexpr int TMEM_COLS = 512;
 constexpr int MN_GROUP_BYTES = 64 * BK * 2;          // one 64-wide MN group of an MN-major tile
 constexpr long long WAIT_LIMIT_CYCLES = 4000000000LL;
@@ -72,24 +80,34 @@ struct SharedTail {   // barriers and flags
 };
 
 // Dynamic shared memory after the operand ring, by epilogue kind:
-//   store staging  4 warps x 2 buffers: 32 rows x 64 B boxes (bf16: dlogits, dW) or 32 rows x 128 B
-//                  boxes (fp32: dX), swizzled, written out by TMA stores while the other buffer fills
+//   store staging  8 warps x 2 buffers of 32 rows x 64 B (32 bf16 or 16 fp32 columns), 64-byte
+//                  swizzle, written out by TMA stores while the other buffer fills
 //   SharedTail
-//   bias           4 warps x BN floats (lse, subset, dlogits)
-//   list           4 warps x (BN indices in U, -1 if the column's class is not selected, + 8 group masks) (dlogits)
-constexpr int stage_box_bytes(int epi) { return epi == EPI_ACCUM_F32 ? 4096 : 2048; }   // one staged box
-constexpr int stage_warp_bytes(int epi) { return 2 * stage_box_bytes(epi); }              // double-buffered
+//   bias           8 warps x 128 floats (lse, subset, dlogits)
+//   list           8 warps x (128 indices in U, -1 if the column's class is not selected, + group masks) (dlogits)
+constexpr int STAGE_BOX_BYTES = 2048;                      // one staged box: 32 rows x 64 B
+constexpr int STAGE_WARP_BYTES = 2 * STAGE_BOX_BYTES;      // double-buffered
 constexpr bool epi_uses_tma_store(int epi) { return epi == EPI_DLOGITS || epi == EPI_ACCUM_F32 || epi == EPI_STORE_OUT; }
 constexpr bool epi_uses_bias(int epi) { return epi == EPI_LSE_PARTIAL || epi == EPI_SUBSET_LOGP || epi == EPI_DLOGITS; }
-constexpr size_t ring_bytes(int ctas) { return (size_t)stages_of(ctas) * (A_STAGE_BYTES + b_stage_bytes(ctas)); }
-static_assert(ring_bytes(1) == ring_bytes(2), "both tile modes use the same operand ring size");
-constexpr size_t RING_BYTES = ring_bytes(1);
-constexpr size_t off_stage() { return RING_BYTES; }
-constexpr size_t off_tail(int epi) { return RING_BYTES + (epi_uses_tma_store(epi) ? 4 * stage_warp_bytes(epi) : 0); }
-constexpr size_t off_bias(int epi) { return off_tail(epi) + 256; }
-constexpr size_t off_list(int epi) { return off_bias(epi) + (epi_uses_bias(epi) ? 4 * BN * 4 : 0); }
-constexpr int LIST_WORDS = BN + 32;
-constexpr size_t smem_bytes(int epi) { return 1024 + off_list(epi) + (epi == EPI_DLOGITS ? 4 * LIST_WORDS * 4 : 0); }
+// ring depth: what is left of the 227 KB after the epilogue's own buffers
+constexpr int stages_of(int ctas, int epi, int ew) {
+  return ctas == 2 ? ((epi_uses_tma_store(epi) && ew == 8) ? 5 : 6) : (epi_uses_tma_store(epi) ? 3 : 4);
+}
+constexpr size_t ring_bytes(int ctas, int epi, int ew) {
+  return (size_t)stages_of(ctas, epi, ew) * (A_STAGE_BYTES + b_stage_bytes(ctas));
+}
+constexpr size_t off_stage(int ctas, int epi, int ew) { return ring_bytes(ctas, epi, ew); }
+constexpr size_t off_tail(int ctas, int epi, int ew) {
+  return ring_bytes(ctas, epi, ew) + (epi_uses_tma_store(epi) ? ew * STAGE_WARP_BYTES : 0);
+}
+constexpr size_t off_bias(int ctas, int epi, int ew) { return off_tail(ctas, epi, ew) + 256; }
+constexpr size_t off_list(int ctas, int epi, int ew) {
+  return off_bias(ctas, epi, ew) + (epi_uses_bias(epi) ? ew * warp_cols(ew) * 4 : 0);
+}
+constexpr int list_words(int ew) { return warp_cols(ew) + 32; }
+constexpr size_t smem_bytes(int ctas, int epi, int ew) {
+  return 1024 + off_list(ctas, epi, ew) + (epi == EPI_DLOGITS ? ew * list_words(ew) * 4 : 0);
+}
 static_assert(sizeof(SharedTail) <= 256, "tail layout");
 
 // ---------------------------------------------------------------------------------------------
@@ -235,25 +253,6 @@ __device__ __forceinline__ void tmem_ld32(unsigned taddr, float* v) {
 #pragma unroll
   for (int i = 0; i < 32; ++i) v[i] = __uint_as_float(r[i]);
 }
-// The same load without the wait: the registers are valid only after tmem_wait_ld() and must be
-// read through tmem_regs_to_float() (volatile moves that stay behind the wait).
-__device__ __forceinline__ void tmem_ld32_issue(unsigned taddr, unsigned* r) {
-  asm volatile(
-      "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
-      "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
-      "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];"
-      : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]),
-        "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]),
-        "=r"(r[16]), "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]),
-        "=r"(r[24]), "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
-      : "r"(taddr)
-      : "memory");
-}
-__device__ __forceinline__ void tmem_wait_ld() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
-__device__ __forceinline__ void tmem_regs_to_float(const unsigned* r, float* v) {
-#pragma unroll
-  for (int i = 0; i < 32; ++i) asm volatile("mov.b32 %0, %1;" : "=f"(v[i]) : "r"(r[i]));
-}
 __device__ __forceinline__ float ex2(float x) {
   float y;
   asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
@@ -293,18 +292,20 @@ __device__ __forceinline__ void decode_unit(int u, int m_tiles, int n_tiles, int
 // ---------------------------------------------------------------------------------------------
 // The kernel
 // ---------------------------------------------------------------------------------------------
-template <int EPI, int CTAS>
-__global__ void __launch_bounds__(NUM_THREADS, 1)
+template <int EPI, int CTAS, int EW>
+__global__ void __launch_bounds__(num_threads(EW), 1)
 k_umma_gemm(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
             const __grid_constant__ CUtensorMap tmC, UmmaArgs a) {
-  constexpr int STAGES = stages_of(CTAS);
+  constexpr int STAGES = stages_of(CTAS, EPI, EW);
   constexpr int B_STAGE_BYTES = b_stage_bytes(CTAS);
+  constexpr int WARP_COLS = warp_cols(EW);
+  constexpr int LIST_WORDS = list_words(EW);
   constexpr int TILE_M = BM * CTAS;            // rows of the tile a CTA (pair) works on
   extern __shared__ unsigned char smem_raw[];
   unsigned char* smem = (unsigned char*)(((size_t)smem_raw + 1023) & ~(size_t)1023);
   unsigned char* sA = smem;
   unsigned char* sB = smem + (size_t)STAGES * A_STAGE_BYTES;
-  SharedTail* st = (SharedTail*)(smem + off_tail(EPI));
+  SharedTail* st = (SharedTail*)(smem + off_tail(CTAS, EPI, EW));
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int rank = (CTAS == 2) ? (int)cluster_ctarank() : 0;     // position inside the pair
@@ -321,7 +322,7 @@ k_umma_gemm(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
 
   if (threadIdx.x == 0) {
     for (int s = 0; s < STAGES; ++s) { mbar_init(&st->full[s], 1); mbar_init(&st->empty[s], 1); }
-    for (int s = 0; s < 2; ++s) { mbar_init(&st->tmem_full[s], 1); mbar_init(&st->tmem_empty[s], 4 * CTAS); }
+    for (int s = 0; s < 2; ++s) { mbar_init(&st->tmem_full[s], 1); mbar_init(&st->tmem_empty[s], EW * CTAS); }
     mbar_init(&st->done, 1);
     st->abort = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -440,15 +441,15 @@ k_umma_gemm(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
     }
   } else {
     // ===================== epilogue warps =====================
-    const int ew = warp - 2;                 // private staging slot
+    const int ew = warp - 2;                 // private staging slot, 0..EW-1
     const int q = warp & 3;                  // tensor-memory lane quarter this warp may read
     const int r = q * 32 + lane;             // accumulator row of this thread
-    float* sb = (float*)(smem + off_bias(EPI)) + ew * BN;
-    int* sj = (int*)(smem + off_list(EPI)) + ew * LIST_WORDS;            // index in U of each tile column, or -1
-    unsigned* sg = (unsigned*)sj + BN;                                    // one mask of selected columns per 32
-    unsigned char* stage = smem + off_stage() + ew * stage_warp_bytes(EPI);   // this warp's two staging boxes
-    const unsigned swz = (unsigned)(lane & 7);          // 128-byte swizzle of a staged 128-byte row (fp32 boxes)
-    const unsigned swz64 = (unsigned)((lane >> 1) & 3); // 64-byte swizzle of a staged 64-byte row (bf16 boxes)
+    const int c_base = (ew >> 2) * WARP_COLS;   // this warp's columns of the tile: [c_base, c_base + WARP_COLS)
+    float* sb = (float*)(smem + off_bias(CTAS, EPI, EW)) + ew * WARP_COLS;     // bias of the warp's columns
+    int* sj = (int*)(smem + off_list(CTAS, EPI, EW)) + ew * LIST_WORDS;         // index in U of each of them, or -1
+    unsigned* sg = (unsigned*)sj + WARP_COLS;                              // one mask of selected columns per 32
+    unsigned char* stage = smem + off_stage(CTAS, EPI, EW) + ew * STAGE_WARP_BYTES;   // this warp's two staging boxes
+    const unsigned swz64 = (unsigned)((lane >> 1) & 3); // 64-byte swizzle of a staged 64-byte row
     unsigned nbox = 0;                                  // boxes stored so far by this warp (buffer parity)
     unsigned it = 0;
     bool ok = true;
@@ -471,8 +472,8 @@ k_umma_gemm(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
         if ((EPI == EPI_LSE_PARTIAL || EPI == EPI_DLOGITS || EPI == EPI_SUBSET_LOGP) && has_bias) {
           const __nv_bfloat16* bias = (const __nv_bfloat16*)a.e.bias;
 #pragma unroll
-          for (int c = lane; c < BN; c += 32) {
-            const int j = n0 + c;
+          for (int c = lane; c < WARP_COLS; c += 32) {
+            const int j = n0 + c_base + c;
             float b = 0.f;
             if (bias && j < n_eff) {
               if (EPI == EPI_SUBSET_LOGP) b = __bfloat162float(bias[a.e.U[j]]);
@@ -483,8 +484,8 @@ k_umma_gemm(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
         }
         if (EPI == EPI_DLOGITS) {
 #pragma unroll
-          for (int c0 = 0; c0 < BN; c0 += 32) {
-            const int j = n0 + c0 + lane;
+          for (int c0 = 0; c0 < WARP_COLS; c0 += 32) {
+            const int j = n0 + c_base + c0 + lane;
             const int jj = (j < n_eff) ? a.e.vmap[a.e.v0 + j] : -1;
             const unsigned mask = __ballot_sync(0xffffffffu, jj >= 0);
             sj[c0 + lane] = jj;
@@ -498,58 +499,56 @@ k_umma_gemm(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
         got = __shfl_sync(0xffffffffu, got, 0);
         if (!got) { ok = false; break; }
         tc_fence_after();
-        const unsigned taddr = tmem_base + ((unsigned)(q * 32) << 16) + acc * BN;
+        const unsigned taddr = tmem_base + ((unsigned)(q * 32) << 16) + acc * BN + c_base;   // lane quarter, buffer, column half
 
         if (epi_uses_tma_store(EPI)) {
-          // ---- staged epilogues: the warp's 32 rows go out as 128-byte-wide boxes through TMA ----
-          // One box per 32 accumulator columns: 32 rows x 128 B (fp32) or 32 rows x 64 B (bf16).  Two
+          // ---- staged epilogues: the warp's 32 rows go out as 64-byte-wide boxes through TMA ----
+          // 32 bf16 columns (one box) or 2 x 16 fp32 columns (two boxes) per 32-column group.  Two
           // buffers alternate, so a box is filled while the TMA engine still reads the previous one.
-          unsigned ra[32], rb[32];                    // the 32-column groups, loaded one group ahead
-          tmem_ld32_issue(taddr, ra);
 #pragma unroll 1
-          for (int cg = 0; cg < BN / 32; cg += 2) {
+          for (int cg = 0; cg < WARP_COLS / 32; ++cg) {
+            const int g0 = cg * 32;                   // first of the warp's columns in this group
+            const int j0 = n0 + c_base + g0;
+            if (j0 >= n_eff) break;                   // warp-uniform
+            float v[32];
+            tmem_ld32(taddr + g0, v);
+            if (EPI == EPI_DLOGITS) {
+              if (has_bias) {
 #pragma unroll
-            for (int half = 0; half < 2; ++half) {
-              const int g0 = (cg + half) * 32;        // first tile column of this group
-              const int j0 = n0 + g0;
-              if (j0 >= n_eff) break;                 // warp-uniform
-              tmem_wait_ld();
-              float v[32];
-              tmem_regs_to_float(half ? rb : ra, v);
-              if (g0 + 32 < BN && j0 + 32 < n_eff)    // next group: the load flies while this one is processed
-                tmem_ld32_issue(taddr + g0 + 32, half ? ra : rb);
-              if (lane == 0) bulk_wait_read1();        // the box stored two groups ago has left its buffer
+                for (int c = 0; c < 32; ++c) v[c] += sb[g0 + c];
+              }
+#pragma unroll
+              for (int c = 0; c < 32; ++c) v[c] = ex2(fmaf(v[c], LOG2E, -lam2));     // p = exp(z - lambda)
+              if (sg[cg] != 0u) {
+                // the group holds selected classes: subtract their occupancy in fp32, before the
+                // rounding to bf16; the loads are issued together, the unselected ones predicated off
+                float g[32];
+#pragma unroll
+                for (int c = 0; c < 32; ++c) {
+                  const int jj = sj[g0 + c];
+                  g[c] = (jj >= 0 && row_ok) ? a.e.gamma[(long long)i * a.e.ld_gamma + jj] : 0.f;
+                }
+#pragma unroll
+                for (int c = 0; c < 32; ++c) v[c] = w * (v[c] - g[c]);
+              } else {
+#pragma unroll
+                for (int c = 0; c < 32; ++c) v[c] *= w;
+              }
+            }
+            constexpr int NBOX = (EPI == EPI_ACCUM_F32) ? 2 : 1;     // boxes per group
+#pragma unroll
+            for (int b = 0; b < NBOX; ++b) {
+              if (NBOX == 2 && j0 + b * 16 >= n_eff) break;          // warp-uniform
+              if (lane == 0) bulk_wait_read1();        // the box stored two boxes ago has left its buffer
               __syncwarp();
-              unsigned char* row = stage + (nbox & 1u) * stage_box_bytes(EPI) + lane * (EPI == EPI_ACCUM_F32 ? 128 : 64);
+              unsigned char* box = stage + (nbox & 1u) * STAGE_BOX_BYTES;
+              unsigned char* row = box + lane * 64;
               if (EPI == EPI_ACCUM_F32) {
 #pragma unroll
-                for (int c4 = 0; c4 < 8; ++c4)
-                  *reinterpret_cast<float4*>(row + (((unsigned)c4 ^ swz) << 4)) =
-                      make_float4(v[c4 * 4], v[c4 * 4 + 1], v[c4 * 4 + 2], v[c4 * 4 + 3]);
+                for (int c4 = 0; c4 < 4; ++c4)
+                  *reinterpret_cast<float4*>(row + (((unsigned)c4 ^ swz64) << 4)) =
+                      make_float4(v[b * 16 + c4 * 4], v[b * 16 + c4 * 4 + 1], v[b * 16 + c4 * 4 + 2], v[b * 16 + c4 * 4 + 3]);
               } else {
-                if (EPI == EPI_DLOGITS) {
-                  if (has_bias) {
-#pragma unroll
-                    for (int c = 0; c < 32; ++c) v[c] += sb[g0 + c];
-                  }
-#pragma unroll
-                  for (int c = 0; c < 32; ++c) v[c] = ex2(fmaf(v[c], LOG2E, -lam2));     // p = exp(z - lambda)
-                  if (sg[g0 >> 5] != 0u) {
-                    // the group holds selected classes: subtract their occupancy in fp32, before the
-                    // rounding to bf16; the loads are issued together, the unselected ones predicated off
-                    float g[32];
-#pragma unroll
-                    for (int c = 0; c < 32; ++c) {
-                      const int jj = sj[g0 + c];
-                      g[c] = (jj >= 0 && row_ok) ? a.e.gamma[(long long)i * a.e.ld_gamma + jj] : 0.f;
-                    }
-#pragma unroll
-                    for (int c = 0; c < 32; ++c) v[c] = w * (v[c] - g[c]);
-                  } else {
-#pragma unroll
-                    for (int c = 0; c < 32; ++c) v[c] *= w;
-                  }
-                }
 #pragma unroll
                 for (int c8 = 0; c8 < 4; ++c8) {
                   uint4 o;
@@ -564,24 +563,22 @@ k_umma_gemm(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
               fence_async_smem();                      // staged data visible to the TMA engine
               __syncwarp();
               if (lane == 0) {
-                const void* box = stage + (nbox & 1u) * stage_box_bytes(EPI);
                 if ((EPI == EPI_ACCUM_F32 || EPI == EPI_STORE_OUT) && a.e.accumulate)
-                  tma_reduce_add_2d(&tmC, box, j0, row0_cta + q * 32);
-                else tma_store_2d(&tmC, box, j0, row0_cta + q * 32);
+                  tma_reduce_add_2d(&tmC, box, j0 + b * 16, row0_cta + q * 32);
+                else tma_store_2d(&tmC, box, j0 + b * 16, row0_cta + q * 32);
                 bulk_commit();
               }
               ++nbox;
             }
           }
-          tmem_wait_ld();     // nothing of this tile is in flight when the accumulator is released
         }
 
 #pragma unroll 1
-        for (int cg = 0; cg < BN / 32 && !epi_uses_tma_store(EPI); ++cg) {
-          if (n0 + cg * 32 >= n_eff) break;          // warp-uniform
+        for (int cg = 0; cg < WARP_COLS / 32 && !epi_uses_tma_store(EPI); ++cg) {
+          const int j0 = n0 + c_base + cg * 32;
+          if (j0 >= n_eff) break;                    // warp-uniform
           float v[32];
           tmem_ld32(taddr + cg * 32, v);
-          const int j0 = n0 + cg * 32;
           if (EPI == EPI_STORE_F32) {
             if (row_ok) {
               float* dst = (float*)a.e.out + (long long)i * a.e.ld + j0;
@@ -621,7 +618,7 @@ k_umma_gemm(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
       }
 
       if (EPI == EPI_LSE_PARTIAL && ok && row_ok)
-        a.e.partial[(long long)i * a.nsplit + sp] = make_float2(run_max2 * LN2, run_sum);
+        a.e.partial[((long long)i * a.nsplit + sp) * (EW / 4) + (ew >> 2)] = make_float2(run_max2 * LN2, run_sum);
     }
     if (epi_uses_tma_store(EPI) && lane == 0) bulk_wait0();   // this warp's stores have completed
   }
@@ -686,54 +683,60 @@ int sm_count() {
 
 constexpr int CTAS_DEFAULT = PCTC_TUNE_CTAS;
 
-template <int EPI>
-cudaError_t launch(const CUtensorMap& tmA, const CUtensorMap& tmB, const CUtensorMap& tmC, const UmmaArgs& a,
-                   int grid, cudaStream_t stream) {
+template <int EPI, int EW>
+cudaError_t launch_ew(const CUtensorMap& tmA, const CUtensorMap& tmB, const CUtensorMap& tmC, const UmmaArgs& a,
+                      int grid, cudaStream_t stream) {
   static bool configured = false;
-  constexpr size_t SMEM = smem_bytes(EPI);
+  static int max_groups = 0;        // CTA groups (clusters) that can be resident at once
+  constexpr size_t SMEM = smem_bytes(CTAS_DEFAULT, EPI, EW);
   static_assert(SMEM <= 227 * 1024, "shared memory budget");
-  auto kern = k_umma_gemm<EPI, CTAS_DEFAULT>;
+  auto kern = k_umma_gemm<EPI, CTAS_DEFAULT, EW>;
   if (!configured) {
     cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)SMEM);
     if (e != cudaSuccess) return e;
     configured = true;
   }
-  cudaLaunchConfig_t cfg = {};
-  static int max_groups = 0;        // CTA groups (clusters) that can be resident at once
-  if (max_groups == 0) {
-    cudaLaunchConfig_t q = {};
-    q.gridDim = dim3((unsigned)(sm_count() / CTAS_DEFAULT * CTAS_DEFAULT));
-    q.blockDim = dim3(NUM_THREADS);
-    q.dynamicSmemBytes = SMEM;
-    cudaLaunchAttribute qa[1];
-    qa[0].id = cudaLaunchAttributeClusterDimension;
-    qa[0].val.clusterDim.x = CTAS_DEFAULT;
-    qa[0].val.clusterDim.y = 1;
-    qa[0].val.clusterDim.z = 1;
-    q.attrs = qa;
-    q.numAttrs = 1;
-    int n = 0;
-    if (cudaOccupancyMaxActiveClusters(&n, kern, &q) != cudaSuccess || n <= 0) n = sm_count() / CTAS_DEFAULT;
-    max_groups = n;
-  }
-  if (grid > max_groups * CTAS_DEFAULT) grid = max_groups * CTAS_DEFAULT;
-  cfg.gridDim = dim3((unsigned)grid);
-  cfg.blockDim = dim3(NUM_THREADS);
-  cfg.dynamicSmemBytes = SMEM;
-  cfg.stream = stream;
   cudaLaunchAttribute attr[1];
   attr[0].id = cudaLaunchAttributeClusterDimension;
   attr[0].val.clusterDim.x = CTAS_DEFAULT;
   attr[0].val.clusterDim.y = 1;
   attr[0].val.clusterDim.z = 1;
+  cudaLaunchConfig_t cfg = {};
+  cfg.blockDim = dim3(num_threads(EW));
+  cfg.dynamicSmemBytes = SMEM;
+  cfg.stream = stream;
   cfg.attrs = attr;
   cfg.numAttrs = 1;
+  if (max_groups == 0) {
+    cfg.gridDim = dim3((unsigned)(sm_count() / CTAS_DEFAULT * CTAS_DEFAULT));
+    int n = 0;
+    if (cudaOccupancyMaxActiveClusters(&n, kern, &cfg) != cudaSuccess || n <= 0) n = sm_count() / CTAS_DEFAULT;
+    max_groups = n;
+  }
+  if (grid > max_groups * CTAS_DEFAULT) grid = max_groups * CTAS_DEFAULT;
+  cfg.gridDim = dim3((unsigned)grid);
   return cudaLaunchKernelEx(&cfg, kern, tmA, tmB, tmC, a);
+}
+
+// Eight epilogue warps when a tile's main loop is short next to its epilogue (k <= 2048), else four.
+constexpr int EW_SWITCH_K = 2048;
+inline int epi_warps_for(int k) {
+  if (PCTC_TUNE_EPI_WARPS == 4 || PCTC_TUNE_EPI_WARPS == 8) return PCTC_TUNE_EPI_WARPS;
+  return k <= EW_SWITCH_K ? 8 : 4;
+}
+
+template <int EPI>
+cudaError_t launch(const CUtensorMap& tmA, const CUtensorMap& tmB, const CUtensorMap& tmC, const UmmaArgs& a,
+                   int grid, cudaStream_t stream) {
+  return epi_warps_for(a.k) == 8 ? launch_ew<EPI, 8>(tmA, tmB, tmC, a, grid, stream)
+                                 : launch_ew<EPI, 4>(tmA, tmB, tmC, a, grid, stream);
 }
 
 }  // namespace
 
 bool umma_available() { return encode_fn() != nullptr; }
+
+int umma_lse_partials_per_split(int k) { return epi_warps_for(k) / 4; }
 
 int umma_lse_splits(int m, int n) {
   // column splits per row tile such that the (row tile, split) units fill whole waves of CTAs
@@ -741,7 +744,7 @@ int umma_lse_splits(int m, int n) {
   const int m_tiles = (m + BM * CTAS_DEFAULT - 1) / (BM * CTAS_DEFAULT), n_tiles = (n + BN - 1) / BN;
   int best = 1;
   double best_cost = 1e30;
-  for (int s = 1; s <= 64 && s <= n_tiles; ++s) {
+  for (int s = 1; s <= 32 && s <= n_tiles; ++s) {     // each split yields two partials per frame (column halves)
     const long long units = (long long)m_tiles * s;
     const long long waves = (units + sms - 1) / sms;
     const int per = (n_tiles + s - 1) / s;                 // column tiles of the largest split
@@ -762,7 +765,7 @@ cudaError_t umma_gemm(const __nv_bfloat16* A, long long lda, bool a_mn_major,
   // output boxes of the staged epilogues: 32 rows x 32 columns, clipped to the [m, n] extent
   if (e.kind == EPI_ACCUM_F32) {
     if ((e.ld % 4) || ((size_t)e.out & 15)) return cudaErrorInvalidValue;
-    ok = ok && make_map(&tmC, e.out, (unsigned long long)n, (unsigned long long)m, (unsigned long long)e.ld, 32, 32, true);
+    ok = ok && make_map(&tmC, e.out, (unsigned long long)n, (unsigned long long)m, (unsigned long long)e.ld, 16, 32, true);
   } else if (e.kind == EPI_DLOGITS || e.kind == EPI_STORE_OUT) {
     if ((e.ld % 8) || ((size_t)e.out & 15)) return cudaErrorInvalidValue;
     ok = ok && make_map(&tmC, e.out, (unsigned long long)n, (unsigned long long)m, (unsigned long long)e.ld, 32, 32);

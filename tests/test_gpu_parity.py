@@ -25,6 +25,11 @@ def test_c1_fp32_full_config(lib):
     ref = H.run_oracle(batch)
     errs = H.assert_parity(gpu, ref, batch)
     assert max(errs.values()) < 1e-4
+    # and against the stored oracle values (tests/golden/c1_oracle.json)
+    import json, os
+    gold = json.load(open(os.path.join(os.path.dirname(os.path.abspath(__file__)), "golden", "c1_oracle.json")))
+    np.testing.assert_allclose(gpu["loss"], gold["loss"], rtol=1e-5)
+    assert list(gpu["subset"][: gold["K"]]) == gold["U"]
 
 
 def test_fp32_with_bias_ragged_chunks_blank_nonzero(lib):

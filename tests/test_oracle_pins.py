@@ -377,3 +377,36 @@ def test_beam_monotone_and_off_encodings():
         assert O.ctc_occupancy(logp, y, 0, beam=off)[0] == exact
     # the best alignment always survives: the loss stays finite at any positive beam
     assert np.isfinite(O.ctc_occupancy(logp, y, 0, beam=1e-9)[0])
+
+
+def test_feasibility_rule_fixture():
+    # tests/golden/feasibility_cases.txt: the paper's rule T >= |y| + (adjacent equal pairs), Appendix B.1
+    import os
+    path = os.path.join(os.path.dirname(os.path.abspath(__file__)), "golden", "feasibility_cases.txt")
+    rows = [ln.split("|") for ln in open(path) if ln.strip() and not ln.startswith("#")]
+    assert len(rows) >= 10
+    rng = np.random.default_rng(0)
+    for T, toks, ok in rows:
+        T, ok = int(T), int(ok)
+        y = [] if toks.strip() == "-" else [int(t) for t in toks.split()]
+        assert O.is_feasible(y, T) == bool(ok)
+        logp, _ = random_logp(rng, T, 9)
+        loss, gamma, flags, _ = O.ctc_occupancy(logp, y, 0)
+        assert (flags == 0) == bool(ok)
+        if not ok:
+            assert loss == 0.0 and gamma is None
+
+
+def test_stored_c1_values_match_the_oracle():
+    # the stored file is written by tests/golden/make_c1_golden.py (oracle only); it guards the
+    # oracle and the generator against silent changes
+    import json, os
+    from paper_2609_33645_b200 import workloads as wl
+    gold = json.load(open(os.path.join(os.path.dirname(os.path.abspath(__file__)), "golden", "c1_oracle.json")))
+    batch = wl.make_batch(wl.CONFIGS["c1"])
+    ref = O.pruned_ctc_reference(batch.hidden, batch.W, None, batch.targets, batch.input_lengths,
+                                 batch.target_lengths, batch.blank)
+    np.testing.assert_allclose(ref["loss"], gold["loss"], rtol=1e-12)
+    assert ref["K"] == gold["K"] and list(ref["U"]) == gold["U"]
+    assert np.linalg.norm(ref["dW"]) == pytest.approx(gold["dW_fro"], rel=1e-12)
+    np.testing.assert_allclose(ref["dW"][0, :8], gold["dW_row_blank"], rtol=1e-10)

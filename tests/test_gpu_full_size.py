@@ -71,3 +71,59 @@ def test_c4_full_size_sampled_parity(lib):
     for k, v in enumerate(rows):
         e = H.rel_fro(got_rows[k], ref["dW"][k])
         assert e <= 3e-2, (int(v), e)
+
+
+def test_c5_full_size_losses_and_beam_gap(lib):
+    """c5 (D=5120, V=151,936, T up to 3000, up to 600 labels): per-utterance loss without a beam and at
+    beams 16 and 8 against the oracle at the same beam; the gap Delta_n = L_beta,n - L_n >= 0 and the
+    discarded mass delta_n = 1 - exp(-Delta_n) of Appendix B.3 are printed for the record."""
+    import torch
+    from oracle import pruned_ctc_oracle as O
+    cfg = wl.CONFIGS["c5"]
+    batch = wl.make_batch(cfg)
+    dev = torch.device("cuda:0")
+    hidden = torch.from_numpy(batch.hidden).to(dev).to(torch.bfloat16)
+    W = torch.from_numpy(batch.W).to(dev).to(torch.bfloat16)
+    targets = torch.from_numpy(batch.targets).to(dev)
+    gpu = {}
+    res = None
+    for beam in (0.0, 16.0, 8.0):
+        res = lib.pruned_ctc_fwd_bwd(hidden, W, None, targets, batch.input_lengths, batch.target_lengths,
+                                     batch.blank, beam=beam, check_status=True,
+                                     workspace=None if res is None else res["workspace"])
+        torch.cuda.synchronize()
+        gpu[beam] = res["loss"].cpu().numpy().astype(np.float64)
+        assert int(res["flags"].abs().sum().item()) == 0
+    del res
+    torch.cuda.empty_cache()
+
+    # oracle: full-vocabulary normaliser per utterance, then the alignment sums on the selected classes
+    # (by Proposition 1 the selected log-probabilities with relabelled targets give the same loss)
+    t0 = time.time()
+    W64 = batch.W.astype(np.float64)
+    ref = {0.0: [], 16.0: [], 8.0: []}
+    for n in range(cfg.N):
+        Tn, Un = int(batch.input_lengths[n]), int(batch.target_lengths[n])
+        y = [int(v) for v in batch.targets[n, :Un]]
+        Z = O.head_logits(batch.hidden[n, :Tn], W64)
+        lam = O.log_normalizer(Z)
+        cols = np.array([batch.blank] + sorted(set(y)), dtype=np.int64)
+        logp = Z[:, cols] - lam[:, None]
+        del Z
+        ytil = [int(np.searchsorted(cols[1:], v)) + 1 for v in y]
+        for beam in ref:
+            ref[beam].append(O.ctc_occupancy(logp, ytil, 0, beam=beam if beam > 0 else None)[0])
+    print(f"oracle took {time.time() - t0:.1f} s")
+    for beam in ref:
+        r = np.array(ref[beam])
+        rel = np.abs(gpu[beam] - r) / np.abs(r)
+        print(f"beam {beam}: oracle {r}, gpu {gpu[beam]}, rel err {rel}")
+        assert np.all(rel <= 2e-3)
+    exact = np.array(ref[0.0])
+    for beam in (16.0, 8.0):
+        Delta, delta = O.discarded_mass(ref[beam], exact)
+        Delta_gpu = gpu[beam] - gpu[0.0]
+        print(f"beam {beam}: Delta_n oracle {Delta}, gpu {Delta_gpu}, delta_n {delta}")
+        assert np.all(Delta >= -1e-9)
+        assert np.all(Delta_gpu >= -2e-3 * exact)          # within the loss tolerance of being an upper bound
+        assert np.all(np.abs(Delta_gpu - Delta) <= 2e-3 * exact)

@@ -69,6 +69,8 @@ typedef struct {
                             computed nor touched (dW may be NULL); dH and dbias still are        */
   int32_t accumulate_dW; /* 1: dW and dbias are added to (gradient accumulation over
                             micro-batches) instead of overwritten                              */
+  int32_t forward_only;  /* 1: losses only (validation): lines 11-17 are skipped, dH, dW and dbias
+                            are neither computed nor touched and may be NULL                    */
   int32_t max_K;         /* 0, or a promise K <= max_K (K = |U| is only known on the device; a
                             data loader that holds the targets on the host knows it).  Sizes the
                             [M, K] buffers by max_K instead of the bound 1 + sum U_n.  If the
@@ -206,6 +208,29 @@ pctc_status_t pruned_ctc_fwd_bwd_host(const pctc_problem_t* problem,
                                       int32_t* subset_out, int32_t* K_out, int32_t* relabeled_out,
                                       int32_t* utt_flags,
                                       void* device_scratch, size_t scratch_bytes, void* stream);
+
+/*
+ * Greedy CTC recognition with the same head (the paper's recognition path for
+ * LLM-CTC, Section 5.1 / Appendix D: the head is applied in vocabulary chunks, the
+ * frame-wise arg-max is taken and the CTC collapse map B of Section 3.1 -- merge
+ * repeats, then drop blanks -- gives the hypothesis).  The logits are never
+ * stored: the projection kernel keeps a running (max, arg-max) per frame.
+ *
+ * Uses N, T, D, V, dtype, blank_id, gemm_path of `problem`.  hidden [N,T,D], W [V,D],
+ * bias [V] or NULL (device); input_lengths HOST [N].  Outputs (device):
+ *   frame_labels [N,T] or NULL: arg-max class of every valid frame, -1 on padded frames
+ *                 (the smallest index wins among equal logits);
+ *   tokens [N,T]: the collapsed hypothesis of each utterance, padded with -1;
+ *   token_lengths [N].
+ * workspace: at least pctc_greedy_workspace_bytes(), 256-byte aligned.
+ */
+pctc_status_t pctc_greedy_workspace_bytes(const pctc_problem_t* problem, const int32_t* input_lengths_host,
+                                          size_t* bytes_out);
+pctc_status_t pctc_greedy_decode(const pctc_problem_t* problem,
+                                 const void* hidden, const void* W, const void* bias,
+                                 const int32_t* input_lengths,
+                                 int32_t* frame_labels, int32_t* tokens, int32_t* token_lengths,
+                                 void* workspace, size_t workspace_bytes, void* stream);
 
 /*
  * Contraction kernel on its own, for validation of the tensor-core path:

@@ -405,6 +405,39 @@ def grouped_reference(hidden, W, bias, targets, input_lengths, target_lengths, b
     return dict(loss=loss, dH=dH, dW=dW, db=db, U=U, K=K, relabeled=rel)
 
 
+# ----------------------------------------------------------------------------
+# Greedy recognition (Section 5.1; Appendix D): frame-wise arg-max, then the
+# collapse map B of Section 3.1
+# ----------------------------------------------------------------------------
+
+def collapse(labels, blank):
+    """B: merge consecutive repetitions, then remove blanks."""
+    out = []
+    prev = None
+    for v in labels:
+        v = int(v)
+        if v != prev and v != blank:
+            out.append(v)
+        prev = v
+    return out
+
+
+def greedy_decode(hidden, W, bias, input_lengths, blank):
+    """Per utterance: arg-max class of every valid frame (first index on ties), the collapsed
+    hypothesis, and the full logits' top value per frame (for near-tie checks)."""
+    hidden = np.asarray(hidden, dtype=np.float64)
+    W64 = np.asarray(W, dtype=np.float64)
+    b64 = None if bias is None else np.asarray(bias, dtype=np.float64)
+    frames, hyps, logits = [], [], []
+    for n in range(hidden.shape[0]):
+        Z = head_logits(hidden[n, : int(input_lengths[n])], W64, b64)
+        lab = np.argmax(Z, axis=1)
+        frames.append(lab)
+        hyps.append(collapse(lab, blank))
+        logits.append(Z)
+    return frames, hyps, logits
+
+
 def discarded_mass(loss_beam, loss_exact):
     """Delta_n = L_beta,n - L_n and delta_n = 1 - exp(-Delta_n)  (Appendix B.3)."""
     delta_big = np.asarray(loss_beam, dtype=np.float64) - np.asarray(loss_exact, dtype=np.float64)

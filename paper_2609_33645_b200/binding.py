@@ -22,7 +22,8 @@ UTT_INFEASIBLE, UTT_NONFINITE, UTT_BAD_TARGET, UTT_SUBSET_OVERFLOW = 1, 2, 4, 8
 
 EXPORTS = ("pctc_workspace_bytes", "pruned_ctc_fwd_bwd", "pruned_ctc_fwd_bwd_traced", "pctc_gemm_bf16",
            "pctc_workspace_status", "pctc_status_string", "pctc_host_call_scratch_bytes",
-           "pruned_ctc_fwd_bwd_host", "pctc_subset_relabel_noalloc")
+           "pruned_ctc_fwd_bwd_host", "pctc_subset_relabel_noalloc", "pctc_greedy_workspace_bytes",
+           "pctc_greedy_decode")
 NOALLOC_MAX_V = 262144
 
 PHASES = ("prep", "lse", "subset_logp", "dp", "dlogits", "dh", "dw", "dbias", "finish")
@@ -35,7 +36,8 @@ class Problem(ctypes.Structure):
         ("dtype", ctypes.c_int32), ("blank_id", ctypes.c_int32),
         ("beam", ctypes.c_float),
         ("chunk", ctypes.c_int32), ("target_stride", ctypes.c_int32), ("gemm_path", ctypes.c_int32),
-        ("skip_dW", ctypes.c_int32), ("accumulate_dW", ctypes.c_int32), ("max_K", ctypes.c_int32),
+        ("skip_dW", ctypes.c_int32), ("accumulate_dW", ctypes.c_int32), ("forward_only", ctypes.c_int32),
+        ("max_K", ctypes.c_int32),
         ("utt_weights", ctypes.c_void_p),
     ]
 
@@ -105,6 +107,10 @@ def load() -> ctypes.CDLL:
     lib.pctc_subset_relabel_noalloc.restype = ctypes.c_int
     lib.pctc_subset_relabel_noalloc.argtypes = [vp, vp, ctypes.c_int32, ctypes.c_int32, ctypes.c_int64,
                                                 ctypes.c_int32, vp, vp, vp, vp, vp]
+    lib.pctc_greedy_workspace_bytes.restype = ctypes.c_int
+    lib.pctc_greedy_workspace_bytes.argtypes = [ctypes.POINTER(Problem), i32p, ctypes.POINTER(ctypes.c_size_t)]
+    lib.pctc_greedy_decode.restype = ctypes.c_int
+    lib.pctc_greedy_decode.argtypes = [ctypes.POINTER(Problem), vp, vp, vp, i32p, vp, vp, vp, vp, ctypes.c_size_t, vp]
     lib.pctc_gemm_bf16.restype = ctypes.c_int
     lib.pctc_gemm_bf16.argtypes = [vp, vp, vp, ctypes.c_int32, ctypes.c_int32, ctypes.c_int32,
                                    ctypes.c_int32, ctypes.c_int32, ctypes.c_int32, vp, vp]
@@ -129,10 +135,10 @@ def _ptr_i32(a: np.ndarray):
 
 
 def make_problem(N, T, D, V, dtype, blank_id, beam=0.0, chunk=0, target_stride=0, gemm_path=GEMM_AUTO,
-                 skip_dW=False, accumulate_dW=False, utt_weights_ptr=None, max_K=0) -> Problem:
+                 skip_dW=False, accumulate_dW=False, utt_weights_ptr=None, max_K=0, forward_only=False) -> Problem:
     return Problem(int(N), int(T), int(D), int(V), int(dtype), int(blank_id), float(beam), int(chunk),
                    int(target_stride), int(gemm_path), int(bool(skip_dW)), int(bool(accumulate_dW)),
-                   int(max_K), utt_weights_ptr)
+                   int(bool(forward_only)), int(max_K), utt_weights_ptr)
 
 
 def workspace_bytes(problem: Problem, input_lengths, target_lengths) -> int:
@@ -151,7 +157,7 @@ def _dptr(t) -> Optional[int]:
 def pruned_ctc_fwd_bwd(hidden, W, bias, targets, input_lengths, target_lengths, blank_id, *, beam=0.0,
                        chunk=0, gemm_path=GEMM_AUTO, workspace=None, out=None, check_status=False,
                        trace: Optional[Trace] = None, skip_dW=False, accumulate_dW=False, utt_weights=None,
-                       max_K=0):
+                       max_K=0, forward_only=False):
     """Algorithm 1 on CUDA tensors.
 
     hidden [N,T,D], W [V,D], bias [V] or None (bf16 or fp32, same dtype), targets
@@ -182,7 +188,7 @@ def pruned_ctc_fwd_bwd(hidden, W, bias, targets, input_lengths, target_lengths, 
     if utt_weights is not None and (utt_weights.dtype != torch.float32 or tuple(utt_weights.shape) != (N,)):
         raise ValueError("utt_weights must be an fp32 CUDA tensor of shape [N]")
     prob = make_problem(N, T, D, V, dt, blank_id, beam, chunk, stride, gemm_path, skip_dW, accumulate_dW,
-                        None if utt_weights is None else utt_weights.data_ptr(), max_K)
+                        None if utt_weights is None else utt_weights.data_ptr(), max_K, forward_only)
     need = workspace_bytes(prob, il, tl)
     dev = hidden.device
     if workspace is None or workspace.numel() < need:
@@ -200,9 +206,9 @@ def pruned_ctc_fwd_bwd(hidden, W, bias, targets, input_lengths, target_lengths, 
         ksum = min(ksum, int(max_K))
     res = dict(
         loss=buf("loss", (N,), torch.float32),
-        dH=buf("dH", (N, T, D), hidden.dtype),
-        dW=None if skip_dW else buf("dW", (V, D), hidden.dtype),
-        dbias=buf("dbias", (V,), hidden.dtype) if bias is not None else None,
+        dH=None if forward_only else buf("dH", (N, T, D), hidden.dtype),
+        dW=None if (skip_dW or forward_only) else buf("dW", (V, D), hidden.dtype),
+        dbias=buf("dbias", (V,), hidden.dtype) if (bias is not None and not forward_only) else None,
         subset=buf("subset", (ksum,), torch.int32),
         K=buf("K", (1,), torch.int32),
         relabeled=buf("relabeled", (N, stride), torch.int32),
@@ -328,3 +334,36 @@ def subset_relabel_noalloc(targets, target_lengths, V, blank_id, out):
     if st != 0:
         raise PctcError(st, "pctc_subset_relabel_noalloc")
     return out
+
+
+def greedy_decode(hidden, W, bias, input_lengths, blank_id, *, gemm_path=GEMM_AUTO, workspace=None):
+    """Greedy CTC recognition: frame arg-max of the head, repeats merged, blanks dropped.
+
+    Returns device tensors frame_labels [N,T] (-1 on padded frames), tokens [N,T] (padded with
+    -1), token_lengths [N], and the reusable workspace.
+    """
+    import torch
+
+    lib = load()
+    dt = PCTC_BF16 if hidden.dtype == torch.bfloat16 else PCTC_FP32
+    N, T, D = hidden.shape
+    V = W.shape[0]
+    il = _i32(input_lengths)
+    prob = make_problem(N, T, D, V, dt, blank_id, gemm_path=gemm_path)
+    need = ctypes.c_size_t(0)
+    st = lib.pctc_greedy_workspace_bytes(ctypes.byref(prob), _ptr_i32(il), ctypes.byref(need))
+    if st != 0:
+        raise PctcError(st, "pctc_greedy_workspace_bytes")
+    dev = hidden.device
+    if workspace is None or workspace.numel() < need.value:
+        workspace = torch.empty(need.value, dtype=torch.uint8, device=dev)
+    frame_labels = torch.empty((N, T), dtype=torch.int32, device=dev)
+    tokens = torch.empty((N, T), dtype=torch.int32, device=dev)
+    token_lengths = torch.empty((N,), dtype=torch.int32, device=dev)
+    stream = ctypes.c_void_p(torch.cuda.current_stream(dev).cuda_stream)
+    st = lib.pctc_greedy_decode(ctypes.byref(prob), _dptr(hidden), _dptr(W), _dptr(bias), _ptr_i32(il),
+                                _dptr(frame_labels), _dptr(tokens), _dptr(token_lengths), _dptr(workspace),
+                                ctypes.c_size_t(workspace.numel()), stream)
+    if st != 0:
+        raise PctcError(st, "pctc_greedy_decode")
+    return dict(frame_labels=frame_labels, tokens=tokens, token_lengths=token_lengths, workspace=workspace)

@@ -38,7 +38,7 @@ pctc_status_t make_plan(const pctc_problem_t* p, const int32_t* Tn, const int32_
   if (p->dtype != PCTC_BF16 && p->dtype != PCTC_FP32) return PCTC_ERR_UNSUPPORTED;
   if (p->gemm_path != PCTC_GEMM_AUTO && p->gemm_path != PCTC_GEMM_SIMT) return PCTC_ERR_INVALID_ARG;
   if (p->chunk < 0) return PCTC_ERR_INVALID_ARG;
-  if ((p->skip_dW | p->accumulate_dW) & ~1) return PCTC_ERR_INVALID_ARG;
+  if ((p->skip_dW | p->accumulate_dW | p->forward_only) & ~1) return PCTC_ERR_INVALID_ARG;
   if (p->max_K < 0) return PCTC_ERR_INVALID_ARG;
   if (std::isnan(p->beam)) return PCTC_ERR_INVALID_ARG;
   long long M = 0, Usum = 0, cells = 0, mcells = 0;
@@ -230,12 +230,13 @@ pctc_status_t pruned_ctc_fwd_bwd_traced(const pctc_problem_t* p, const void* hid
     if (!trace->events || !trace->kinds || trace->capacity < 12 + 4 * pl.nchunks) return PCTC_ERR_INVALID_ARG;
     trace->used = 0;
   }
-  if (!hidden || !W || !loss || !dH || (!dW && !p->skip_dW) || !workspace) return PCTC_ERR_INVALID_ARG;
+  if (!hidden || !W || !loss || !workspace) return PCTC_ERR_INVALID_ARG;
+  if (!p->forward_only && (!dH || (!dW && !p->skip_dW))) return PCTC_ERR_INVALID_ARG;
   if (!targets && pl.Usum > 0) return PCTC_ERR_INVALID_ARG;
   if (workspace_bytes < pl.total) return PCTC_ERR_WORKSPACE_TOO_SMALL;
   if (((size_t)workspace & (ALIGN - 1)) || ((size_t)hidden & 15) || ((size_t)W & 15) || ((size_t)dH & 15) ||
       ((size_t)dW & 15))
-    return PCTC_ERR_INVALID_ARG;
+    return PCTC_ERR_INVALID_ARG;   // (null dH / dW are aligned)
   if (pl.use_umma && !umma_available()) return PCTC_ERR_CUDA;
   cudaStream_t stream = (cudaStream_t)stream_v;
   Aux aux;
@@ -384,7 +385,7 @@ pctc_status_t pruned_ctc_fwd_bwd_traced(const pctc_problem_t* p, const void* hid
   PCTC_CUDA(finalize_loss(d_lambda, bm, N, loss, d_flags, dp.roww, stream));
 
   // ---- lines 11-17: backward, one vocabulary chunk at a time ----
-  for (int ci = 0; ci < pl.nchunks; ++ci) {
+  for (int ci = 0; ci < pl.nchunks && !p->forward_only; ++ci) {
     const long long v0 = (long long)ci * pl.chunk;
     const int Cc = (int)((V - v0 < pl.chunk) ? (V - v0) : pl.chunk);
     const char* Wc = (const char*)W + (size_t)v0 * D * pl.elem;
@@ -432,7 +433,7 @@ pctc_status_t pruned_ctc_fwd_bwd_traced(const pctc_problem_t* p, const void* hid
     }
   }
   PCTC_MARK(PCTC_PHASE_FINISH);
-  PCTC_CUDA(unstack_cast(d_dHacc, dH, N, pl.T, D, pl.bf16, bm.T_n, bm.row0, stream));
+  if (!p->forward_only) PCTC_CUDA(unstack_cast(d_dHacc, dH, N, pl.T, D, pl.bf16, bm.T_n, bm.row0, stream));
 
   // ---- optional integer outputs ----
   if (subset_out)
@@ -449,6 +450,41 @@ pctc_status_t pruned_ctc_fwd_bwd_traced(const pctc_problem_t* p, const void* hid
 }
 
 namespace {
+struct GreedyPlan {
+  int N, T, D, M, elem, nsplit;
+  long long V;
+  bool bf16, use_umma;
+  size_t o_status, o_meta, o_X, o_partial, o_labels, total, meta_ints;
+};
+pctc_status_t greedy_plan(const pctc_problem_t* p, const int32_t* Tn, GreedyPlan* g) {
+  if (!p || !Tn) return PCTC_ERR_INVALID_ARG;
+  if (p->N <= 0 || p->T <= 0 || p->D <= 0 || p->V <= 0) return PCTC_ERR_INVALID_ARG;
+  if (p->V > 0x7fffffffLL) return PCTC_ERR_UNSUPPORTED;
+  if (p->blank_id < 0 || (long long)p->blank_id >= p->V) return PCTC_ERR_INVALID_ARG;
+  if (p->dtype != PCTC_BF16 && p->dtype != PCTC_FP32) return PCTC_ERR_UNSUPPORTED;
+  if (p->gemm_path != PCTC_GEMM_AUTO && p->gemm_path != PCTC_GEMM_SIMT) return PCTC_ERR_INVALID_ARG;
+  long long M = 0;
+  for (int n = 0; n < p->N; ++n) {
+    if (Tn[n] < 1 || Tn[n] > p->T) return PCTC_ERR_INVALID_ARG;
+    M += Tn[n];
+  }
+  if (M > 0x3fffffffLL) return PCTC_ERR_UNSUPPORTED;
+  g->N = p->N; g->T = p->T; g->D = p->D; g->V = p->V; g->M = (int)M;
+  g->bf16 = p->dtype == PCTC_BF16;
+  g->elem = g->bf16 ? 2 : 4;
+  g->use_umma = g->bf16 && p->gemm_path == PCTC_GEMM_AUTO && (p->D % 8 == 0);
+  g->meta_ints = (size_t)g->N + (g->N + 1) + g->M;      // T_n | row0 | row_utt
+  size_t o = 0;
+  auto take = [&](size_t bytes) { size_t r = o; o = up(o + bytes); return r; };
+  g->o_status = take(256);
+  g->o_meta = take(g->meta_ints * 4);
+  g->o_X = take((size_t)g->M * g->D * g->elem);
+  g->o_partial = take((size_t)g->M * 64 * 8);
+  g->o_labels = take((size_t)g->M * 4);
+  g->total = o;
+  return PCTC_OK;
+}
+
 struct HostLayout {
   size_t o_hidden, o_W, o_bias, o_targets, o_loss, o_dH, o_dW, o_dbias, o_subset, o_K, o_rel, o_flags, o_ws;
   size_t b_hidden, b_W, b_bias, b_targets, b_rel, b_subset, ws_bytes, total;
@@ -506,7 +542,7 @@ pctc_status_t pruned_ctc_fwd_bwd_host(const pctc_problem_t* p, const void* hidde
   pctc_status_t st = host_layout(p, input_lengths, target_lengths, bias != nullptr, &h);
   if (st != PCTC_OK) return st;
   if (!hidden || !W || !loss || !dH || !dW || !device_scratch) return PCTC_ERR_INVALID_ARG;
-  if (p->skip_dW || p->accumulate_dW || p->utt_weights) return PCTC_ERR_UNSUPPORTED;   // device entry point only
+  if (p->skip_dW || p->accumulate_dW || p->utt_weights || p->forward_only) return PCTC_ERR_UNSUPPORTED;   // device entry point only
   if (!targets && h.b_targets > 0) return PCTC_ERR_INVALID_ARG;
   if ((size_t)device_scratch & (ALIGN - 1)) return PCTC_ERR_INVALID_ARG;
   if (scratch_bytes < h.total) return PCTC_ERR_WORKSPACE_TOO_SMALL;
@@ -536,6 +572,71 @@ pctc_status_t pruned_ctc_fwd_bwd_host(const pctc_problem_t* p, const void* hidde
   if (relabeled_out && h.b_rel)
     PCTC_CUDA(cudaMemcpyAsync(relabeled_out, d + h.o_rel, h.b_rel, cudaMemcpyDeviceToHost, stream));
   if (utt_flags) PCTC_CUDA(cudaMemcpyAsync(utt_flags, d + h.o_flags, (size_t)p->N * 4, cudaMemcpyDeviceToHost, stream));
+#undef PCTC_CUDA
+  return PCTC_OK;
+}
+
+pctc_status_t pctc_greedy_workspace_bytes(const pctc_problem_t* problem, const int32_t* input_lengths_host,
+                                          size_t* bytes_out) {
+  if (!bytes_out) return PCTC_ERR_INVALID_ARG;
+  GreedyPlan g;
+  pctc_status_t st = greedy_plan(problem, input_lengths_host, &g);
+  if (st != PCTC_OK) return st;
+  *bytes_out = g.total;
+  return PCTC_OK;
+}
+
+pctc_status_t pctc_greedy_decode(const pctc_problem_t* p, const void* hidden, const void* W, const void* bias,
+                                 const int32_t* input_lengths, int32_t* frame_labels, int32_t* tokens,
+                                 int32_t* token_lengths, void* workspace, size_t workspace_bytes, void* stream_v) {
+  GreedyPlan g;
+  pctc_status_t st = greedy_plan(p, input_lengths, &g);
+  if (st != PCTC_OK) return st;
+  if (!hidden || !W || !tokens || !token_lengths || !workspace) return PCTC_ERR_INVALID_ARG;
+  if (workspace_bytes < g.total) return PCTC_ERR_WORKSPACE_TOO_SMALL;
+  if (((size_t)workspace & (ALIGN - 1)) || ((size_t)hidden & 15) || ((size_t)W & 15)) return PCTC_ERR_INVALID_ARG;
+  if (g.use_umma && !umma_available()) return PCTC_ERR_CUDA;
+  cudaStream_t stream = (cudaStream_t)stream_v;
+  char* ws = (char*)workspace;
+  const int N = g.N, M = g.M, D = g.D;
+#define PCTC_CUDA(call)                              \
+  do {                                               \
+    if ((call) != cudaSuccess) return PCTC_ERR_CUDA; \
+  } while (0)
+  std::vector<int> meta(g.meta_ints);
+  {
+    int* Tn = meta.data();
+    int* row0 = Tn + N;
+    int* row_utt = row0 + N + 1;
+    int r = 0;
+    for (int n = 0; n < N; ++n) {
+      Tn[n] = input_lengths[n];
+      row0[n] = r;
+      for (int t = 0; t < Tn[n]; ++t) row_utt[r + t] = n;
+      r += Tn[n];
+    }
+    row0[N] = r;
+  }
+  int* d_meta = (int*)(ws + g.o_meta);
+  PCTC_CUDA(cudaMemcpyAsync(d_meta, meta.data(), g.meta_ints * 4, cudaMemcpyHostToDevice, stream));
+  PCTC_CUDA(cudaMemsetAsync(ws + g.o_status, 0, 256, stream));
+  const int* d_Tn = d_meta;
+  const int* d_row0 = d_meta + N;
+  const int* d_row_utt = d_meta + 2 * N + 1;
+  void* d_X = ws + g.o_X;
+  float2* d_partial = (float2*)(ws + g.o_partial);
+  int* d_labels = (int*)(ws + g.o_labels);
+  PCTC_CUDA(stack_frames(hidden, d_X, N, g.T, D, g.elem, d_row_utt, d_row0, M, stream));
+  Epilogue e;
+  e.kind = EPI_ARGMAX_PARTIAL;
+  e.bias = bias;
+  e.partial = d_partial;
+  e.nsplit = g.use_umma ? umma_lse_splits(M, (int)g.V) : 32;
+  GemmCall c{d_X, D, false, W, D, false, M, (int)g.V, D};
+  PCTC_CUDA(run_gemm(g.use_umma, g.bf16, c, e, (int*)(ws + g.o_status), stream));
+  PCTC_CUDA(argmax_combine(d_partial, g.use_umma ? umma_lse_partials_per_split(D) * e.nsplit : e.nsplit, M, d_labels,
+                           stream));
+  PCTC_CUDA(greedy_collapse(d_labels, d_row0, d_Tn, N, g.T, p->blank_id, frame_labels, tokens, token_lengths, stream));
 #undef PCTC_CUDA
   return PCTC_OK;
 }

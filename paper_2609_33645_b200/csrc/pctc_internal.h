@@ -19,7 +19,8 @@ enum EpiKind : int {
   EPI_SUBSET_LOGP = 2,  // S[i*ld + j] = acc + bias[U[j]] - lambda[i],  j < K  (Algorithm 1 line 6); lambda null: no shift
   EPI_DLOGITS = 3,      // chunk[i*ld + j] = w_i (exp(acc + bias[v0+j] - lambda[i]) - gamma[i, vmap[v0+j]])
   EPI_ACCUM_F32 = 4,    // acc_out[i*ld + j] (+)= acc                          (dH across chunks)
-  EPI_STORE_OUT = 5     // out[i*ld + j] = T(acc)                              (rows of dW)
+  EPI_STORE_OUT = 5,    // out[i*ld + j] = T(acc)                              (rows of dW)
+  EPI_ARGMAX_PARTIAL = 6  // running (max, argmax) of z = acc + bias[j] over a column range (recognition)
 };
 
 struct Epilogue {
@@ -61,6 +62,14 @@ bool umma_available();   // the driver entry point for tensor maps could be reso
 int umma_lse_splits(int m, int n);   // column splits (<= 32) for EPI_LSE_PARTIAL on this device
 int umma_lse_partials_per_split(int k);   // the kernel writes this many partials per split (1 or 2):
                                           // partial[(i*nsplit + sp)*pps + h]
+
+// Combine argmax partials (value, column index as int bits): labels[i] = argmax, smallest index on ties.
+cudaError_t argmax_combine(const float2* partial, int nparts, int M, int* labels, cudaStream_t stream);
+
+// Greedy CTC hypothesis per utterance: merge repeated frame labels, drop blanks.  frame_labels (may be
+// null) and tokens are [N, T] padded with -1; token_lengths [N].
+cudaError_t greedy_collapse(const int* labels, const int* row0, const int* T_n, int N, int T, int blank,
+                            int* frame_labels, int* tokens, int* token_lengths, cudaStream_t stream);
 
 // Combine LSE partials: lambda[i] = log sum over splits.
 cudaError_t lse_combine(const float2* partial, int nsplit, int M, float* lambda, cudaStream_t stream);

@@ -169,7 +169,57 @@ __global__ void k_lse_combine(const float2* __restrict__ partial, int nsplit, in
   lambda[i] = mx + logf(sum);
 }
 
+// --- recognition: frame arg-max from per-split partials, then the collapse map B of Section 3.1 ---
+__global__ void k_argmax_combine(const float2* __restrict__ partial, int nparts, int M, int* __restrict__ labels) {
+  int i = blockIdx.x * blockDim.x + threadIdx.x;
+  if (i >= M) return;
+  float best = -CUDART_INF_F;
+  int idx = 0x7fffffff;
+  for (int s = 0; s < nparts; ++s) {
+    const float2 p = partial[(size_t)i * nparts + s];
+    const int j = __float_as_int(p.y);
+    if (j < 0) continue;                                   // empty split
+    if (p.x > best || (p.x == best && j < idx)) { best = p.x; idx = j; }
+  }
+  labels[i] = (idx == 0x7fffffff) ? 0 : idx;
+}
+
+// One warp per utterance, 32 frames at a time: a frame emits its label iff the label is not blank
+// and differs from the previous frame's label.
+__global__ void k_greedy_collapse(const int* __restrict__ labels, const int* __restrict__ row0,
+                                  const int* __restrict__ T_n, int T, int blank, int* frame_labels,
+                                  int* tokens, int* token_lengths) {
+  const int n = blockIdx.x, lane = threadIdx.x;
+  const int Tn = T_n[n], r0 = row0[n];
+  int count = 0, prev_last = -1;
+  for (int t0 = 0; t0 < T; t0 += 32) {
+    const int t = t0 + lane;
+    const int lab = (t < Tn) ? labels[r0 + t] : -1;
+    if (frame_labels && t < T) frame_labels[(size_t)n * T + t] = lab;
+    int prev = __shfl_up_sync(0xffffffffu, lab, 1);
+    if (lane == 0) prev = prev_last;
+    const bool emit = (t < Tn) && lab != blank && lab != prev;
+    const unsigned mask = __ballot_sync(0xffffffffu, emit);
+    if (emit) tokens[(size_t)n * T + count + __popc(mask & ((1u << lane) - 1u))] = lab;
+    count += __popc(mask);
+    prev_last = __shfl_sync(0xffffffffu, lab, 31);
+  }
+  for (int t = count + lane; t < T; t += 32) tokens[(size_t)n * T + t] = -1;
+  if (lane == 0) token_lengths[n] = count;
+}
+
 }  // namespace
+
+cudaError_t argmax_combine(const float2* partial, int nparts, int M, int* labels, cudaStream_t stream) {
+  k_argmax_combine<<<(M + 127) / 128, 128, 0, stream>>>(partial, nparts, M, labels);
+  return cudaGetLastError();
+}
+
+cudaError_t greedy_collapse(const int* labels, const int* row0, const int* T_n, int N, int T, int blank,
+                            int* frame_labels, int* tokens, int* token_lengths, cudaStream_t stream) {
+  k_greedy_collapse<<<N, 32, 0, stream>>>(labels, row0, T_n, T, blank, frame_labels, tokens, token_lengths);
+  return cudaGetLastError();
+}
 
 cudaError_t subset_and_relabel(const int* targets, int target_stride, const int* U_n_dev, int N,
                                long long V, int blank, unsigned* bitmap, int* word_rank,

@@ -40,8 +40,9 @@ __global__ void __launch_bounds__(NT) k_simt_gemm(const T* __restrict__ A, const
   const int Kdev = (EPI == EPI_SUBSET_LOGP) ? *e.Kdev : 0;
 
   float run_max[4], run_sum[4];
+  int run_idx[4];
 #pragma unroll
-  for (int r = 0; r < 4; ++r) { run_max[r] = -CUDART_INF_F; run_sum[r] = 0.f; }
+  for (int r = 0; r < 4; ++r) { run_max[r] = -CUDART_INF_F; run_sum[r] = 0.f; run_idx[r] = -1; }
 
   for (int jt = jt_begin; jt < jt_end; ++jt) {
     const int j0 = jt * TN;
@@ -105,6 +106,9 @@ __global__ void __launch_bounds__(NT) k_simt_gemm(const T* __restrict__ A, const
           } else {
             run_sum[r] += __expf(z - run_max[r]);
           }
+        } else if (EPI == EPI_ARGMAX_PARTIAL) {
+          const float z = a + bias_at<T>(e.bias, e.v0 + j);
+          if (z > run_max[r]) { run_max[r] = z; run_idx[r] = j; }     // ascending j: first maximum wins
         } else if (EPI == EPI_SUBSET_LOGP) {
           if (j < Kdev)
             reinterpret_cast<float*>(e.out)[(long long)i * e.ld + j] = a + bias_at<T>(e.bias, e.U[j]) - lam;
@@ -125,6 +129,25 @@ __global__ void __launch_bounds__(NT) k_simt_gemm(const T* __restrict__ A, const
     }
   }
 
+  if (EPI == EPI_ARGMAX_PARTIAL) {
+    __shared__ int s_idx[TM][17];
+#pragma unroll
+    for (int r = 0; r < 4; ++r) { s_red[0][ty * 4 + r][tx] = run_max[r]; s_idx[ty * 4 + r][tx] = run_idx[r]; }
+    __syncthreads();
+    if (tid < TM) {
+      const int i = i0 + tid;
+      if (i < g.m) {
+        float best = -CUDART_INF_F;
+        int idx = -1;
+        for (int q = 0; q < 16; ++q) {
+          const float v = s_red[0][tid][q];
+          const int j = s_idx[tid][q];
+          if (j >= 0 && (v > best || (v == best && j < idx) || idx < 0)) { best = v; idx = j; }
+        }
+        e.partial[(long long)i * e.nsplit + blockIdx.x] = make_float2(best, __int_as_float(idx));
+      }
+    }
+  }
   if (EPI == EPI_LSE_PARTIAL) {
     // merge the 16 threads that share a row, in a fixed order
 #pragma unroll
@@ -151,7 +174,7 @@ template <typename T, int EPI>
 cudaError_t launch(const void* A, const void* B, const GemmShape& g, const Epilogue& e, cudaStream_t stream) {
   const int ntiles = (g.n + TN - 1) / TN;
   int tiles_per_cta = 1, gx = ntiles;
-  if (EPI == EPI_LSE_PARTIAL) {
+  if (EPI == EPI_LSE_PARTIAL || EPI == EPI_ARGMAX_PARTIAL) {
     tiles_per_cta = (ntiles + e.nsplit - 1) / e.nsplit;
     gx = e.nsplit;
   }
@@ -170,6 +193,7 @@ cudaError_t dispatch(const void* A, const void* B, const GemmShape& g, const Epi
     case EPI_DLOGITS: return launch<T, EPI_DLOGITS>(A, B, g, e, s);
     case EPI_ACCUM_F32: return launch<T, EPI_ACCUM_F32>(A, B, g, e, s);
     case EPI_STORE_OUT: return launch<T, EPI_STORE_OUT>(A, B, g, e, s);
+    case EPI_ARGMAX_PARTIAL: return launch<T, EPI_ARGMAX_PARTIAL>(A, B, g, e, s);
   }
   return cudaErrorInvalidValue;
 }

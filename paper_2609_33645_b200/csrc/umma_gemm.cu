@@ -88,7 +88,10 @@ struct SharedTail {   // barriers and flags
 constexpr int STAGE_BOX_BYTES = 2048;                      // one staged box: 32 rows x 64 B
 constexpr int STAGE_WARP_BYTES = 2 * STAGE_BOX_BYTES;      // double-buffered
 constexpr bool epi_uses_tma_store(int epi) { return epi == EPI_DLOGITS || epi == EPI_ACCUM_F32 || epi == EPI_STORE_OUT; }
-constexpr bool epi_uses_bias(int epi) { return epi == EPI_LSE_PARTIAL || epi == EPI_SUBSET_LOGP || epi == EPI_DLOGITS; }
+constexpr bool epi_uses_bias(int epi) {
+  return epi == EPI_LSE_PARTIAL || epi == EPI_SUBSET_LOGP || epi == EPI_DLOGITS || epi == EPI_ARGMAX_PARTIAL;
+}
+constexpr bool epi_walks_splits(int epi) { return epi == EPI_LSE_PARTIAL || epi == EPI_ARGMAX_PARTIAL; }
 // ring depth: what is left of the 227 KB after the epilogue's own buffers
 constexpr int stages_of(int ctas, int epi, int ew) {
   return ctas == 2 ? ((epi_uses_tma_store(epi) && ew == 8) ? 5 : 6) : (epi_uses_tma_store(epi) ? 3 : 4);
@@ -316,7 +319,7 @@ k_umma_gemm(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
   if (EPI == EPI_SUBSET_LOGP) n_eff = min(a.n, *a.e.Kdev);
   const int m_tiles = (a.m + TILE_M - 1) / TILE_M;
   const int n_tiles = (n_eff + BN - 1) / BN;
-  const int splits = (EPI == EPI_LSE_PARTIAL) ? a.nsplit : n_tiles;
+  const int splits = epi_walks_splits(EPI) ? a.nsplit : n_tiles;
   const int units = m_tiles * splits;
   const int k_blocks = (a.k + BK - 1) / BK;
 
@@ -463,13 +466,15 @@ k_umma_gemm(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
       if ((EPI == EPI_DLOGITS || (EPI == EPI_SUBSET_LOGP && a.e.lambda)) && row_ok) { lam = a.e.lambda[i]; lam2 = lam * LOG2E; }
       if (EPI == EPI_DLOGITS && row_ok) w = a.e.roww[i];
       float run_max2 = -CUDART_INF_F, run_sum = 0.f;     // EPI_LSE_PARTIAL, base-2 domain
+      float best_z = -CUDART_INF_F;                      // EPI_ARGMAX_PARTIAL
+      int best_j = -1;
 
       for (int nt = nt0; nt < nt0 + cnt && ok; ++nt, ++it) {
         const unsigned acc = it & 1u, aph = (it >> 1) & 1u;
         const int n0 = nt * BN;
         // ---- warp-private staging of per-column data (overlaps the MMAs of this tile) ----
         const bool has_bias = a.e.bias != nullptr;        // without a bias the staged zeros are never read
-        if ((EPI == EPI_LSE_PARTIAL || EPI == EPI_DLOGITS || EPI == EPI_SUBSET_LOGP) && has_bias) {
+        if (epi_uses_bias(EPI) && has_bias) {
           const __nv_bfloat16* bias = (const __nv_bfloat16*)a.e.bias;
 #pragma unroll
           for (int c = lane; c < WARP_COLS; c += 32) {
@@ -593,6 +598,12 @@ k_umma_gemm(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
               for (int c = 0; c < 32; ++c)
                 if (j0 + c < n_eff) dst[c] = v[c] + (has_bias ? sb[cg * 32 + c] : 0.f) - lam;
             }
+          } else if (EPI == EPI_ARGMAX_PARTIAL) {
+#pragma unroll
+            for (int c = 0; c < 32; ++c) {
+              const float z = has_bias ? v[c] + sb[cg * 32 + c] : v[c];
+              if (j0 + c < n_eff && z > best_z) { best_z = z; best_j = j0 + c; }   // ascending columns: first maximum wins
+            }
           } else if (EPI == EPI_LSE_PARTIAL) {
             float gmax = -CUDART_INF_F;
 #pragma unroll
@@ -619,6 +630,8 @@ k_umma_gemm(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
 
       if (EPI == EPI_LSE_PARTIAL && ok && row_ok)
         a.e.partial[((long long)i * a.nsplit + sp) * (EW / 4) + (ew >> 2)] = make_float2(run_max2 * LN2, run_sum);
+      if (EPI == EPI_ARGMAX_PARTIAL && ok && row_ok)
+        a.e.partial[((long long)i * a.nsplit + sp) * (EW / 4) + (ew >> 2)] = make_float2(best_z, __int_as_float(best_j));
     }
     if (epi_uses_tma_store(EPI) && lane == 0) bulk_wait0();   // this warp's stores have completed
   }
@@ -786,8 +799,9 @@ cudaError_t umma_gemm(const __nv_bfloat16* A, long long lda, bool a_mn_major,
   a.status = status;
   a.e = e;
   const int m_tiles = (m + BM * CTAS_DEFAULT - 1) / (BM * CTAS_DEFAULT), n_tiles = (n + BN - 1) / BN;
-  long long units = (long long)m_tiles * (e.kind == EPI_LSE_PARTIAL ? e.nsplit : n_tiles);
-  if (e.kind == EPI_LSE_PARTIAL && (e.nsplit < 1 || e.nsplit > n_tiles)) return cudaErrorInvalidValue;
+  const bool walks = e.kind == EPI_LSE_PARTIAL || e.kind == EPI_ARGMAX_PARTIAL;
+  long long units = (long long)m_tiles * (walks ? e.nsplit : n_tiles);
+  if (walks && (e.nsplit < 1 || e.nsplit > n_tiles)) return cudaErrorInvalidValue;
   const int groups = sm_count() / CTAS_DEFAULT;
   const int grid = (int)(units < groups ? units : groups) * CTAS_DEFAULT;
   switch (e.kind) {
@@ -797,6 +811,7 @@ cudaError_t umma_gemm(const __nv_bfloat16* A, long long lda, bool a_mn_major,
     case EPI_DLOGITS: return launch<EPI_DLOGITS>(tmA, tmB, tmC, a, grid, stream);
     case EPI_ACCUM_F32: return launch<EPI_ACCUM_F32>(tmA, tmB, tmC, a, grid, stream);
     case EPI_STORE_OUT: return launch<EPI_STORE_OUT>(tmA, tmB, tmC, a, grid, stream);
+    case EPI_ARGMAX_PARTIAL: return launch<EPI_ARGMAX_PARTIAL>(tmA, tmB, tmC, a, grid, stream);
   }
   return cudaErrorInvalidValue;
 }

@@ -214,3 +214,57 @@ def test_paper_grid_shape_many_short_utterances(lib):
     batch = wl.make_batch(cfg, permute_ids=True)
     gpu = H.run_gpu(lib, batch)
     H.assert_parity(gpu, H.run_oracle(batch), batch)
+
+
+def test_forward_only_matches_full_call(lib):
+    batch = wl.make_batch(small("c3", V=8192, D=256, N=4, T_div=4, U_div=2), permute_ids=True)
+    full = H.run_gpu(lib, batch)
+    fwd = H.run_gpu(lib, batch, forward_only=True)
+    assert fwd["dH"] is None and fwd["dW"] is None
+    np.testing.assert_array_equal(fwd["loss"], full["loss"])
+    np.testing.assert_array_equal(fwd["subset"], full["subset"])
+    fwd_beam = H.run_gpu(lib, batch, forward_only=True, beam=8.0)
+    np.testing.assert_array_equal(fwd_beam["loss"], H.run_gpu(lib, batch, beam=8.0)["loss"])
+
+
+@pytest.mark.parametrize("path,dtype", [(SIMT, "fp32"), (SIMT, "bf16"), (AUTO, "bf16")])
+def test_greedy_recognition_matches_oracle(lib, path, dtype):
+    import torch
+    from oracle import pruned_ctc_oracle as O
+    cfg = dataclasses.replace(wl.CONFIGS["c2"], name="greedy", N=5, T_lo=40, T_hi=90, D=64, V=5000 - 5000 % 8,
+                              dtype=dtype, blank=3, seed=99)
+    batch = wl.make_batch(cfg, with_bias=True)
+    batch.W[batch.blank] *= 3.0                      # make blanks and repeats frequent enough to matter
+    for t in range(0, batch.T - 1, 3):
+        batch.hidden[:, t + 1] = batch.hidden[:, t]  # repeated frames, so that merging repeats matters
+    if dtype == "bf16":
+        batch.W = wl.round_to_bf16(batch.W)
+    dev = torch.device("cuda:0")
+    tdt = torch.bfloat16 if dtype == "bf16" else torch.float32
+    out = lib.greedy_decode(torch.from_numpy(batch.hidden).to(dev).to(tdt), torch.from_numpy(batch.W).to(dev).to(tdt),
+                            torch.from_numpy(batch.bias).to(dev).to(tdt), batch.input_lengths, batch.blank,
+                            gemm_path=path)
+    torch.cuda.synchronize()
+    fl = out["frame_labels"].cpu().numpy()
+    tok = out["tokens"].cpu().numpy()
+    tlen = out["token_lengths"].cpu().numpy()
+    frames, hyps, logits = O.greedy_decode(batch.hidden, batch.W, batch.bias, batch.input_lengths, batch.blank)
+    tol = 1e-4 if dtype == "fp32" else 1e-3
+    exact = 0
+    for n in range(cfg.N):
+        Tn = int(batch.input_lengths[n])
+        assert np.all(fl[n, Tn:] == -1)
+        got = fl[n, :Tn]
+        # the arg-max is unique up to rounding: where it differs from the oracle's, the logit of the
+        # class the GPU chose must be within the arithmetic's rounding of the largest logit
+        z = logits[n]
+        assert np.all(z[np.arange(Tn), got] >= z.max(axis=1) - tol)
+        exact += int(np.sum(got == frames[n]))
+        # the hypothesis is the collapse of the frame labels the GPU itself chose (bit-exact), and
+        # equals the oracle's hypothesis whenever the frame labels agree
+        mine = O.collapse(got, batch.blank)
+        assert int(tlen[n]) == len(mine) and list(tok[n, : tlen[n]]) == mine and np.all(tok[n, tlen[n]:] == -1)
+        if np.array_equal(got, frames[n]):
+            assert mine == hyps[n]
+    assert exact >= 0.999 * int(batch.input_lengths.sum())
+    assert sum(len(h) for h in hyps) > 0

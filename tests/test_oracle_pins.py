@@ -410,3 +410,18 @@ def test_stored_c1_values_match_the_oracle():
     assert ref["K"] == gold["K"] and list(ref["U"]) == gold["U"]
     assert np.linalg.norm(ref["dW"]) == pytest.approx(gold["dW_fro"], rel=1e-12)
     np.testing.assert_allclose(ref["dW"][0, :8], gold["dW_row_blank"], rtol=1e-10)
+
+
+def test_collapse_map_and_greedy_decode():
+    # B merges repeats first, then drops blanks (Section 3.1): a blank between equal labels keeps both
+    assert O.collapse([0, 3, 3, 0, 3, 5, 5, 0, 0, 2], 0) == [3, 3, 5, 2]
+    assert O.collapse([4, 4, 4], 4) == [] and O.collapse([], 0) == []
+    assert collapse([0, 3, 3, 0, 3, 5, 5, 0, 0, 2], 0) == [3, 3, 5, 2]     # the test's own B agrees
+    rng = np.random.default_rng(8)
+    H = rng.standard_normal((2, 7, 4))
+    W = rng.standard_normal((6, 4))
+    frames, hyps, logits = O.greedy_decode(H, W, None, [7, 5], 2)
+    for n, Tn in enumerate((7, 5)):
+        Z = H[n, :Tn] @ W.T
+        assert list(frames[n]) == [int(np.argmax(z)) for z in Z]
+        assert hyps[n] == collapse(list(frames[n]), 2)

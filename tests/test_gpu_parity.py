@@ -268,3 +268,32 @@ def test_greedy_recognition_matches_oracle(lib, path, dtype):
             assert mine == hyps[n]
     assert exact >= 0.999 * int(batch.input_lengths.sum())
     assert sum(len(h) for h in hyps) > 0
+
+
+@pytest.mark.parametrize("path", [SIMT, AUTO])
+@pytest.mark.parametrize("case", range(12))
+def test_random_small_shapes(lib, path, case):
+    # seeded sweep over odd shapes: single frames, empty targets, heavy repeats, any blank id,
+    # vocabularies smaller than a tile, widths that are no multiple of a tile, bias on or off, beams
+    rng = np.random.default_rng(1000 + case)
+    N = int(rng.integers(1, 7))
+    D = int(rng.choice([8, 24, 64, 136, 200]))
+    V = int(rng.integers(2, 260)) * 8
+    T_hi = int(rng.integers(1, 70))
+    U_hi = int(rng.integers(0, max(1, min(T_hi, 40)) + 1))
+    dtype = "bf16" if (path == AUTO or case % 2) else "fp32"
+    cfg = dataclasses.replace(wl.CONFIGS["c1"], name=f"rnd{case}", N=N, T_lo=max(1, T_hi // 3), T_hi=T_hi, D=D, V=V,
+                              dtype=dtype, U_lo=0, U_hi=U_hi, zipf_s=1.0 if case % 3 else None,
+                              blank=int(rng.integers(0, V)), seed=5000 + case)
+    batch = wl.make_batch(cfg, with_bias=bool(case % 2), poison_padding=True, permute_ids=bool(case % 4 == 1))
+    for n in range(N):                                   # inject runs of equal labels
+        u = int(batch.target_lengths[n])
+        if u >= 3 and rng.random() < 0.6:
+            s0 = int(rng.integers(0, u - 2))
+            batch.targets[n, s0:s0 + 3] = batch.targets[n, s0]
+    beam = [0.0, 0.0, 4.0, 32.0][case % 4]
+    chunk = [0, 64, 128, 1024][case % 4]
+    gpu = H.run_gpu(lib, batch, gemm_path=path, beam=beam, chunk=chunk)
+    ref = H.run_oracle(batch, beam=beam if beam > 0 else None)
+    tol = (2e-3, 1e-2) if dtype == "bf16" else (2e-5, 5e-4)
+    H.assert_parity(gpu, ref, batch, tol=tol)

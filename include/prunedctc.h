@@ -188,9 +188,13 @@ pctc_status_t pruned_ctc_fwd_bwd_traced(const pctc_problem_t* problem,
  * pruned_ctc_fwd_bwd is a host pointer here; `device_scratch` is one device
  * buffer of at least pctc_host_call_scratch_bytes() bytes, 256-byte aligned,
  * that the call carves into input staging, output staging and the workspace.
- * Order on `stream`: host-to-device copies of hidden, W, bias, targets; Algorithm
- * 1; device-to-host copies of loss, dH, dW, dbias and the optional integer
- * outputs.  The call does not synchronise: the host outputs are valid once
+ * Order: host-to-device copies of hidden, bias, targets on `stream`; W follows on a
+ * copy stream of the library in four row segments, and the normaliser kernel of a
+ * segment starts as soon as that segment has landed (for V >= 16,384; the summation
+ * order of lambda then differs from the device entry point in the last bits);
+ * Algorithm 1; the rows of dW go back to the host chunk by chunk while later
+ * chunks are still being computed; loss, dH, dbias and the optional integer
+ * outputs at the end.  `stream` waits for all of it.  The call does not synchronise: the host outputs are valid once
  * `stream` has been synchronised, and the host inputs must stay unchanged until
  * then.  Same return codes as pruned_ctc_fwd_bwd.  skip_dW, accumulate_dW and utt_weights
  * belong to the device entry point only: here they return PCTC_ERR_UNSUPPORTED.

@@ -111,11 +111,25 @@ pctc_status_t make_plan(const pctc_problem_t* p, const int32_t* Tn, const int32_
   return PCTC_OK;
 }
 
-// One auxiliary stream and a fork/join event pair per device, created at the first call on that
+// Two auxiliary streams and a few events per device, created at the first call on that
 // device and kept until exit.  Calls on one device are therefore not re-entrant across host threads.
 struct Aux {
-  cudaStream_t side = nullptr;
+  cudaStream_t side = nullptr;          // alignment DP, beside the normaliser kernel
+  cudaStream_t copy_out = nullptr;      // host entry point: rows of dW leave while later chunks compute
+  cudaStream_t copy_in = nullptr;       // host entry point: W arrives in segments while the normaliser runs
   cudaEvent_t fork = nullptr, join = nullptr;
+  cudaEvent_t chunk_done[2] = {nullptr, nullptr}, copies_done = nullptr;
+  cudaEvent_t w_ready[4] = {nullptr, nullptr, nullptr, nullptr}, entry = nullptr;
+};
+
+// Set by the host-buffer entry point: where finished rows of dW go.
+struct HostPipe {
+  char* dW_host = nullptr;
+  // W arrives in `nseg` row segments of `seg_rows` rows (the last one shorter); w_ready[s] is
+  // recorded on the copy stream behind segment s.  nseg == 0: W is already on the device.
+  int nseg = 0;
+  long long seg_rows = 0;
+  cudaEvent_t w_ready[4] = {nullptr, nullptr, nullptr, nullptr};
 };
 cudaError_t get_aux(Aux* out) {
   static std::mutex mu;
@@ -128,8 +142,12 @@ cudaError_t get_aux(Aux* out) {
   Aux& a = table[dev];
   if (!a.side) {
     if ((e = cudaStreamCreateWithFlags(&a.side, cudaStreamNonBlocking)) != cudaSuccess) return e;
-    if ((e = cudaEventCreateWithFlags(&a.fork, cudaEventDisableTiming)) != cudaSuccess) return e;
-    if ((e = cudaEventCreateWithFlags(&a.join, cudaEventDisableTiming)) != cudaSuccess) return e;
+    if ((e = cudaStreamCreateWithFlags(&a.copy_out, cudaStreamNonBlocking)) != cudaSuccess) return e;
+    if ((e = cudaStreamCreateWithFlags(&a.copy_in, cudaStreamNonBlocking)) != cudaSuccess) return e;
+    cudaEvent_t* evs[] = {&a.fork,       &a.join,       &a.chunk_done[0], &a.chunk_done[1], &a.copies_done,
+                          &a.w_ready[0], &a.w_ready[1], &a.w_ready[2],    &a.w_ready[3],    &a.entry};
+    for (cudaEvent_t* ev : evs)
+      if ((e = cudaEventCreateWithFlags(ev, cudaEventDisableTiming)) != cudaSuccess) return e;
   }
   *out = a;
   return cudaSuccess;
@@ -217,12 +235,15 @@ pctc_status_t pruned_ctc_fwd_bwd(const pctc_problem_t* p, const void* hidden, co
                                    stream_v, nullptr);
 }
 
-pctc_status_t pruned_ctc_fwd_bwd_traced(const pctc_problem_t* p, const void* hidden, const void* W,
-                                        const void* bias, const int32_t* targets, const int32_t* input_lengths,
-                                        const int32_t* target_lengths, float* loss, void* dH, void* dW,
-                                        void* dbias, int32_t* subset_out, int32_t* K_out,
-                                        int32_t* relabeled_out, int32_t* utt_flags, void* workspace,
-                                        size_t workspace_bytes, void* stream_v, pctc_trace_t* trace) {
+}  // extern "C"
+
+namespace {
+// The whole call.  `pipe` is non-null only for the host-buffer entry point.
+pctc_status_t run_call(const pctc_problem_t* p, const void* hidden, const void* W, const void* bias,
+                       const int32_t* targets, const int32_t* input_lengths, const int32_t* target_lengths,
+                       float* loss, void* dH, void* dW, void* dbias, int32_t* subset_out, int32_t* K_out,
+                       int32_t* relabeled_out, int32_t* utt_flags, void* workspace, size_t workspace_bytes,
+                       void* stream_v, pctc_trace_t* trace, const HostPipe* pipe) {
   Plan pl;
   pctc_status_t st = make_plan(p, input_lengths, target_lengths, &pl);
   if (st != PCTC_OK) return st;
@@ -336,50 +357,86 @@ pctc_status_t pruned_ctc_fwd_bwd_traced(const pctc_problem_t* p, const void* hid
   // ---- line 4: stack the valid frames ----
   PCTC_CUDA(stack_frames(hidden, d_X, N, pl.T, D, pl.elem, bm.row_utt, bm.row0, M, stream));
 
-  // ---- line 6 first: logits of the selected classes, Z_U = X W_U^T + b_U ----
-  // The alignment sum of Eq. "ctc-factorization" needs no normaliser, so the DP runs on Z_U while
-  // the full-vocabulary normaliser is still being computed; lambda enters the loss at the end.
-  PCTC_MARK(PCTC_PHASE_SUBSET_LOGP);
-  {
-    PCTC_CUDA(gather_rows(W, d_WU, d_U, d_K, pl.Kcap, D, pl.elem, stream));
-    Epilogue e;
-    e.kind = EPI_SUBSET_LOGP;
-    e.out = d_S;
-    e.ld = (long long)pl.ldS;
-    e.lambda = nullptr;
-    e.bias = bias;
-    e.U = d_U;
-    e.Kdev = d_K;
-    GemmCall c{d_X, D, false, d_WU, D, false, M, pl.Kcap, D};
-    PCTC_CUDA(run_gemm(pl.use_umma, pl.bf16, c, e, d_status, stream));
-  }
-  // ---- lines 7-10 on the auxiliary stream: alignment DP, occupancies ----
-  PCTC_MARK(-2);
-  PCTC_CUDA(cudaEventRecord(aux.fork, stream));
-  PCTC_CUDA(cudaStreamWaitEvent(aux.side, aux.fork, 0));
-  {
-    cudaStream_t main_stream = stream;
-    stream = aux.side;
-    PCTC_MARK(PCTC_PHASE_DP);
-    PCTC_CUDA(alignment_dp(d_S, (long long)pl.ldS, d_rel, p->target_stride, bm, N, M, pl.Lmax,
-                           pl.beam ? p->beam : 0.f, dp, d_G, (long long)pl.ldS, d_K, loss, d_flags, stream));
+  // ---- line 6: logits of the selected classes, Z_U = X W_U^T + b_U; lines 7-10: the DP ----
+  // The alignment sum of Eq. "ctc-factorization" needs no normaliser, so the DP runs on Z_U (on the
+  // auxiliary stream) while the full-vocabulary normaliser is still being computed; lambda enters
+  // the loss at the end.
+  auto subset_logits_and_dp = [&]() -> pctc_status_t {
+    PCTC_MARK(PCTC_PHASE_SUBSET_LOGP);
+    {
+      PCTC_CUDA(gather_rows(W, d_WU, d_U, d_K, pl.Kcap, D, pl.elem, stream));
+      Epilogue e;
+      e.kind = EPI_SUBSET_LOGP;
+      e.out = d_S;
+      e.ld = (long long)pl.ldS;
+      e.lambda = nullptr;
+      e.bias = bias;
+      e.U = d_U;
+      e.Kdev = d_K;
+      GemmCall c{d_X, D, false, d_WU, D, false, M, pl.Kcap, D};
+      PCTC_CUDA(run_gemm(pl.use_umma, pl.bf16, c, e, d_status, stream));
+    }
     PCTC_MARK(-2);
-    stream = main_stream;
-  }
-  PCTC_CUDA(cudaEventRecord(aux.join, aux.side));
+    PCTC_CUDA(cudaEventRecord(aux.fork, stream));
+    PCTC_CUDA(cudaStreamWaitEvent(aux.side, aux.fork, 0));
+    {
+      cudaStream_t main_stream = stream;
+      stream = aux.side;
+      PCTC_MARK(PCTC_PHASE_DP);
+      PCTC_CUDA(alignment_dp(d_S, (long long)pl.ldS, d_rel, p->target_stride, bm, N, M, pl.Lmax,
+                             pl.beam ? p->beam : 0.f, dp, d_G, (long long)pl.ldS, d_K, loss, d_flags, stream));
+      PCTC_MARK(-2);
+      stream = main_stream;
+    }
+    PCTC_CUDA(cudaEventRecord(aux.join, aux.side));
+    return PCTC_OK;
+  };
 
-  // ---- line 5: normaliser, online over the vocabulary (concurrent with the DP) ----
-  PCTC_MARK(PCTC_PHASE_LSE);
-  {
-    Epilogue e;
-    e.kind = EPI_LSE_PARTIAL;
-    e.bias = bias;
-    e.partial = d_partial;
-    e.nsplit = pl.use_umma ? umma_lse_splits(M, (int)V) : 32;
-    GemmCall c{d_X, D, false, W, D, false, M, (int)V, D};
-    PCTC_CUDA(run_gemm(pl.use_umma, pl.bf16, c, e, d_status, stream));
-    PCTC_CUDA(lse_combine(d_partial, pl.use_umma ? umma_lse_partials_per_split(D) * e.nsplit : e.nsplit, M, d_lambda,
-                          stream));
+  // ---- line 5: normaliser, online over the vocabulary ----
+  // One launch over all of W; or, when W is still arriving from the host in row segments, one
+  // launch per segment as it lands, each writing its own split slots of the partial buffer.
+  auto normaliser = [&]() -> pctc_status_t {
+    PCTC_MARK(PCTC_PHASE_LSE);
+    const int pps = pl.use_umma ? umma_lse_partials_per_split(D) : 1;
+    const int nseg = (pipe && pipe->nseg > 0) ? pipe->nseg : 1;
+    const long long seg_rows = nseg > 1 ? pipe->seg_rows : V;
+    int per_seg = pl.use_umma ? umma_lse_splits(M, (int)(seg_rows < V ? seg_rows : V)) : 32;
+    if (per_seg * nseg * pps > 64) per_seg = 64 / (nseg * pps);
+    int slots = 0;
+    for (int sg = 0; sg < nseg; ++sg) {
+      const long long v0 = (long long)sg * seg_rows;
+      if (v0 >= V) break;
+      const long long rows = (V - v0 < seg_rows) ? (V - v0) : seg_rows;
+      if (nseg > 1) PCTC_CUDA(cudaStreamWaitEvent(stream, pipe->w_ready[sg], 0));
+      Epilogue e;
+      e.kind = EPI_LSE_PARTIAL;
+      e.bias = bias;
+      e.v0 = v0;
+      e.partial = d_partial;
+      e.nsplit = per_seg;
+      if (pl.use_umma) {                       // never more splits than column tiles of the segment
+        const int tiles = (int)((rows + 255) / 256);
+        if (e.nsplit > tiles) e.nsplit = tiles;
+      }
+      e.partial_stride = per_seg * nseg;
+      e.partial_offset = slots;
+      GemmCall c{d_X, D, false, (const char*)W + (size_t)v0 * D * pl.elem, D, false, M, (int)rows, D};
+      PCTC_CUDA(run_gemm(pl.use_umma, pl.bf16, c, e, d_status, stream));
+      slots += e.nsplit;
+    }
+    // unused slots of the stride hold (-inf, 0) so that the combine may read the full stride
+    PCTC_CUDA(lse_combine(d_partial, per_seg * nseg * pps, M, d_lambda, stream));
+    return PCTC_OK;
+  };
+
+  if (pipe && pipe->nseg > 1) {
+    // W is still in flight: start with what can run on its first rows, do the DP once it is complete
+    PCTC_CUDA(cudaMemsetAsync(d_partial, 0, (size_t)M * 64 * 8, stream));   // (0, 0): empty slots are skipped
+    if ((st = normaliser()) != PCTC_OK) return st;
+    if ((st = subset_logits_and_dp()) != PCTC_OK) return st;
+  } else {
+    if ((st = subset_logits_and_dp()) != PCTC_OK) return st;
+    if ((st = normaliser()) != PCTC_OK) return st;
   }
   PCTC_CUDA(cudaStreamWaitEvent(stream, aux.join, 0));
   PCTC_CUDA(finalize_loss(d_lambda, bm, N, loss, d_flags, dp.roww, stream));
@@ -431,6 +488,17 @@ pctc_status_t pruned_ctc_fwd_bwd_traced(const pctc_problem_t* p, const void* hid
       PCTC_MARK(PCTC_PHASE_DBIAS);
       PCTC_CUDA(column_sums(d_chunk, pl.bf16, pl.chunk, M, Cc, dbias, pl.bf16, v0, p->accumulate_dW != 0, stream));
     }
+    if (pipe && pipe->dW_host && !p->skip_dW) {          // these rows of dW are final: send them home now
+      cudaEvent_t ev = aux.chunk_done[ci & 1];
+      PCTC_CUDA(cudaEventRecord(ev, stream));
+      PCTC_CUDA(cudaStreamWaitEvent(aux.copy_out, ev, 0));
+      PCTC_CUDA(cudaMemcpyAsync(pipe->dW_host + (size_t)v0 * D * pl.elem, (const char*)dW + (size_t)v0 * D * pl.elem,
+                                (size_t)Cc * D * pl.elem, cudaMemcpyDeviceToHost, aux.copy_out));
+    }
+  }
+  if (pipe && pipe->dW_host && !p->skip_dW && !p->forward_only) {   // the caller's stream covers those copies
+    PCTC_CUDA(cudaEventRecord(aux.copies_done, aux.copy_out));
+    PCTC_CUDA(cudaStreamWaitEvent(stream, aux.copies_done, 0));
   }
   PCTC_MARK(PCTC_PHASE_FINISH);
   if (!p->forward_only) PCTC_CUDA(unstack_cast(d_dHacc, dH, N, pl.T, D, pl.bf16, bm.T_n, bm.row0, stream));
@@ -447,6 +515,19 @@ pctc_status_t pruned_ctc_fwd_bwd_traced(const pctc_problem_t* p, const void* hid
 #undef PCTC_MARK
 #undef PCTC_CUDA
   return PCTC_OK;
+}
+}  // namespace
+
+extern "C" {
+
+pctc_status_t pruned_ctc_fwd_bwd_traced(const pctc_problem_t* p, const void* hidden, const void* W,
+                                        const void* bias, const int32_t* targets, const int32_t* input_lengths,
+                                        const int32_t* target_lengths, float* loss, void* dH, void* dW,
+                                        void* dbias, int32_t* subset_out, int32_t* K_out,
+                                        int32_t* relabeled_out, int32_t* utt_flags, void* workspace,
+                                        size_t workspace_bytes, void* stream_v, pctc_trace_t* trace) {
+  return run_call(p, hidden, W, bias, targets, input_lengths, target_lengths, loss, dH, dW, dbias, subset_out, K_out,
+                  relabeled_out, utt_flags, workspace, workspace_bytes, stream_v, trace, nullptr);
 }
 
 namespace {
@@ -553,19 +634,41 @@ pctc_status_t pruned_ctc_fwd_bwd_host(const pctc_problem_t* p, const void* hidde
   do {                                               \
     if ((call) != cudaSuccess) return PCTC_ERR_CUDA; \
   } while (0)
+  Aux aux;
+  if (get_aux(&aux) != cudaSuccess) return PCTC_ERR_CUDA;
+  HostPipe pipe;
+  pipe.dW_host = (char*)dW;       // rows of dW are copied out chunk by chunk while the backward pass runs
+  // The small inputs go first on the caller's stream; W follows on a copy stream in four row
+  // segments, and the normaliser kernel of each segment starts as soon as that segment has landed.
+  const int elem = (p->dtype == PCTC_BF16) ? 2 : 4;
+  const size_t row_bytes = (size_t)p->D * elem;
+  pipe.nseg = (p->V >= 4 * 4096) ? 4 : 0;
+  pipe.seg_rows = ((p->V + 3) / 4 + 255) / 256 * 256;
   PCTC_CUDA(cudaMemcpyAsync(d + h.o_hidden, hidden, h.b_hidden, cudaMemcpyHostToDevice, stream));
-  PCTC_CUDA(cudaMemcpyAsync(d + h.o_W, W, h.b_W, cudaMemcpyHostToDevice, stream));
   if (bias) PCTC_CUDA(cudaMemcpyAsync(d + h.o_bias, bias, h.b_bias, cudaMemcpyHostToDevice, stream));
   if (h.b_targets) PCTC_CUDA(cudaMemcpyAsync(d + h.o_targets, targets, h.b_targets, cudaMemcpyHostToDevice, stream));
-  st = pruned_ctc_fwd_bwd(p, d + h.o_hidden, d + h.o_W, bias ? d + h.o_bias : nullptr,
-                          (const int32_t*)(d + h.o_targets), input_lengths, target_lengths, (float*)(d + h.o_loss),
-                          d + h.o_dH, d + h.o_dW, want_db ? d + h.o_dbias : nullptr, (int32_t*)(d + h.o_subset),
-                          (int32_t*)(d + h.o_K), (int32_t*)(d + h.o_rel), (int32_t*)(d + h.o_flags), d + h.o_ws,
-                          h.ws_bytes, stream_v);
+  if (pipe.nseg > 1) {
+    PCTC_CUDA(cudaEventRecord(aux.entry, stream));          // the staging area is free once earlier work is done
+    PCTC_CUDA(cudaStreamWaitEvent(aux.copy_in, aux.entry, 0));
+    for (int sg = 0; sg < pipe.nseg; ++sg) {
+      const long long v0 = (long long)sg * pipe.seg_rows;
+      if (v0 >= p->V) { pipe.nseg = sg; break; }
+      const long long rows = (p->V - v0 < pipe.seg_rows) ? (p->V - v0) : pipe.seg_rows;
+      PCTC_CUDA(cudaMemcpyAsync(d + h.o_W + (size_t)v0 * row_bytes, (const char*)W + (size_t)v0 * row_bytes,
+                                (size_t)rows * row_bytes, cudaMemcpyHostToDevice, aux.copy_in));
+      pipe.w_ready[sg] = aux.w_ready[sg];
+      PCTC_CUDA(cudaEventRecord(aux.w_ready[sg], aux.copy_in));
+    }
+  } else {
+    PCTC_CUDA(cudaMemcpyAsync(d + h.o_W, W, h.b_W, cudaMemcpyHostToDevice, stream));
+  }
+  st = run_call(p, d + h.o_hidden, d + h.o_W, bias ? d + h.o_bias : nullptr, (const int32_t*)(d + h.o_targets),
+                input_lengths, target_lengths, (float*)(d + h.o_loss), d + h.o_dH, d + h.o_dW,
+                want_db ? d + h.o_dbias : nullptr, (int32_t*)(d + h.o_subset), (int32_t*)(d + h.o_K),
+                (int32_t*)(d + h.o_rel), (int32_t*)(d + h.o_flags), d + h.o_ws, h.ws_bytes, stream_v, nullptr, &pipe);
   if (st != PCTC_OK) return st;
   PCTC_CUDA(cudaMemcpyAsync(loss, d + h.o_loss, (size_t)p->N * 4, cudaMemcpyDeviceToHost, stream));
   PCTC_CUDA(cudaMemcpyAsync(dH, d + h.o_dH, h.b_hidden, cudaMemcpyDeviceToHost, stream));
-  PCTC_CUDA(cudaMemcpyAsync(dW, d + h.o_dW, h.b_W, cudaMemcpyDeviceToHost, stream));
   if (want_db) PCTC_CUDA(cudaMemcpyAsync(dbias, d + h.o_dbias, h.b_bias, cudaMemcpyDeviceToHost, stream));
   if (subset_out) PCTC_CUDA(cudaMemcpyAsync(subset_out, d + h.o_subset, h.b_subset, cudaMemcpyDeviceToHost, stream));
   if (K_out) PCTC_CUDA(cudaMemcpyAsync(K_out, d + h.o_K, 4, cudaMemcpyDeviceToHost, stream));

@@ -36,8 +36,10 @@ struct Epilogue {
   const float* roww = nullptr;  // [M] 1 for frames of utterances in N+, else 0
   const int* U = nullptr;       // [K] selected classes
   const int* Kdev = nullptr;    // device scalar K
-  float2* partial = nullptr;    // [M, nsplit] (max, sum)
-  int nsplit = 1;
+  float2* partial = nullptr;    // [M, partial_stride] (max, sum) or (max, arg-max)
+  int nsplit = 1;               // column splits of this launch
+  int partial_stride = 0;       // split slots per row in `partial` (0: nsplit); a launch over a row
+  int partial_offset = 0;       // segment of B writes its splits at partial_offset .. +nsplit-1
   int accumulate = 0;           // EPI_ACCUM_F32 / EPI_STORE_OUT: add to the destination instead of overwriting
   int out_is_bf16 = 0;          // EPI_DLOGITS / EPI_STORE_OUT destination type
 };

@@ -144,7 +144,8 @@ __global__ void __launch_bounds__(NT) k_simt_gemm(const T* __restrict__ A, const
           const int j = s_idx[tid][q];
           if (j >= 0 && (v > best || (v == best && j < idx) || idx < 0)) { best = v; idx = j; }
         }
-        e.partial[(long long)i * e.nsplit + blockIdx.x] = make_float2(best, __int_as_float(idx));
+        e.partial[(long long)i * (e.partial_stride ? e.partial_stride : e.nsplit) + e.partial_offset + blockIdx.x] =
+            make_float2(best, __int_as_float(idx));
       }
     }
   }
@@ -164,7 +165,8 @@ __global__ void __launch_bounds__(NT) k_simt_gemm(const T* __restrict__ A, const
         float sum = 0.f;
         for (int q = 0; q < 16; ++q)
           if (!(s_red[1][tid][q] <= 0.f)) sum += s_red[1][tid][q] * __expf(s_red[0][tid][q] - mx);
-        e.partial[(long long)i * e.nsplit + blockIdx.x] = make_float2(mx, sum);
+        e.partial[(long long)i * (e.partial_stride ? e.partial_stride : e.nsplit) + e.partial_offset + blockIdx.x] =
+            make_float2(mx, sum);
       }
     }
   }

@@ -454,6 +454,7 @@ k_umma_gemm(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
     unsigned char* stage = smem + off_stage(CTAS, EPI, EW) + ew * STAGE_WARP_BYTES;   // this warp's two staging boxes
     const unsigned swz64 = (unsigned)((lane >> 1) & 3); // 64-byte swizzle of a staged 64-byte row
     unsigned nbox = 0;                                  // boxes stored so far by this warp (buffer parity)
+    const int pstride = a.e.partial_stride ? a.e.partial_stride : a.nsplit;   // split slots per row
     unsigned it = 0;
     bool ok = true;
     for (int u = group; u < units && ok; u += ngroups) {
@@ -629,9 +630,11 @@ k_umma_gemm(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
       }
 
       if (EPI == EPI_LSE_PARTIAL && ok && row_ok)
-        a.e.partial[((long long)i * a.nsplit + sp) * (EW / 4) + (ew >> 2)] = make_float2(run_max2 * LN2, run_sum);
+        a.e.partial[((long long)i * pstride + a.e.partial_offset + sp) * (EW / 4) + (ew >> 2)] =
+            make_float2(run_max2 * LN2, run_sum);
       if (EPI == EPI_ARGMAX_PARTIAL && ok && row_ok)
-        a.e.partial[((long long)i * a.nsplit + sp) * (EW / 4) + (ew >> 2)] = make_float2(best_z, __int_as_float(best_j));
+        a.e.partial[((long long)i * pstride + a.e.partial_offset + sp) * (EW / 4) + (ew >> 2)] =
+            make_float2(best_z, __int_as_float(best_j));
     }
     if (epi_uses_tma_store(EPI) && lane == 0) bulk_wait0();   // this warp's stores have completed
   }

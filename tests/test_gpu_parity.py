@@ -297,3 +297,36 @@ def test_random_small_shapes(lib, path, case):
     ref = H.run_oracle(batch, beam=beam if beam > 0 else None)
     tol = (2e-3, 1e-2) if dtype == "bf16" else (2e-5, 5e-4)
     H.assert_parity(gpu, ref, batch, tol=tol)
+
+
+@pytest.mark.parametrize("V,D", [(8192 + 384, 256), (4 * 4096 + 1000, 64)])   # one upload / four segments of W
+def test_host_buffer_entry_point_matches_device_entry_point(lib, V, D):
+    import torch
+    batch = wl.make_batch(small("c3", V=V, D=D, N=4, T_div=4, U_div=2), with_bias=True, permute_ids=True)
+    dev_out = H.run_gpu(lib, batch, chunk=2048)
+    tdt = torch.bfloat16
+    hid = torch.from_numpy(batch.hidden).to(tdt).pin_memory()
+    W = torch.from_numpy(batch.W).to(tdt).pin_memory()
+    bias = torch.from_numpy(batch.bias).to(tdt).pin_memory()
+    tg = torch.from_numpy(batch.targets).pin_memory()
+    res = None
+    for _ in range(2):                                   # the scratch buffer and outputs are reusable
+        res = lib.pruned_ctc_fwd_bwd_host(hid, W, bias, tg, batch.input_lengths, batch.target_lengths, batch.blank,
+                                          chunk=2048, scratch=None if res is None else res["scratch"], out=res)
+        torch.cuda.synchronize()
+        for k in ("loss", "dH", "dW", "dbias"):
+            got = res[k].float().numpy()
+            if V < 4 * 4096:
+                np.testing.assert_array_equal(got, dev_out[k])
+            else:
+                # W arrives in four segments and the normaliser is summed per segment: another
+                # summation order, so the last bits of lambda (and a few bf16 roundings) may differ
+                assert H.rel_fro(got, dev_out[k]) <= 1e-3
+        K = int(res["K"][0])
+        np.testing.assert_array_equal(res["subset"].numpy()[:K], dev_out["subset"][:K])
+        np.testing.assert_array_equal(res["relabeled"].numpy(), dev_out["relabeled"])
+        np.testing.assert_array_equal(res["flags"].numpy(), dev_out["flags"])
+    ref = H.run_oracle(batch)
+    host = {k: (v.float().numpy() if v.is_floating_point() else v.numpy()) for k, v in res.items()
+            if hasattr(v, "numpy") and k != "scratch"}
+    H.assert_parity(host, ref, batch)

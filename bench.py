@@ -332,8 +332,9 @@ def main():
                              tflops=round(split_flops[k] / (phase_ms[k] * 1e-3) / 1e12, 2))
 
     # kernels launched by the library inside the timed region
-    dp_launches = 3 if args.beam > 0 else 2
-    launches_per_step = 3 + 1 + 2 + 2 + dp_launches + 1 + (2 if args.frozen_head else 3) * nchunks + 1
+    dp_launches = 4 if args.beam > 0 else 2      # sweeps (+ best-alignment sweeps, arc flags), occupancies
+    # subset (3), stacking, gather + Z_U, DP, normaliser + combine, loss, row clean-up, chunks, un-stacking
+    launches_per_step = 3 + 1 + 2 + dp_launches + 2 + 1 + 1 + (2 if args.frozen_head else 3) * nchunks + 1
     gpu_launches = launches_per_step * args.steps
 
     # ---- end to end through the host-buffer entry point ----

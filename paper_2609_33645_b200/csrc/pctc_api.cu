@@ -440,6 +440,7 @@ pctc_status_t run_call(const pctc_problem_t* p, const void* hidden, const void* 
   }
   PCTC_CUDA(cudaStreamWaitEvent(stream, aux.join, 0));
   PCTC_CUDA(finalize_loss(d_lambda, bm, N, loss, d_flags, dp.roww, stream));
+  if (!p->forward_only) PCTC_CUDA(zero_nonfinite_rows(d_X, M, D, pl.elem, bm.row_utt, d_flags, stream));
 
   // ---- lines 11-17: backward, one vocabulary chunk at a time ----
   for (int ci = 0; ci < pl.nchunks && !p->forward_only; ++ci) {

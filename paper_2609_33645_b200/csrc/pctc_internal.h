@@ -98,6 +98,10 @@ cudaError_t subset_and_relabel(const int* targets, int target_stride, const int*
 cudaError_t stack_frames(const void* hidden, void* X, int N, int T, int D, int elem_bytes,
                          const int* row_utt, const int* row0, int M, cudaStream_t stream);
 
+// Zero the stacked frames of utterances flagged non-finite (flag 2), before the backward pass.
+cudaError_t zero_nonfinite_rows(void* X, int M, int D, int elem_bytes, const int* row_utt, const int* utt_flags,
+                                cudaStream_t stream);
+
 // dH[n,t,:] = T(acc[row0[n]+t,:]) for t < T_n, zero for padded frames.
 cudaError_t unstack_cast(const float* acc, void* dH, int N, int T, int D, bool out_bf16,
                          const int* T_n, const int* row0, cudaStream_t stream);

@@ -136,6 +136,14 @@ __global__ void k_gather_rows(const char* __restrict__ W, char* __restrict__ W_U
   else zero_row(dst, row_bytes);
 }
 
+// --- frames of an utterance with a non-finite loss (NaN/Inf in its states): the stacked copy is
+// zeroed before the backward pass, so that 0 * NaN cannot leak into dW through dZ^T X ---
+__global__ void k_zero_nonfinite_rows(char* __restrict__ X, size_t row_bytes, const int* __restrict__ row_utt,
+                                      const int* __restrict__ flags) {
+  const int m = blockIdx.x;
+  if (flags[row_utt[m]] & 2) zero_row(X + (size_t)m * row_bytes, row_bytes);
+}
+
 // --- db_c = dZ_c^T 1 (Algorithm 1 line 16): fixed summation order, no atomics -------------------
 template <typename TIn, typename TOut>
 __global__ void k_column_sums(const TIn* __restrict__ chunk, long long ld, int M, int cols,
@@ -245,6 +253,12 @@ cudaError_t stack_frames(const void* hidden, void* X, int N, int T, int D, int e
                          const int* row_utt, const int* row0, int M, cudaStream_t stream) {
   (void)N;
   k_stack_frames<<<M, 128, 0, stream>>>((const char*)hidden, (char*)X, T, (size_t)D * elem_bytes, row_utt, row0);
+  return cudaGetLastError();
+}
+
+cudaError_t zero_nonfinite_rows(void* X, int M, int D, int elem_bytes, const int* row_utt, const int* utt_flags,
+                                cudaStream_t stream) {
+  k_zero_nonfinite_rows<<<M, 64, 0, stream>>>((char*)X, (size_t)D * elem_bytes, row_utt, utt_flags);
   return cudaGetLastError();
 }
 

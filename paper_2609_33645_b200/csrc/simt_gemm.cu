@@ -117,7 +117,7 @@ __global__ void __launch_bounds__(NT) k_simt_gemm(const T* __restrict__ A, const
           const float p = __expf(a + bias_at<T>(e.bias, v) - lam);
           const int jj = e.vmap[v];
           const float gam = (jj >= 0) ? e.gamma[(long long)i * e.ld_gamma + jj] : 0.f;
-          reinterpret_cast<T*>(e.out)[(long long)i * e.ld + j] = T(w * (p - gam));
+          reinterpret_cast<T*>(e.out)[(long long)i * e.ld + j] = T(w == 0.f ? 0.f : w * (p - gam));
         } else if (EPI == EPI_ACCUM_F32) {
           float* dst = reinterpret_cast<float*>(e.out) + (long long)i * e.ld + j;
           *dst = e.accumulate ? (*dst + a) : a;

@@ -540,6 +540,10 @@ k_umma_gemm(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
 #pragma unroll
                 for (int c = 0; c < 32; ++c) v[c] *= w;
               }
+              if (w == 0.f) {                          // excluded utterance: exact zeros, whatever its logits are
+#pragma unroll
+                for (int c = 0; c < 32; ++c) v[c] = 0.f;
+              }
             }
             constexpr int NBOX = (EPI == EPI_ACCUM_F32) ? 2 : 1;     // boxes per group
 #pragma unroll

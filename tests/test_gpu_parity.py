@@ -330,3 +330,26 @@ def test_host_buffer_entry_point_matches_device_entry_point(lib, V, D):
     host = {k: (v.float().numpy() if v.is_floating_point() else v.numpy()) for k, v in res.items()
             if hasattr(v, "numpy") and k != "scratch"}
     H.assert_parity(host, ref, batch)
+
+
+@pytest.mark.parametrize("path", [SIMT, AUTO])
+def test_non_finite_states_exclude_only_their_utterance(lib, path):
+    cfg = small("c2", V=4096, D=128, N=4, T_div=8, U_div=4)
+    batch = wl.make_batch(cfg, with_bias=True)
+    clean = wl.make_batch(cfg, with_bias=True)
+    batch.hidden[1, 3, 5] = np.nan                     # one NaN state in utterance 1
+    batch.hidden[2, 0, :4] = np.inf                    # Inf states in utterance 2
+    gpu = H.run_gpu(lib, batch, gemm_path=path)
+    assert list(gpu["flags"]) == [0, 2, 2, 0]
+    assert gpu["loss"][1] == 0 and gpu["loss"][2] == 0
+    assert np.all(gpu["dH"][1] == 0) and np.all(gpu["dH"][2] == 0)
+    assert np.isfinite(gpu["dW"]).all() and np.isfinite(gpu["dbias"]).all() and np.isfinite(gpu["dH"]).all()
+    # the other utterances are untouched: same result as a batch that holds only them
+    keep = [0, 3]
+    sub = dataclasses.replace(clean, hidden=clean.hidden[keep], targets=clean.targets[keep],
+                              input_lengths=clean.input_lengths[keep], target_lengths=clean.target_lengths[keep],
+                              cfg=dataclasses.replace(cfg, N=2))
+    ref = H.run_oracle(sub)
+    np.testing.assert_allclose(gpu["loss"][keep], ref["loss"], rtol=2e-3)
+    assert H.rel_fro(gpu["dW"], ref["dW"]) <= 1e-2
+    assert H.rel_fro(gpu["dH"][keep][:, : sub.hidden.shape[1]], ref["dH"]) <= 1e-2

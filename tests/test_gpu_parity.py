@@ -353,3 +353,35 @@ def test_non_finite_states_exclude_only_their_utterance(lib, path):
     np.testing.assert_allclose(gpu["loss"][keep], ref["loss"], rtol=2e-3)
     assert H.rel_fro(gpu["dW"], ref["dW"]) <= 1e-2
     assert H.rel_fro(gpu["dH"][keep][:, : sub.hidden.shape[1]], ref["dH"]) <= 1e-2
+
+
+def test_workspace_guards_stay_intact_and_trace_is_well_formed(lib):
+    import torch
+    batch = wl.make_batch(small("c3", V=8192 + 384, D=256, N=4, T_div=4, U_div=2), with_bias=True, permute_ids=True)
+    dev = torch.device("cuda:0")
+    hidden = torch.from_numpy(batch.hidden).to(dev).to(torch.bfloat16)
+    W = torch.from_numpy(batch.W).to(dev).to(torch.bfloat16)
+    bias = torch.from_numpy(batch.bias).to(dev).to(torch.bfloat16)
+    targets = torch.from_numpy(batch.targets).to(dev)
+    N, T, D = hidden.shape
+    for beam in (0.0, 8.0):
+        prob = lib.make_problem(N, T, D, W.shape[0], lib.PCTC_BF16, batch.blank, beam, 2048, targets.shape[1])
+        need = lib.workspace_bytes(prob, batch.input_lengths, batch.target_lengths)
+        guard = 4096
+        buf = torch.full((guard + need + guard,), 0xA5, dtype=torch.uint8, device=dev)
+        ws = buf[guard:guard + need]                      # the library is told about exactly `need` bytes
+        trace = lib.Trace(lib.Trace.capacity_for(W.shape[0], 2048))
+        res = lib.pruned_ctc_fwd_bwd(hidden, W, bias, targets, batch.input_lengths, batch.target_lengths,
+                                     batch.blank, beam=beam, chunk=2048, workspace=ws, trace=trace, check_status=True)
+        torch.cuda.synchronize()
+        assert res["workspace"].data_ptr() == ws.data_ptr()
+        assert bool((buf[:guard] == 0xA5).all()) and bool((buf[guard + need:] == 0xA5).all())
+        spans = trace.spans()
+        kinds = [k for k, _ in spans if k >= 0]
+        names = [lib.PHASES[k] for k in kinds]
+        nchunks = (W.shape[0] + 2047) // 2048
+        assert names.count("dlogits") == nchunks and names.count("dh") == nchunks and names.count("dw") == nchunks
+        assert names.count("dbias") == nchunks and names.count("lse") == 1 and names.count("dp") == 1
+        assert all(ms >= 0 for k, ms in spans if k >= 0)
+    ref = H.run_oracle(batch, beam=8.0)
+    np.testing.assert_allclose(res["loss"].cpu().numpy(), ref["loss"], rtol=2e-3)

@@ -231,11 +231,19 @@ def main():
     local_rank = int(os.environ.get("LOCAL_RANK", "0"))
     if not torch.cuda.is_available():
         raise SystemExit("bench.py needs a CUDA device: the hot path has no CPU implementation")
-    torch.cuda.set_device(local_rank)
-    dev = torch.device("cuda", local_rank)
+    local_dev = local_rank % torch.cuda.device_count()
+    torch.cuda.set_device(local_dev)
+    dev = torch.device("cuda", local_dev)
+    # NCCL over NVLink for the timing reduction; PCTC_BENCH_BACKEND=gloo lets several ranks share one
+    # GPU when the multi-rank code path is exercised on a single-GPU machine
+    backend = os.environ.get("PCTC_BENCH_BACKEND", "nccl")
+    red_dev = dev if backend == "nccl" else None
     if world > 1:
         import torch.distributed as dist
-        dist.init_process_group("nccl", device_id=dev)
+        if backend == "nccl":
+            dist.init_process_group("nccl", device_id=dev)
+        else:
+            dist.init_process_group(backend)
     if rank == 0:
         build.build()
     if world > 1:
@@ -280,7 +288,7 @@ def main():
     torch.cuda.synchronize()
 
     traces = [binding.Trace(binding.Trace.capacity_for(V, chunk)) for _ in range(args.steps)]
-    sampler = ClockSampler(local_rank)
+    sampler = ClockSampler(local_dev)
     if rank == 0:
         sampler.start()
         time.sleep(0.25)
@@ -301,7 +309,7 @@ def main():
     status = binding.workspace_status(res["workspace"])
     if status != 0:
         raise SystemExit(f"device status word {status}: a bounded wait gave up")
-    ms_total, frames_all, flops_all = reduce_over_ranks(ms_total, float(M), flops_per_step, dev)
+    ms_total, frames_all, flops_all = reduce_over_ranks(ms_total, float(M), flops_per_step, red_dev)
     ms_per_step = ms_total / args.steps
     value = frames_all / (ms_per_step * 1e-3)
 
@@ -354,7 +362,7 @@ def main():
         e1.record()
         torch.cuda.synchronize()
         ms_e2e = e0.elapsed_time(e1) / args.e2e_steps
-        ms_e2e, _, _ = reduce_over_ranks(ms_e2e, 0.0, 0.0, dev)
+        ms_e2e, _, _ = reduce_over_ranks(ms_e2e, 0.0, 0.0, red_dev)
         h2d = h_hidden.numel() * h_hidden.element_size() + h_W.numel() * h_W.element_size() + h_targets.numel() * 4
         d2h = (N * 4 + h_hidden.numel() * h_hidden.element_size() + h_W.numel() * h_W.element_size()
                + (int(tl.sum()) + 1) * 4 + 4 + h_targets.numel() * 4 + N * 4)

@@ -8,13 +8,15 @@
 // memory and runs its own epilogue.  B then crosses L2 -> shared memory once per pair instead of
 // once per CTA, and the freed shared memory deepens the ring to six stages.
 //
-// One persistent CTA per SM, 320 threads in three roles:
-//   warp 0      TMA producer: 128-byte-swizzled operand tiles into a 4-stage ring
-//   warp 1      MMA issuer: tcgen05.mma 128x256x16 from shared-memory descriptors
-//               into one of two 256-column accumulators in tensor memory
-//   warps 2..9  epilogue: tcgen05.ld (one accumulator row per thread; two warps per
-//               tensor-memory lane quarter, 128 columns each), the fused arithmetic,
-//               stores; runs while the next tile's MMAs issue
+// One persistent CTA per SM, 192 or 320 threads in three roles:
+//   warp 0      TMA producer: 128-byte-swizzled operand tiles into a 5- or 6-stage ring
+//   warp 1      MMA issuer (in the pair's leader): tcgen05.mma 256x256x16 from shared-memory
+//               descriptors into one of two 256-column accumulators in tensor memory
+//   warps 2..   epilogue, 4 or 8 warps (template parameter EW): tcgen05.ld (one accumulator
+//               row per thread; with 8 warps two share a tensor-memory lane quarter and take
+//               128 columns each), the fused arithmetic, stores (staged through shared
+//               memory and written by TMA for dlogits, dX, dW); runs while the next tile's
+//               MMAs issue
 // Operands may be K-major (k contiguous) or MN-major (the transposed storage),
 // chosen at run time through the descriptors, so that dX += dZ W and
 // dW = dZ^T X need no transposed copies.
@@ -41,11 +43,12 @@ namespace {
 #define PCTC_TUNE_CTAS 2          // CTAs per tile: 2 = tcgen05 cta_group::2 pairs, 1 = independent CTAs
 #endif
 
-constexpr int BM = 128, BN = 256, BK = 64;
-constexpr int MAX_STAGES = 6;
 #ifndef PCTC_TUNE_EPI_WARPS
 #define PCTC_TUNE_EPI_WARPS 0     // 0: by the contraction depth; 4 or 8: forced
 #endif
+
+constexpr int BM = 128, BN = 256, BK = 64;
+constexpr int MAX_STAGES = 6;
 // Epilogue warps per CTA (template parameter EW): 4 = one per tensor-memory lane quarter, 256
 // columns each; 8 = two per quarter, 128 columns each.  Eight hide the latency of a math-heavy
 // epilogue when the main loop of a tile is short (narrow heads); four leave the ring one stage

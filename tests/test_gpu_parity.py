@@ -385,3 +385,11 @@ def test_workspace_guards_stay_intact_and_trace_is_well_formed(lib):
         assert all(ms >= 0 for k, ms in spans if k >= 0)
     ref = H.run_oracle(batch, beam=8.0)
     np.testing.assert_allclose(res["loss"].cpu().numpy(), ref["loss"], rtol=2e-3)
+
+
+def test_bf16_shapes_the_tensor_core_path_does_not_cover_fall_to_the_fma_kernels(lib):
+    # V and D that are no multiples of 8: TMA row pitches would be misaligned, so AUTO uses the FMA kernels
+    cfg = small("c2", V=5003, D=100, N=3, T_div=10, U_div=5)
+    batch = wl.make_batch(cfg, with_bias=True, permute_ids=True)
+    gpu = H.run_gpu(lib, batch, gemm_path=AUTO)
+    H.assert_parity(gpu, H.run_oracle(batch), batch)

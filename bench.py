@@ -339,6 +339,13 @@ def main():
         per_kernel[k] = dict(ms=round(phase_ms[k], 4), launches=phase_cnt[k] // args.steps,
                              tflops=round(split_flops[k] / (phase_ms[k] * 1e-3) / 1e12, 2))
 
+    # DRAM bytes of the dominant kernel's launches of one step, from the ncu capture summarised in
+    # profiles/umma_gemm_c4_speed_of_light.md (default workload and chunk only)
+    traffic = None
+    if args.config == "c4" and not args.vocab and chunk == 8192 and not args.frozen_head and args.beam == 0:
+        traffic = dict(bytes_per_step=51.1e9, launches_per_step=58, bytes_per_launch_avg=51.1e9 / 58,
+                       source="ncu dram__bytes.sum.per_second x duration, one launch of each kind, scaled by launches")
+
     # kernels launched by the library inside the timed region
     dp_launches = 4 if args.beam > 0 else 2      # sweeps (+ best-alignment sweeps, arc flags), occupancies
     # subset (3), stacking, gather + Z_U, DP, normaliser + combine, loss, row clean-up, chunks, un-stacking
@@ -406,7 +413,7 @@ def main():
         flops_per_step=flops_per_step,
         phase_ms={k: round(v, 4) for k, v in phase_ms.items()},
         roofline=dict(bound="tensor", achieved=achieved_tflops, peak=peak, unit="TFLOP/s",
-                      frac=achieved_tflops / peak, traffic=None,
+                      frac=achieved_tflops / peak, traffic=traffic,
                       kernel="k_umma_gemm (all fused-epilogue instances: lse, dlogits, dh, dw)",
                       launches_per_step=gemm_launches, ms_per_step=gemm_ms,
                       peak_source="%s bf16_tflops_sustained (kernel timed inside a long step)" % peaks["source"],

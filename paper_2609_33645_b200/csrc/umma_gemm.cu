@@ -90,7 +90,10 @@ struct SharedTail {   // barriers and flags
 //   list           8 warps x (128 indices in U, -1 if the column's class is not selected, + group masks) (dlogits)
 constexpr int STAGE_BOX_BYTES = 2048;                      // one staged box: 32 rows x 64 B
 constexpr int STAGE_WARP_BYTES = 2 * STAGE_BOX_BYTES;      // double-buffered
-constexpr bool epi_uses_tma_store(int epi) { return epi == EPI_DLOGITS || epi == EPI_ACCUM_F32 || epi == EPI_STORE_OUT; }
+constexpr bool epi_uses_tma_store(int epi) {
+  return epi == EPI_DLOGITS || epi == EPI_ACCUM_F32 || epi == EPI_STORE_OUT || epi == EPI_SUBSET_LOGP;
+}
+constexpr bool epi_fp32_boxes(int epi) { return epi == EPI_ACCUM_F32 || epi == EPI_SUBSET_LOGP; }
 constexpr bool epi_uses_bias(int epi) {
   return epi == EPI_LSE_PARTIAL || epi == EPI_SUBSET_LOGP || epi == EPI_DLOGITS || epi == EPI_ARGMAX_PARTIAL;
 }
@@ -521,6 +524,11 @@ k_umma_gemm(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
             if (j0 >= n_eff) break;                   // warp-uniform
             float v[32];
             tmem_ld32(taddr + g0, v);
+            if (EPI == EPI_SUBSET_LOGP) {               // Z_U (or S = Z_U - lambda); columns past K are written as 0
+#pragma unroll
+              for (int c = 0; c < 32; ++c)
+                v[c] = (j0 + c < n_eff) ? v[c] + (has_bias ? sb[g0 + c] : 0.f) - lam : 0.f;
+            }
             if (EPI == EPI_DLOGITS) {
               if (has_bias) {
 #pragma unroll
@@ -548,7 +556,7 @@ k_umma_gemm(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
                 for (int c = 0; c < 32; ++c) v[c] = 0.f;
               }
             }
-            constexpr int NBOX = (EPI == EPI_ACCUM_F32) ? 2 : 1;     // boxes per group
+            constexpr int NBOX = epi_fp32_boxes(EPI) ? 2 : 1;        // boxes per group
 #pragma unroll
             for (int b = 0; b < NBOX; ++b) {
               if (NBOX == 2 && j0 + b * 16 >= n_eff) break;          // warp-uniform
@@ -556,7 +564,7 @@ k_umma_gemm(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
               __syncwarp();
               unsigned char* box = stage + (nbox & 1u) * STAGE_BOX_BYTES;
               unsigned char* row = box + lane * 64;
-              if (EPI == EPI_ACCUM_F32) {
+              if (epi_fp32_boxes(EPI)) {
 #pragma unroll
                 for (int c4 = 0; c4 < 4; ++c4)
                   *reinterpret_cast<float4*>(row + (((unsigned)c4 ^ swz64) << 4)) =
@@ -598,13 +606,6 @@ k_umma_gemm(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
 #pragma unroll
               for (int c = 0; c < 32; ++c)
                 if (j0 + c < n_eff) dst[c] = v[c];
-            }
-          } else if (EPI == EPI_SUBSET_LOGP) {
-            if (row_ok) {
-              float* dst = (float*)a.e.out + (long long)i * a.e.ld + j0;
-#pragma unroll
-              for (int c = 0; c < 32; ++c)
-                if (j0 + c < n_eff) dst[c] = v[c] + (has_bias ? sb[cg * 32 + c] : 0.f) - lam;
             }
           } else if (EPI == EPI_ARGMAX_PARTIAL) {
 #pragma unroll
@@ -786,7 +787,7 @@ cudaError_t umma_gemm(const __nv_bfloat16* A, long long lda, bool a_mn_major,
   bool ok = true;
   tmC = CUtensorMap{};
   // output boxes of the staged epilogues: 32 rows x 32 columns, clipped to the [m, n] extent
-  if (e.kind == EPI_ACCUM_F32) {
+  if (e.kind == EPI_ACCUM_F32 || e.kind == EPI_SUBSET_LOGP) {
     if ((e.ld % 4) || ((size_t)e.out & 15)) return cudaErrorInvalidValue;
     ok = ok && make_map(&tmC, e.out, (unsigned long long)n, (unsigned long long)m, (unsigned long long)e.ld, 16, 32, true);
   } else if (e.kind == EPI_DLOGITS || e.kind == EPI_STORE_OUT) {

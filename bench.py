@@ -34,7 +34,6 @@ from paper_2609_33645_b200 import workloads as wl  # noqa: E402
 
 METRIC = "pruned_ctc_fwd_bwd_frames_per_s"
 UNIT = "frames/s"
-DEFAULT_CHUNK = 8192      # vocabulary chunk width C passed to the library
 
 
 def load_peaks():
@@ -264,15 +263,13 @@ def main():
     M, D, V, N = batch.M, cfg.D, cfg.V, cfg.N
     flops_per_step = (6.0 if args.frozen_head else 8.0) * M * D * V
 
-    chunk = args.chunk or DEFAULT_CHUNK
     max_K_pre = 0
     if args.promise_k:
         max_K_pre = 1 + int(np.unique(np.concatenate([batch.targets[n, : tl[n]] for n in range(N)])).size)
     prob = binding.make_problem(N, batch.T, D, V, binding.PCTC_BF16 if cfg.dtype == "bf16" else binding.PCTC_FP32,
-                                batch.blank, args.beam, chunk, batch.targets.shape[1], max_K=max_K_pre)
+                                batch.blank, args.beam, args.chunk, batch.targets.shape[1], max_K=max_K_pre)
     ws_bytes = binding.workspace_bytes(prob, il, tl)
-    chunk = args.chunk or DEFAULT_CHUNK
-    nchunks = (V + chunk - 1) // chunk
+    chunk, nchunks = binding.chunk_width(prob, il, tl)     # the library's default unless --chunk is given
     call = dict(beam=args.beam, chunk=chunk)
     max_K = 0
     if args.promise_k:

@@ -95,6 +95,21 @@ pctc_status_t pctc_workspace_bytes(const pctc_problem_t* problem,
                                    size_t* bytes_out);
 
 /*
+ * The vocabulary chunk width C a call on this problem will use, and the number of
+ * chunks ceil(V / C) (host-only; touches no device).  With problem->chunk > 0 it
+ * is that value rounded up to the tile width of the path that runs; with 0 it is
+ * the library's choice: 4,096 for fp32; for bf16 32,768 (D <= 1,024), 16,384
+ * (D <= 2,048) or 8,192 columns, halved down to no less than 8,192 while the
+ * [M, C] chunk temporary of Algorithm 1 (lines 12-13) would exceed 512 MiB.  The
+ * chunk width changes the order of summation only, never what is computed.
+ * nchunks_out may be NULL.  Same argument checks as pctc_workspace_bytes.
+ */
+pctc_status_t pctc_chunk_width(const pctc_problem_t* problem,
+                               const int32_t* input_lengths_host,
+                               const int32_t* target_lengths_host,
+                               int32_t* chunk_out, int32_t* nchunks_out);
+
+/*
  * Algorithm 1, forward and backward in one call.
  *
  * Steps, all on `stream`:

@@ -20,7 +20,7 @@ PCTC_BF16, PCTC_FP32 = 0, 1
 GEMM_AUTO, GEMM_SIMT = 0, 1
 UTT_INFEASIBLE, UTT_NONFINITE, UTT_BAD_TARGET, UTT_SUBSET_OVERFLOW = 1, 2, 4, 8
 
-EXPORTS = ("pctc_workspace_bytes", "pruned_ctc_fwd_bwd", "pruned_ctc_fwd_bwd_traced", "pctc_gemm_bf16",
+EXPORTS = ("pctc_workspace_bytes", "pctc_chunk_width", "pruned_ctc_fwd_bwd", "pruned_ctc_fwd_bwd_traced", "pctc_gemm_bf16",
            "pctc_workspace_status", "pctc_status_string", "pctc_host_call_scratch_bytes",
            "pruned_ctc_fwd_bwd_host", "pctc_subset_relabel_noalloc", "pctc_greedy_workspace_bytes",
            "pctc_greedy_decode")
@@ -94,6 +94,8 @@ def load() -> ctypes.CDLL:
     vp, i32p = ctypes.c_void_p, ctypes.POINTER(ctypes.c_int32)
     lib.pctc_workspace_bytes.restype = ctypes.c_int
     lib.pctc_workspace_bytes.argtypes = [ctypes.POINTER(Problem), i32p, i32p, ctypes.POINTER(ctypes.c_size_t)]
+    lib.pctc_chunk_width.restype = ctypes.c_int
+    lib.pctc_chunk_width.argtypes = [ctypes.POINTER(Problem), i32p, i32p, i32p, i32p]
     lib.pruned_ctc_fwd_bwd.restype = ctypes.c_int
     lib.pruned_ctc_fwd_bwd.argtypes = [ctypes.POINTER(Problem), vp, vp, vp, vp, i32p, i32p,
                                        vp, vp, vp, vp, vp, vp, vp, vp, vp, ctypes.c_size_t, vp]
@@ -148,6 +150,16 @@ def workspace_bytes(problem: Problem, input_lengths, target_lengths) -> int:
     if st != 0:
         raise PctcError(st, "pctc_workspace_bytes")
     return int(out.value)
+
+
+def chunk_width(problem: Problem, input_lengths, target_lengths):
+    """(C, number of chunks) the library will use for this problem (its default when problem.chunk is 0)."""
+    il, tl = _i32(input_lengths), _i32(target_lengths)
+    c, n = ctypes.c_int32(0), ctypes.c_int32(0)
+    st = load().pctc_chunk_width(ctypes.byref(problem), _ptr_i32(il), _ptr_i32(tl), ctypes.byref(c), ctypes.byref(n))
+    if st != 0:
+        raise PctcError(st, "pctc_chunk_width")
+    return int(c.value), int(n.value)
 
 
 def _dptr(t) -> Optional[int]:

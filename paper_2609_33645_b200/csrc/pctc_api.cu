@@ -28,7 +28,15 @@ struct Plan {
   size_t meta_ints;  // T_n[N] | U_n[N] | row0[N+1] | row_utt[M]
 };
 
-int default_chunk(bool bf16) { return bf16 ? 8192 : 4096; }
+// Default chunk width C.  Every chunk costs three launches whose length grows with M*C*D, so a
+// narrow head (small D) is given wider chunks to keep each launch long against its start-up and tail;
+// the [M, C] temporary is held under 512 MiB whatever the shape, so it never grows with V.
+int default_chunk(bool bf16, int D, long long M) {
+  if (!bf16) return 4096;
+  int chunk = D <= 1024 ? 32768 : (D <= 2048 ? 16384 : 8192);
+  while (chunk > 8192 && M * chunk * 2 > (512LL << 20)) chunk /= 2;
+  return chunk;
+}
 
 pctc_status_t make_plan(const pctc_problem_t* p, const int32_t* Tn, const int32_t* Un, Plan* pl) {
   if (!p || !Tn || !Un) return PCTC_ERR_INVALID_ARG;
@@ -63,7 +71,7 @@ pctc_status_t make_plan(const pctc_problem_t* p, const int32_t* Tn, const int32_
   pl->elem = pl->bf16 ? 2 : 4;
   pl->use_umma = pl->bf16 && p->gemm_path == PCTC_GEMM_AUTO && (p->D % 8 == 0) && (p->V % 8 == 0);
   pl->beam = (p->beam > 0.f) && std::isfinite(p->beam);
-  int chunk = p->chunk > 0 ? p->chunk : default_chunk(pl->bf16);
+  int chunk = p->chunk > 0 ? p->chunk : default_chunk(pl->bf16, p->D, M);
   if (pl->use_umma) chunk = (chunk + 127) / 128 * 128;   // operand tiles of the tensor-core path
   if ((long long)chunk > p->V) chunk = (int)(pl->use_umma ? (p->V + 7) / 8 * 8 : p->V);
   pl->chunk = chunk;
@@ -196,6 +204,17 @@ pctc_status_t pctc_workspace_bytes(const pctc_problem_t* problem, const int32_t*
   pctc_status_t st = make_plan(problem, input_lengths_host, target_lengths_host, &pl);
   if (st != PCTC_OK) return st;
   *bytes_out = pl.total;
+  return PCTC_OK;
+}
+
+pctc_status_t pctc_chunk_width(const pctc_problem_t* problem, const int32_t* input_lengths_host,
+                               const int32_t* target_lengths_host, int32_t* chunk_out, int32_t* nchunks_out) {
+  if (!chunk_out) return PCTC_ERR_INVALID_ARG;
+  Plan pl;
+  pctc_status_t st = make_plan(problem, input_lengths_host, target_lengths_host, &pl);
+  if (st != PCTC_OK) return st;
+  *chunk_out = pl.chunk;
+  if (nchunks_out) *nchunks_out = pl.nchunks;
   return PCTC_OK;
 }
 

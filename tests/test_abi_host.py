@@ -58,6 +58,21 @@ def test_workspace_has_no_M_times_V_term(lib):
     assert lib.workspace_bytes(_prob(lib, beam=8.0), il, tl) > lib.workspace_bytes(_prob(lib), il, tl)
 
 
+@pytest.mark.parametrize("kw,il,want", [
+    (dict(dtype=1), [50, 40], (1000, 1)),                           # fp32: 4,096, capped by V
+    (dict(dtype=1, V=10000), [50, 40], (4096, 3)),
+    (dict(dtype=0, D=512, V=180000), [50, 40], (32768, 6)),         # narrow head: wide chunks
+    (dict(dtype=0, D=2048, V=180000), [50, 40], (16384, 11)),
+    (dict(dtype=0, D=4096, V=151936), [50, 40], (8192, 19)),
+    (dict(dtype=0, D=512, V=180000, N=2, T=16000), [16000, 1], (16384, 11)),   # [M, C] temporary <= 512 MiB
+    (dict(dtype=0, D=512, V=180000, N=2, T=64000), [64000, 1], (8192, 22)),
+    (dict(dtype=0, D=512, V=180000, chunk=1000), [50, 40], (1024, 176)),       # rounded up to the tile width
+    (dict(dtype=0, D=512, V=180000, chunk=1000, gemm_path=1), [50, 40], (1000, 180)),
+])
+def test_chunk_width_default_and_rounding(lib, kw, il, want):
+    assert lib.chunk_width(_prob(lib, **kw), il, [10, 3]) == want
+
+
 @pytest.mark.parametrize("kw,il,tl", [
     (dict(N=0), [50, 50], [3, 3]),
     (dict(V=0), [50, 50], [3, 3]),

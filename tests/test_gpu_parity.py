@@ -43,13 +43,13 @@ def test_fp32_with_bias_ragged_chunks_blank_nonzero(lib):
 
 
 @pytest.mark.parametrize("path", [SIMT, AUTO])
-@pytest.mark.parametrize("name,kw", [
-    ("c2", dict(V=8192, N=6, T_div=4)),                 # D=512, several row and column tiles
-    ("c3", dict(V=12288 + 384, D=256, N=4, T_div=4, U_div=2)),   # ragged last chunk, RMS-normalised frames
+@pytest.mark.parametrize("name,kw,chunk", [
+    ("c2", dict(V=8192, N=6, T_div=4), 0),              # D=512, several row and column tiles, default chunk
+    ("c3", dict(V=12288 + 384, D=256, N=4, T_div=4, U_div=2), 4096),   # ragged last chunk, RMS-normalised frames
 ])
-def test_bf16_reduced_configs(lib, path, name, kw):
+def test_bf16_reduced_configs(lib, path, name, kw, chunk):
     batch = wl.make_batch(small(name, **kw), permute_ids=True, poison_padding=True)
-    gpu = H.run_gpu(lib, batch, gemm_path=path)
+    gpu = H.run_gpu(lib, batch, gemm_path=path, chunk=chunk)
     ref = H.run_oracle(batch)
     H.assert_parity(gpu, ref, batch)
 

@@ -130,6 +130,12 @@ def reduce_over_ranks(ms: float, frames: float, flops: float, device=None):
     return float(t[0].item()), float(s[0].item()), float(s[1].item())
 
 
+def _traced_call(binding, hidden, W, targets, il, tl, batch, res, trace, call):
+    binding.pruned_ctc_fwd_bwd(hidden, W, None, targets, il, tl, batch.blank, workspace=res["workspace"], out=res,
+                               trace=trace, **call)
+    return trace
+
+
 def oracle_sample(batch, frames: int):
     """The first `frames` frames of utterance 0 with a proportional prefix of its labels."""
     n = 0
@@ -209,6 +215,10 @@ def main():
                          "would (default for the g* grid workloads)")
     ap.add_argument("--frozen-head", action="store_true",
                     help="skip dW (the LLM-CTC setting): 6 M D V FLOPs per step instead of 8")
+    ap.add_argument("--allreduce-dw", action="store_true",
+                    help="data-parallel training step: dW of every step is summed over the ranks, one NCCL "
+                         "all-reduce per vocabulary chunk on a communication stream (off by default: the "
+                         "head-and-loss path itself has no exchange step)")
     ap.add_argument("--e2e-steps", type=int, default=3)
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--cpu-frames", type=int, default=1024)
@@ -237,9 +247,13 @@ def main():
     # GPU when the multi-rank code path is exercised on a single-GPU machine
     backend = os.environ.get("PCTC_BENCH_BACKEND", "nccl")
     red_dev = dev if backend == "nccl" else None
-    if world > 1:
+    if world > 1 or args.allreduce_dw:
         import torch.distributed as dist
-        if backend == "nccl":
+        if world == 1:
+            os.environ.setdefault("MASTER_ADDR", "127.0.0.1")
+            os.environ.setdefault("MASTER_PORT", str(29400 + os.getpid() % 500))
+            dist.init_process_group("nccl", rank=0, world_size=1, device_id=dev)
+        elif backend == "nccl":
             dist.init_process_group("nccl", device_id=dev)
         else:
             dist.init_process_group(backend)
@@ -285,6 +299,15 @@ def main():
     torch.cuda.synchronize()
 
     traces = [binding.Trace(binding.Trace.capacity_for(V, chunk)) for _ in range(args.steps)]
+    sum_dW = args.allreduce_dw and not args.frozen_head
+    if sum_dW:
+        from paper_2609_33645_b200 import data_parallel as dp
+        comm = torch.cuda.Stream(dev)
+        dw_rows = dp.chunk_rows(V, chunk)
+        for _ in range(2):                       # NCCL sets up its channels at the first collective
+            dp.allreduce_rows(res["dW"], dw_rows, dp.dw_ready_events(
+                _traced_call(binding, hidden, W, targets, il, tl, batch, res, traces[0], dev_call)), comm_stream=comm)
+        torch.cuda.synchronize()
     sampler = ClockSampler(local_dev)
     if rank == 0:
         sampler.start()
@@ -297,6 +320,8 @@ def main():
     for s in range(args.steps):
         binding.pruned_ctc_fwd_bwd(hidden, W, None, targets, il, tl, batch.blank, workspace=res["workspace"],
                                    out=res, trace=traces[s], **dev_call)
+        if sum_dW:
+            dp.allreduce_rows(res["dW"], dw_rows, dp.dw_ready_events(traces[s]), comm_stream=comm)
     ev1.record()
     torch.cuda.synchronize()
     if world > 1:
@@ -402,7 +427,8 @@ def main():
         config=dict(workload=cfg.name, N=N, T_range=[cfg.T_lo, cfg.T_hi], D=D, V=V, M_frames=M,
                     K_selected=int(res["K"].item()), beam=args.beam, chunk=chunk, frozen_head=args.frozen_head, max_K=max_K,
                     l2="inputs larger than L2 (W and dW are %.2f GB each)" % (W.numel() * 2 / 1e9),
-                    parallelism="independent utterance batches per GPU, no collective"),
+                    parallelism=("utterance-sharded data parallel, dW all-reduced per vocabulary chunk (NCCL)"
+                                 if sum_dW else "independent utterance batches per GPU, no collective")),
         tflops=flops_all / (ms_per_step * 1e-3) / 1e12,
         frac_of_bf16_peak=dict(burst=flops_all / (ms_per_step * 1e-3) / 1e12 / (peaks["bf16_tflops"] * world),
                                sustained=flops_all / (ms_per_step * 1e-3) / 1e12 / (peak * world),
@@ -420,7 +446,7 @@ def main():
         e2e=e2e, gpu_launches=gpu_launches, clocks=clocks, cpu_baseline=cpu,
     )
     print(json.dumps(line), flush=True)
-    if world > 1:
+    if world > 1 or args.allreduce_dw:
         dist.destroy_process_group()
     return 0
 

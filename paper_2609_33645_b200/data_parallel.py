@@ -1,7 +1,7 @@
 """Utterance-sharded data parallelism for the Pruned-CTC head (one process per GPU).
 
 Every rank holds the full head W[V, D] (the head is replicated, not sharded:
-Appendix B.2) and a slice of the batch's utterances.  A rank builds the selected
+Appendix B.1) and a slice of the batch's utterances.  A rank builds the selected
 class set U of *its own* utterances: by Proposition 1 any superset of an
 utterance's labels gives that utterance's exact loss and gradient, so per-rank
 subsets change nothing.  Losses and dH stay local.  The one exchange step is the

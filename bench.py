@@ -365,8 +365,9 @@ def main():
     # profiles/umma_gemm_c4_speed_of_light.md (default workload and chunk only)
     traffic = None
     if args.config == "c4" and not args.vocab and chunk == 8192 and not args.frozen_head and args.beam == 0:
-        traffic = dict(bytes_per_step=51.1e9, launches_per_step=58, bytes_per_launch_avg=51.1e9 / 58,
-                       source="ncu dram__bytes.sum.per_second x duration, one launch of each kind, scaled by launches")
+        traffic = dict(bytes_per_step=38.3e9, launches_per_step=58, bytes_per_launch_avg=38.3e9 / 58,
+                       source="ncu dram__bytes_read.sum + dram__bytes_write.sum: the LSE launch and chunks 0-1 of each "
+                              "chunk kernel, chunk averages scaled by launches")
 
     # kernels launched by the library inside the timed region
     dp_launches = 4 if args.beam > 0 else 2      # sweeps (+ best-alignment sweeps, arc flags), occupancies

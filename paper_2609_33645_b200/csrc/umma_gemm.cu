@@ -35,8 +35,11 @@ namespace pctc {
 namespace {
 
 // Tunables (overridable at compile time for experiments)
-#ifndef PCTC_TUNE_N_FASTEST
-#define PCTC_TUNE_N_FASTEST 1     // dX / dW kernels walk column tiles first
+#ifndef PCTC_TUNE_RASTER_G
+#define PCTC_TUNE_RASTER_G 8      // row tiles per band of the tile order (kernels with one tile per unit)
+#endif
+#ifndef PCTC_TUNE_WALK_MB
+#define PCTC_TUNE_WALK_MB 32      // MB of A rows that a band of the column-walking kernels keeps hot in L2
 #endif
 
 #ifndef PCTC_TUNE_CTAS
@@ -67,7 +70,7 @@ struct UmmaArgs {
   int m, n, k;
   int a_mn, b_mn;
   int nsplit;          // EPI_LSE_PARTIAL: column splits per row tile
-  int n_fastest;       // tile order: consecutive CTAs walk the column tiles of one row tile first
+  int raster_g;        // tile order: row tiles per band (see decode_unit)
   int* status;
   Epilogue e;
 };
@@ -288,13 +291,20 @@ __device__ __forceinline__ void split_range(int n_tiles, int splits, int sp, int
   start = sp * base + min(sp, rem);
 }
 
-// Unit u -> (row tile, first column tile, number of column tiles).  The order decides which operand
-// streams through L2 once and which stays resident while a wave of CTAs runs: row tile fastest
-// keeps A (all row tiles) resident and streams B; column tile fastest does the opposite.
-__device__ __forceinline__ void decode_unit(int u, int m_tiles, int n_tiles, int splits, bool n_fastest,
+// Unit u -> (row tile, first column tile, number of column tiles).  The order decides what the
+// CTA groups that run at the same time have in common, i.e. what L2 serves more than once per DRAM
+// read.  Row tiles are taken in bands of g: inside a band the row tile runs fastest, then the
+// column split, so a wave of W groups covers g row tiles x W/g column splits and touches
+// g A-panels + W/g B-panels instead of all A-panels (g = m_tiles) or all B-panels (g = 1).
+// Odd bands walk the splits backwards, so a band starts on the B-panels the previous one ended on.
+__device__ __forceinline__ void decode_unit(int u, int m_tiles, int n_tiles, int splits, int g,
                                             int& mt, int& sp, int& nt0, int& cnt) {
-  if (n_fastest) { sp = u % splits; mt = u / splits; }
-  else { mt = u % m_tiles; sp = u / m_tiles; }
+  const int band_units = g * splits;
+  const int band = u / band_units, r = u - band * band_units;
+  const int rows = min(g, m_tiles - band * g);
+  sp = r / rows;
+  mt = band * g + (r - sp * rows);
+  if (band & 1) sp = splits - 1 - sp;
   split_range(n_tiles, splits, sp, nt0, cnt);
 }
 
@@ -368,7 +378,7 @@ k_umma_gemm(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
       };
       for (int u = group; u < units && ok; u += ngroups) {
         int mt, sp, nt0, cnt;
-        decode_unit(u, m_tiles, n_tiles, splits, a.n_fastest != 0, mt, sp, nt0, cnt);
+        decode_unit(u, m_tiles, n_tiles, splits, a.raster_g, mt, sp, nt0, cnt);
         const int row_a = mt * TILE_M + rank * BM;               // this CTA's rows of A
         for (int nt = nt0; nt < nt0 + cnt && ok; ++nt) {
           const int row_b = nt * BN + rank * (BN / CTAS);        // this CTA's columns of the tile (rows of B)
@@ -417,7 +427,7 @@ k_umma_gemm(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
       bool ok = true;
       for (int u = group; u < units && ok; u += ngroups) {
         int mt, sp, nt0, cnt;
-        decode_unit(u, m_tiles, n_tiles, splits, a.n_fastest != 0, mt, sp, nt0, cnt);
+        decode_unit(u, m_tiles, n_tiles, splits, a.raster_g, mt, sp, nt0, cnt);
         (void)mt;
         for (int nt = nt0; nt < nt0 + cnt && ok; ++nt, ++it) {
           const unsigned acc = it & 1u, aph = (it >> 1) & 1u;
@@ -465,7 +475,7 @@ k_umma_gemm(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
     bool ok = true;
     for (int u = group; u < units && ok; u += ngroups) {
       int mt, sp, nt0, cnt;
-      decode_unit(u, m_tiles, n_tiles, splits, a.n_fastest != 0, mt, sp, nt0, cnt);
+      decode_unit(u, m_tiles, n_tiles, splits, a.raster_g, mt, sp, nt0, cnt);
       const int row0_cta = mt * TILE_M + rank * BM;      // first row of this CTA's half of the tile
       const int i = row0_cta + r;
       const bool row_ok = i < a.m;
@@ -805,12 +815,21 @@ cudaError_t umma_gemm(const __nv_bfloat16* A, long long lda, bool a_mn_major,
   a.a_mn = a_mn_major ? 1 : 0;
   a.b_mn = b_mn_major ? 1 : 0;
   a.nsplit = e.nsplit;
-  // dX += dZ W and dW = dZ^T X read a large A (the dZ chunk) against a smaller B: keep B resident
-  a.n_fastest = (PCTC_TUNE_N_FASTEST && (e.kind == EPI_ACCUM_F32 || e.kind == EPI_STORE_OUT)) ? 1 : 0;
   a.status = status;
   a.e = e;
   const int m_tiles = (m + BM * CTAS_DEFAULT - 1) / (BM * CTAS_DEFAULT), n_tiles = (n + BN - 1) / BN;
   const bool walks = e.kind == EPI_LSE_PARTIAL || e.kind == EPI_ARGMAX_PARTIAL;
+  {
+    // a unit of the walking kernels re-reads its A rows for every column tile: the band's A rows must
+    // stay in L2 (and leave room for the streaming B); the other kernels read each panel once per
+    // unit, and a near-square patch of tiles per wave touches the fewest panels
+    long long g = PCTC_TUNE_RASTER_G;
+    if (walks) g = ((long long)PCTC_TUNE_WALK_MB << 20) / ((long long)BM * CTAS_DEFAULT * k * 2);
+    if (g < 1) g = 1;
+    if (g > m_tiles) g = m_tiles;
+    const int bands = (int)((m_tiles + g - 1) / g);
+    a.raster_g = (m_tiles + bands - 1) / bands;          // bands of equal height
+  }
   long long units = (long long)m_tiles * (walks ? e.nsplit : n_tiles);
   if (walks && (e.nsplit < 1 || e.nsplit > n_tiles)) return cudaErrorInvalidValue;
   const int groups = sm_count() / CTAS_DEFAULT;

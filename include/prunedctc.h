@@ -58,7 +58,7 @@ typedef struct {
   int32_t N;             /* utterances                                                        */
   int32_t T;             /* padded frames per utterance (row count of hidden[n])              */
   int32_t D;             /* head input width; bf16 tensor-core path needs D % 8 == 0          */
-  int64_t V;             /* classes, blank included; bf16 tensor-core path needs V % 8 == 0   */
+  int64_t V;             /* classes, blank included (any value >= 1)                          */
   int32_t dtype;         /* pctc_dtype_t of hidden, W, bias, dH, dW, dbias; loss is fp32      */
   int32_t blank_id;      /* in [0, V)                                                         */
   float   beam;          /* alignment beam in nats (Section 3.3); <= 0 or +inf: no pruning    */

@@ -69,7 +69,7 @@ pctc_status_t make_plan(const pctc_problem_t* p, const int32_t* Tn, const int32_
   if (pl->Lmax > dp_max_states()) return PCTC_ERR_UNSUPPORTED;
   pl->bf16 = (p->dtype == PCTC_BF16);
   pl->elem = pl->bf16 ? 2 : 4;
-  pl->use_umma = pl->bf16 && p->gemm_path == PCTC_GEMM_AUTO && (p->D % 8 == 0) && (p->V % 8 == 0);
+  pl->use_umma = pl->bf16 && p->gemm_path == PCTC_GEMM_AUTO && (p->D % 8 == 0);   // 16-byte rows for TMA
   pl->beam = (p->beam > 0.f) && std::isfinite(p->beam);
   int chunk = p->chunk > 0 ? p->chunk : default_chunk(pl->bf16, p->D, M);
   if (pl->use_umma) chunk = (chunk + 127) / 128 * 128;   // operand tiles of the tensor-core path

@@ -56,11 +56,19 @@ def test_bf16_reduced_configs(lib, path, name, kw, chunk):
 
 @pytest.mark.parametrize("path", [SIMT, AUTO])
 def test_bf16_bias_blank_nonzero_small_chunk(lib, path):
-    cfg = small("c2", V=5000 if path == SIMT else 5000 - 5000 % 8, D=192, N=5, T_div=6, U_div=3, blank=4097)
+    cfg = small("c2", V=5001, D=192, N=5, T_div=6, U_div=3, blank=4097)      # odd V: ragged last chunk of 905
     batch = wl.make_batch(cfg, with_bias=True, permute_ids=True, poison_padding=True)
     gpu = H.run_gpu(lib, batch, gemm_path=path, chunk=1024)
     ref = H.run_oracle(batch)
     H.assert_parity(gpu, ref, batch)
+
+
+@pytest.mark.parametrize("V", [1001, 257, 9])
+def test_bf16_odd_vocabulary_narrower_than_one_chunk(lib, V):
+    cfg = small("c2", V=V, D=64, N=4, T_div=10, U_div=8, zipf_s=None)
+    batch = wl.make_batch(cfg, with_bias=True)
+    gpu = H.run_gpu(lib, batch)
+    H.assert_parity(gpu, H.run_oracle(batch), batch)
 
 
 @pytest.mark.parametrize("path", [SIMT, AUTO])

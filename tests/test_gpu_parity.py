@@ -100,9 +100,11 @@ def test_single_frame_and_single_utterance(lib):
     H.assert_parity(gpu, ref, batch)
 
 
-@pytest.mark.parametrize("U,T", [(14, 40), (30, 90), (60, 150), (120, 300), (250, 520), (500, 1010), (1000, 2005)])
+@pytest.mark.parametrize("U,T", [(14, 40), (30, 90), (60, 150), (120, 300), (250, 520), (500, 1010), (1000, 2005),
+                                 (2047, 4100)])
 def test_every_trellis_width_of_the_dp(lib, U, T):
-    # one utterance per DP kernel configuration (32 ... 2048 positions), with adjacent repeats
+    # one utterance per DP kernel configuration (32 ... 4096 positions, the widest the library takes:
+    # 2 * 2047 + 1 = 4095), with adjacent repeats
     cfg = dataclasses.replace(wl.CONFIGS["c1"], name=f"dp{U}", N=2, T_lo=T - 3, T_hi=T, U_lo=U - 2, U_hi=U,
                               V=300, D=16, zipf_s=1.0, seed=U)
     batch = wl.make_batch(cfg)

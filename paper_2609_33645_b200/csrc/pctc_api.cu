@@ -13,10 +13,12 @@ namespace {
 using namespace pctc;
 
 constexpr size_t ALIGN = 256;
+constexpr size_t DH_SPLIT_EXTRA_BYTES = 128u << 20;   // most that extra dX accumulators may take
 inline size_t up(size_t x, size_t a = ALIGN) { return (x + a - 1) / a * a; }
 
 struct Plan {
   int N, T, D, M, Usum, Kcap, Lmax, chunk, nsplit, nchunks;
+  int ksplit, slab_rows;   // dX accumulator: k-split slabs of slab_rows rows each (1 slab of M rows without)
   long long V, cells, mcells;
   size_t ldS;
   int elem;          // bytes per element of hidden/W
@@ -114,7 +116,11 @@ pctc_status_t make_plan(const pctc_problem_t* p, const int32_t* Tn, const int32_
     pl->o_mcell0 = take((size_t)pl->N * 8);
   }
   pl->o_chunk = take((size_t)pl->M * pl->chunk * pl->elem);
-  pl->o_dHacc = take((size_t)pl->M * pl->D * 4);
+  // few output tiles (small M x D): the dX contraction of a chunk is cut along k into ksplit ranges, each
+  // with its own fp32 accumulator, summed in a fixed order when dH is written (deterministic)
+  pl->ksplit = pl->use_umma ? umma_accum_splits(pl->M, pl->D, pl->chunk, DH_SPLIT_EXTRA_BYTES) : 1;
+  pl->slab_rows = pl->ksplit > 1 ? umma_accum_slab_rows(pl->M) : pl->M;
+  pl->o_dHacc = take((size_t)pl->ksplit * pl->slab_rows * pl->D * 4);
   pl->total = o;
   return PCTC_OK;
 }
@@ -462,6 +468,7 @@ pctc_status_t run_call(const pctc_problem_t* p, const void* hidden, const void* 
   if (!p->forward_only) PCTC_CUDA(zero_nonfinite_rows(d_X, M, D, pl.elem, bm.row_utt, d_flags, stream));
 
   // ---- lines 11-17: backward, one vocabulary chunk at a time ----
+  int dh_slabs = 1;                  // dX accumulator slabs in use (k-split of the dX contraction)
   for (int ci = 0; ci < pl.nchunks && !p->forward_only; ++ci) {
     const long long v0 = (long long)ci * pl.chunk;
     const int Cc = (int)((V - v0 < pl.chunk) ? (V - v0) : pl.chunk);
@@ -490,6 +497,15 @@ pctc_status_t run_call(const pctc_problem_t* p, const void* hidden, const void* 
       e.out = d_dHacc;
       e.ld = D;
       e.accumulate = ci > 0;
+      if (pl.ksplit > 1) {
+        // the first chunk stores into (and so initialises) its slabs; a shorter chunk later on may
+        // cut k into fewer ranges and then adds to the first slabs only
+        int s = umma_accum_splits(M, D, Cc, DH_SPLIT_EXTRA_BYTES);
+        if (s > pl.ksplit) s = pl.ksplit;
+        if (ci == 0) dh_slabs = s;
+        e.ksplit = s < dh_slabs ? s : dh_slabs;
+        e.ksplit_rows = pl.slab_rows;
+      }
       GemmCall c{d_chunk, pl.chunk, false, Wc, D, true, M, D, Cc};
       PCTC_CUDA(run_gemm(pl.use_umma, pl.bf16, c, e, d_status, stream));
     }
@@ -521,7 +537,7 @@ pctc_status_t run_call(const pctc_problem_t* p, const void* hidden, const void* 
     PCTC_CUDA(cudaStreamWaitEvent(stream, aux.copies_done, 0));
   }
   PCTC_MARK(PCTC_PHASE_FINISH);
-  if (!p->forward_only) PCTC_CUDA(unstack_cast(d_dHacc, dH, N, pl.T, D, pl.bf16, bm.T_n, bm.row0, stream));
+  if (!p->forward_only) PCTC_CUDA(unstack_cast(d_dHacc, dh_slabs, (size_t)pl.slab_rows * D, dH, N, pl.T, D, pl.bf16, bm.T_n, bm.row0, stream));
 
   // ---- optional integer outputs ----
   if (subset_out)

@@ -42,6 +42,8 @@ struct Epilogue {
   int partial_offset = 0;       // segment of B writes its splits at partial_offset .. +nsplit-1
   int accumulate = 0;           // EPI_ACCUM_F32 / EPI_STORE_OUT: add to the destination instead of overwriting
   int out_is_bf16 = 0;          // EPI_DLOGITS / EPI_STORE_OUT destination type
+  int ksplit = 1;               // EPI_ACCUM_F32 on the tensor-core path: the contraction is cut into this many
+  int ksplit_rows = 0;          //   ranges of k; range s accumulates into rows [s * ksplit_rows, ...) of `out`
 };
 
 struct GemmShape {
@@ -62,6 +64,11 @@ cudaError_t umma_gemm(const __nv_bfloat16* A, long long lda, bool a_mn_major,
                       int m, int n, int k, const Epilogue& e, int* status, cudaStream_t stream);
 bool umma_available();   // the driver entry point for tensor maps could be resolved
 int umma_lse_splits(int m, int n);   // column splits (<= 32) for EPI_LSE_PARTIAL on this device
+// EPI_ACCUM_F32 with few output tiles (small m x n): how many k-ranges per tile fill the device, given
+// that every range beyond the first costs another [slab_rows, n] fp32 accumulator (at most max_extra_bytes
+// in total); and the slab height (m rounded up to whole row tiles) that goes with it.
+int umma_accum_splits(int m, int n, int k, size_t max_extra_bytes);
+int umma_accum_slab_rows(int m);
 int umma_lse_partials_per_split(int k);   // the kernel writes this many partials per split (1 or 2):
                                           // partial[(i*nsplit + sp)*pps + h]
 
@@ -102,9 +109,10 @@ cudaError_t stack_frames(const void* hidden, void* X, int N, int T, int D, int e
 cudaError_t zero_nonfinite_rows(void* X, int M, int D, int elem_bytes, const int* row_utt, const int* utt_flags,
                                 cudaStream_t stream);
 
-// dH[n,t,:] = T(acc[row0[n]+t,:]) for t < T_n, zero for padded frames.
-cudaError_t unstack_cast(const float* acc, void* dH, int N, int T, int D, bool out_bf16,
-                         const int* T_n, const int* row0, cudaStream_t stream);
+// dH[n,t,:] = T(sum over slabs s < nslab, in ascending s, of acc[s*slab_stride + (row0[n]+t)*D + :]) for
+// t < T_n, zero for padded frames.
+cudaError_t unstack_cast(const float* acc, int nslab, size_t slab_stride, void* dH, int N, int T, int D,
+                         bool out_bf16, const int* T_n, const int* row0, cudaStream_t stream);
 
 // W_U[j,:] = W[U[j],:] for j < K (rows K.. of the [Kcap, D] buffer are zeroed).
 cudaError_t gather_rows(const void* W, void* W_U, const int* U, const int* Kdev, int Kcap, int D,

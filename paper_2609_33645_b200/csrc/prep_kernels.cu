@@ -116,8 +116,8 @@ __global__ void k_stack_frames(const char* __restrict__ hidden, char* __restrict
 }
 
 template <typename TOut>
-__global__ void k_unstack_cast(const float* __restrict__ acc, TOut* __restrict__ dH, int T, int D,
-                               const int* __restrict__ T_n, const int* __restrict__ row0) {
+__global__ void k_unstack_cast(const float* __restrict__ acc, int nslab, size_t slab_stride, TOut* __restrict__ dH,
+                               int T, int D, const int* __restrict__ T_n, const int* __restrict__ row0) {
   const int n = blockIdx.x / T, t = blockIdx.x - n * T;
   TOut* dst = dH + ((size_t)n * T + t) * D;
   if (t >= T_n[n]) {
@@ -125,7 +125,11 @@ __global__ void k_unstack_cast(const float* __restrict__ acc, TOut* __restrict__
     return;
   }
   const float* src = acc + ((size_t)row0[n] + t) * D;
-  for (int d = threadIdx.x; d < D; d += blockDim.x) dst[d] = TOut(src[d]);
+  for (int d = threadIdx.x; d < D; d += blockDim.x) {
+    float v = src[d];
+    for (int s = 1; s < nslab; ++s) v += src[s * slab_stride + d];     // k-split partial sums, fixed order
+    dst[d] = TOut(v);
+  }
 }
 
 __global__ void k_gather_rows(const char* __restrict__ W, char* __restrict__ W_U, const int* __restrict__ U,
@@ -262,12 +266,12 @@ cudaError_t zero_nonfinite_rows(void* X, int M, int D, int elem_bytes, const int
   return cudaGetLastError();
 }
 
-cudaError_t unstack_cast(const float* acc, void* dH, int N, int T, int D, bool out_bf16,
-                         const int* T_n, const int* row0, cudaStream_t stream) {
+cudaError_t unstack_cast(const float* acc, int nslab, size_t slab_stride, void* dH, int N, int T, int D,
+                         bool out_bf16, const int* T_n, const int* row0, cudaStream_t stream) {
   if (out_bf16)
-    k_unstack_cast<__nv_bfloat16><<<N * T, 128, 0, stream>>>(acc, (__nv_bfloat16*)dH, T, D, T_n, row0);
+    k_unstack_cast<__nv_bfloat16><<<N * T, 128, 0, stream>>>(acc, nslab, slab_stride, (__nv_bfloat16*)dH, T, D, T_n, row0);
   else
-    k_unstack_cast<float><<<N * T, 128, 0, stream>>>(acc, (float*)dH, T, D, T_n, row0);
+    k_unstack_cast<float><<<N * T, 128, 0, stream>>>(acc, nslab, slab_stride, (float*)dH, T, D, T_n, row0);
   return cudaGetLastError();
 }
 

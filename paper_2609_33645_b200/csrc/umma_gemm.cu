@@ -71,6 +71,8 @@ struct UmmaArgs {
   int a_mn, b_mn;
   int nsplit;          // EPI_LSE_PARTIAL: column splits per row tile
   int raster_g;        // tile order: row tiles per band (see decode_unit)
+  int ksplit;          // EPI_ACCUM_F32: units per output tile, each contracting its own range of k
+  int ksplit_rows;     //   ... and writing its own accumulator slab, this many rows further down
   int* status;
   Epilogue e;
 };
@@ -265,6 +267,26 @@ __device__ __forceinline__ void tmem_ld32(unsigned taddr, float* v) {
 #pragma unroll
   for (int i = 0; i < 32; ++i) v[i] = __uint_as_float(r[i]);
 }
+// Two fp32 FMAs in one instruction (sm_100 packed fp32): d = a * b + c on both halves.
+__device__ __forceinline__ void ffma2(float& d0, float& d1, float a0, float a1, float b0, float b1, float c0, float c1) {
+  asm("{\n\t.reg .b64 ra, rb, rc, rd;\n\t"
+      "mov.b64 ra, {%2, %3};\n\tmov.b64 rb, {%4, %5};\n\tmov.b64 rc, {%6, %7};\n\t"
+      "fma.rn.f32x2 rd, ra, rb, rc;\n\tmov.b64 {%0, %1}, rd;\n\t}"
+      : "=f"(d0), "=f"(d1)
+      : "f"(a0), "f"(a1), "f"(b0), "f"(b1), "f"(c0), "f"(c1));
+}
+__device__ __forceinline__ void fmul2(float& d0, float& d1, float a0, float a1, float b0, float b1) {
+  asm("{\n\t.reg .b64 ra, rb, rd;\n\t"
+      "mov.b64 ra, {%2, %3};\n\tmov.b64 rb, {%4, %5};\n\t"
+      "mul.rn.f32x2 rd, ra, rb;\n\tmov.b64 {%0, %1}, rd;\n\t}"
+      : "=f"(d0), "=f"(d1)
+      : "f"(a0), "f"(a1), "f"(b0), "f"(b1));
+}
+__device__ __forceinline__ float lg2(float x) {
+  float y;
+  asm("lg2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+  return y;
+}
 __device__ __forceinline__ float ex2(float x) {
   float y;
   asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
@@ -297,14 +319,17 @@ __device__ __forceinline__ void split_range(int n_tiles, int splits, int sp, int
 // column split, so a wave of W groups covers g row tiles x W/g column splits and touches
 // g A-panels + W/g B-panels instead of all A-panels (g = m_tiles) or all B-panels (g = 1).
 // Odd bands walk the splits backwards, so a band starts on the B-panels the previous one ended on.
-__device__ __forceinline__ void decode_unit(int u, int m_tiles, int n_tiles, int splits, int g,
-                                            int& mt, int& sp, int& nt0, int& cnt) {
-  const int band_units = g * splits;
+__device__ __forceinline__ void decode_unit(int u, int m_tiles, int n_tiles, int splits, int ksplit, int g,
+                                            int& mt, int& sp, int& ks, int& nt0, int& cnt) {
+  const int cols = splits * ksplit;              // a column split may itself be cut along k
+  const int band_units = g * cols;
   const int band = u / band_units, r = u - band * band_units;
   const int rows = min(g, m_tiles - band * g);
-  sp = r / rows;
-  mt = band * g + (r - sp * rows);
-  if (band & 1) sp = splits - 1 - sp;
+  int c = r / rows;
+  mt = band * g + (r - c * rows);
+  if (band & 1) c = cols - 1 - c;
+  sp = c / ksplit;
+  ks = c - sp * ksplit;
   split_range(n_tiles, splits, sp, nt0, cnt);
 }
 
@@ -336,7 +361,8 @@ k_umma_gemm(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
   const int m_tiles = (a.m + TILE_M - 1) / TILE_M;
   const int n_tiles = (n_eff + BN - 1) / BN;
   const int splits = epi_walks_splits(EPI) ? a.nsplit : n_tiles;
-  const int units = m_tiles * splits;
+  const int ksplit = (EPI == EPI_ACCUM_F32) ? a.ksplit : 1;
+  const int units = m_tiles * splits * ksplit;
   const int k_blocks = (a.k + BK - 1) / BK;
 
   if (threadIdx.x == 0) {
@@ -377,12 +403,13 @@ k_umma_gemm(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
         else tma_load_2d(dst, map, c0, c1, bar);
       };
       for (int u = group; u < units && ok; u += ngroups) {
-        int mt, sp, nt0, cnt;
-        decode_unit(u, m_tiles, n_tiles, splits, a.raster_g, mt, sp, nt0, cnt);
+        int mt, sp, ks, nt0, cnt, kb0, kcnt;
+        decode_unit(u, m_tiles, n_tiles, splits, ksplit, a.raster_g, mt, sp, ks, nt0, cnt);
+        split_range(k_blocks, ksplit, ks, kb0, kcnt);            // this unit's share of the contraction
         const int row_a = mt * TILE_M + rank * BM;               // this CTA's rows of A
         for (int nt = nt0; nt < nt0 + cnt && ok; ++nt) {
           const int row_b = nt * BN + rank * (BN / CTAS);        // this CTA's columns of the tile (rows of B)
-          for (int kb = 0; kb < k_blocks; ++kb, ++g) {
+          for (int kb = kb0; kb < kb0 + kcnt; ++kb, ++g) {
             const int s = g % STAGES;
             const unsigned ph = (g / STAGES) & 1u;
             if (!mbar_wait(&st->empty[s], ph ^ 1u, abort_flag, a.status, 1)) { ok = false; break; }
@@ -426,15 +453,16 @@ k_umma_gemm(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
       unsigned g = 0, it = 0;
       bool ok = true;
       for (int u = group; u < units && ok; u += ngroups) {
-        int mt, sp, nt0, cnt;
-        decode_unit(u, m_tiles, n_tiles, splits, a.raster_g, mt, sp, nt0, cnt);
+        int mt, sp, ks, nt0, cnt, kb0, kcnt;
+        decode_unit(u, m_tiles, n_tiles, splits, ksplit, a.raster_g, mt, sp, ks, nt0, cnt);
+        split_range(k_blocks, ksplit, ks, kb0, kcnt);
         (void)mt;
         for (int nt = nt0; nt < nt0 + cnt && ok; ++nt, ++it) {
           const unsigned acc = it & 1u, aph = (it >> 1) & 1u;
           if (!mbar_wait(&st->tmem_empty[acc], aph ^ 1u, abort_flag, a.status, 2)) { ok = false; break; }
           tc_fence_after();
           const unsigned d_tmem = tmem_base + acc * BN;
-          for (int kb = 0; kb < k_blocks; ++kb, ++g) {
+          for (int kb = kb0; kb < kb0 + kcnt; ++kb, ++g) {
             const int s = g % STAGES;
             const unsigned ph = (g / STAGES) & 1u;
             if (!mbar_wait(&st->full[s], ph, abort_flag, a.status, 3)) { ok = false; break; }
@@ -445,8 +473,8 @@ k_umma_gemm(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
             for (int kk = 0; kk < BK / 16; ++kk) {
               const unsigned long long ad = adesc + (unsigned long long)(kk * a_step);
               const unsigned long long bd = bdesc + (unsigned long long)(kk * b_step);
-              if (CTAS == 2) tc_mma_bf16_pair(d_tmem, ad, bd, idesc, (kb | kk) != 0 ? 1u : 0u);
-              else tc_mma_bf16(d_tmem, ad, bd, idesc, (kb | kk) != 0 ? 1u : 0u);
+              if (CTAS == 2) tc_mma_bf16_pair(d_tmem, ad, bd, idesc, (kb != kb0 || kk != 0) ? 1u : 0u);
+              else tc_mma_bf16(d_tmem, ad, bd, idesc, (kb != kb0 || kk != 0) ? 1u : 0u);
             }
             // frees the stage (in both CTAs) once these MMAs have read it
             if (CTAS == 2) tc_commit_pair(&st->empty[s]); else tc_commit(&st->empty[s]);
@@ -473,15 +501,43 @@ k_umma_gemm(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
     const int pstride = a.e.partial_stride ? a.e.partial_stride : a.nsplit;   // split slots per row
     unsigned it = 0;
     bool ok = true;
+    // EPI_DLOGITS: the per-row and per-column inputs of a tile (lambda, row weight, class map) are
+    // fetched one unit ahead, so their latency is spent under the previous tile's epilogue
+    constexpr int NGRP = WARP_COLS / 32;
+    float pre_lam = 0.f, pre_w = 0.f;
+    int pre_jj[NGRP];
+    auto prefetch = [&](int u2) {
+      int mt2, sp2, ks2, nt2, cnt2;
+      decode_unit(u2, m_tiles, n_tiles, splits, ksplit, a.raster_g, mt2, sp2, ks2, nt2, cnt2);
+      const int i2 = mt2 * TILE_M + rank * BM + r;
+      pre_lam = 0.f; pre_w = 0.f;
+      if (i2 < a.m) { pre_lam = a.e.lambda[i2]; pre_w = a.e.roww[i2]; }
+#pragma unroll
+      for (int gq = 0; gq < NGRP; ++gq) {
+        const int j = nt2 * BN + c_base + gq * 32 + lane;
+        pre_jj[gq] = (j < n_eff) ? a.e.vmap[a.e.v0 + j] : -1;
+      }
+    };
+    if (EPI == EPI_DLOGITS && group < units) prefetch(group);
     for (int u = group; u < units && ok; u += ngroups) {
-      int mt, sp, nt0, cnt;
-      decode_unit(u, m_tiles, n_tiles, splits, a.raster_g, mt, sp, nt0, cnt);
+      int mt, sp, ks, nt0, cnt;
+      decode_unit(u, m_tiles, n_tiles, splits, ksplit, a.raster_g, mt, sp, ks, nt0, cnt);
       const int row0_cta = mt * TILE_M + rank * BM;      // first row of this CTA's half of the tile
+      const int row0_out = row0_cta + ks * a.ksplit_rows; // ... and where it lands in the output (k-split slab)
       const int i = row0_cta + r;
       const bool row_ok = i < a.m;
       float lam2 = 0.f, lam = 0.f, w = 0.f;
-      if ((EPI == EPI_DLOGITS || (EPI == EPI_SUBSET_LOGP && a.e.lambda)) && row_ok) { lam = a.e.lambda[i]; lam2 = lam * LOG2E; }
-      if (EPI == EPI_DLOGITS && row_ok) w = a.e.roww[i];
+      if (EPI == EPI_SUBSET_LOGP && a.e.lambda && row_ok) lam = a.e.lambda[i];
+      int cur_jj[NGRP];
+      if (EPI == EPI_DLOGITS) {
+        lam = pre_lam; w = pre_w; lam2 = lam * LOG2E;
+#pragma unroll
+        for (int gq = 0; gq < NGRP; ++gq) cur_jj[gq] = pre_jj[gq];
+        if (u + ngroups < units) prefetch(u + ngroups);
+      }
+      // a positive row weight goes into the exponent; any other (zero, negative) is multiplied in afterwards
+      const float wmul = (w > 0.f) ? 1.f : w;
+      const float off2 = (w > 0.f) ? lg2(w) - lam2 : -lam2;
       float run_max2 = -CUDART_INF_F, run_sum = 0.f;     // EPI_LSE_PARTIAL, base-2 domain
       float best_z = -CUDART_INF_F;                      // EPI_ARGMAX_PARTIAL
       int best_j = -1;
@@ -504,14 +560,13 @@ k_umma_gemm(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
             sb[c] = b;
           }
         }
-        if (EPI == EPI_DLOGITS) {
+        if (EPI == EPI_DLOGITS) {                       // one tile per unit: the prefetched class map is this tile's
 #pragma unroll
-          for (int c0 = 0; c0 < WARP_COLS; c0 += 32) {
-            const int j = n0 + c_base + c0 + lane;
-            const int jj = (j < n_eff) ? a.e.vmap[a.e.v0 + j] : -1;
+          for (int gq = 0; gq < NGRP; ++gq) {
+            const int jj = cur_jj[gq];
             const unsigned mask = __ballot_sync(0xffffffffu, jj >= 0);
-            sj[c0 + lane] = jj;
-            if (lane == 0) sg[c0 >> 5] = mask;
+            sj[gq * 32 + lane] = jj;
+            if (lane == 0) sg[gq] = mask;
           }
         }
         __syncwarp();
@@ -544,11 +599,17 @@ k_umma_gemm(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
 #pragma unroll
                 for (int c = 0; c < 32; ++c) v[c] += sb[g0 + c];
               }
+              // w p = exp2(z log2(e) + off2), off2 = log2(w) - lambda log2(e): one packed FMA per two logits
 #pragma unroll
-              for (int c = 0; c < 32; ++c) v[c] = ex2(fmaf(v[c], LOG2E, -lam2));     // p = exp(z - lambda)
+              for (int c = 0; c < 32; c += 2) {
+                float x0, x1;
+                ffma2(x0, x1, v[c], v[c + 1], LOG2E, LOG2E, off2, off2);
+                v[c] = ex2(x0);
+                v[c + 1] = ex2(x1);
+              }
               if (sg[cg] != 0u) {
-                // the group holds selected classes: subtract their occupancy in fp32, before the
-                // rounding to bf16; the loads are issued together, the unselected ones predicated off
+                // the group holds selected classes: subtract their weighted occupancy in fp32, before
+                // the rounding to bf16; the loads are issued together, the unselected ones predicated off
                 float g[32];
 #pragma unroll
                 for (int c = 0; c < 32; ++c) {
@@ -556,14 +617,16 @@ k_umma_gemm(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
                   g[c] = (jj >= 0 && row_ok) ? a.e.gamma[(long long)i * a.e.ld_gamma + jj] : 0.f;
                 }
 #pragma unroll
-                for (int c = 0; c < 32; ++c) v[c] = w * (v[c] - g[c]);
-              } else {
+                for (int c = 0; c < 32; ++c) v[c] = fmaf(-w, g[c], wmul * v[c]);
+              } else if (__any_sync(0xffffffffu, wmul != 1.f)) {      // rows whose weight is not in the exponent
 #pragma unroll
-                for (int c = 0; c < 32; ++c) v[c] *= w;
+                for (int c = 0; c < 32; ++c) v[c] *= wmul;
               }
-              if (w == 0.f) {                          // excluded utterance: exact zeros, whatever its logits are
+              if (__any_sync(0xffffffffu, w == 0.f)) {
+                if (w == 0.f) {                        // excluded utterance: exact zeros, whatever its logits are
 #pragma unroll
-                for (int c = 0; c < 32; ++c) v[c] = 0.f;
+                  for (int c = 0; c < 32; ++c) v[c] = 0.f;
+                }
               }
             }
             constexpr int NBOX = epi_fp32_boxes(EPI) ? 2 : 1;        // boxes per group
@@ -595,8 +658,8 @@ k_umma_gemm(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
               __syncwarp();
               if (lane == 0) {
                 if ((EPI == EPI_ACCUM_F32 || EPI == EPI_STORE_OUT) && a.e.accumulate)
-                  tma_reduce_add_2d(&tmC, box, j0 + b * 16, row0_cta + q * 32);
-                else tma_store_2d(&tmC, box, j0 + b * 16, row0_cta + q * 32);
+                  tma_reduce_add_2d(&tmC, box, j0 + b * 16, row0_out + q * 32);
+                else tma_store_2d(&tmC, box, j0 + b * 16, row0_out + q * 32);
                 bulk_commit();
               }
               ++nbox;
@@ -624,21 +687,45 @@ k_umma_gemm(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
               if (j0 + c < n_eff && z > best_z) { best_z = z; best_j = j0 + c; }   // ascending columns: first maximum wins
             }
           } else if (EPI == EPI_LSE_PARTIAL) {
-            float gmax = -CUDART_INF_F;
+            // running (max, sum of exp) in the base-2 domain: x = z * log2(e)
+            if (!has_bias && j0 + 32 <= n_eff) {
+              // whole group inside the matrix, no bias: max over the raw logits, then one packed FMA per
+              // two logits forms x - max and feeds the exponentials
+              float gm = v[0];
 #pragma unroll
-            for (int c = 0; c < 32; ++c) {
-              v[c] = (j0 + c < n_eff) ? (has_bias ? v[c] + sb[cg * 32 + c] : v[c]) * LOG2E : -CUDART_INF_F;
-              gmax = fmaxf(gmax, v[c]);
-            }
-            if (gmax > run_max2) {
-              run_sum *= ex2(run_max2 - gmax);     // ex2(-inf) = 0 on the first group
-              run_max2 = gmax;
-            }
-            float s = 0.f;
+              for (int c = 1; c < 32; ++c) gm = fmaxf(gm, v[c]);
+              const float gmax = gm * LOG2E;
+              if (gmax > run_max2) {
+                run_sum *= ex2(run_max2 - gmax);     // ex2(-inf) = 0 on the first group
+                run_max2 = gmax;
+              }
+              const float nm = -run_max2;
+              float s0 = 0.f, s1 = 0.f;
 #pragma unroll
-            for (int c = 0; c < 32; ++c) s += ex2(v[c] - run_max2);
-            run_sum += s;
-            if (gmax != gmax) run_sum = gmax;      // NaN logits poison the normaliser
+              for (int c = 0; c < 32; c += 2) {
+                float x0, x1;
+                ffma2(x0, x1, v[c], v[c + 1], LOG2E, LOG2E, nm, nm);
+                s0 += ex2(x0);
+                s1 += ex2(x1);
+              }
+              run_sum += s0 + s1;                    // a NaN logit makes the sum NaN
+            } else {
+              float gmax = -CUDART_INF_F;
+#pragma unroll
+              for (int c = 0; c < 32; ++c) {
+                v[c] = (j0 + c < n_eff) ? (has_bias ? v[c] + sb[cg * 32 + c] : v[c]) * LOG2E : -CUDART_INF_F;
+                gmax = fmaxf(gmax, v[c]);
+              }
+              if (gmax > run_max2) {
+                run_sum *= ex2(run_max2 - gmax);
+                run_max2 = gmax;
+              }
+              float s = 0.f;
+#pragma unroll
+              for (int c = 0; c < 32; ++c) s += ex2(v[c] - run_max2);
+              run_sum += s;
+              if (gmax != gmax) run_sum = gmax;      // NaN logits poison the normaliser
+            }
           }
         }
 
@@ -788,6 +875,31 @@ int umma_lse_splits(int m, int n) {
   return best;
 }
 
+int umma_accum_slab_rows(int m) {
+  const int tile_m = BM * CTAS_DEFAULT;
+  return (m + tile_m - 1) / tile_m * tile_m;
+}
+
+int umma_accum_splits(int m, int n, int k, size_t max_extra_bytes) {
+  const int groups = 148 / CTAS_DEFAULT;            // planned for a full B200, without asking the device: the
+                                                    // workspace size must not depend on where it is computed
+  const long long tiles = (long long)(umma_accum_slab_rows(m) / (BM * CTAS_DEFAULT)) * ((n + BN - 1) / BN);
+  const int k_blocks = (k + BK - 1) / BK;
+  if (tiles >= 4LL * groups) return 1;              // enough tiles: the last wave is a small share
+  const size_t slab = (size_t)umma_accum_slab_rows(m) * n * 4;
+  int best = 1;
+  double best_cost = 1e30;
+  for (int s = 1; s <= 16; ++s) {
+    if (s > 1 && ((size_t)(s - 1) * slab > max_extra_bytes || k_blocks / s < 16)) break;
+    const long long waves = (tiles * s + groups - 1) / groups;
+    // k-blocks on the busiest CTA group; a unit costs about 12 k-blocks on top of its own (pipeline
+    // refill, accumulator hand-over)
+    const double cost = (double)waves * ((double)k_blocks / s + 12.0);
+    if (cost < best_cost * 0.97) { best_cost = cost; best = s; }       // split only for a clear gain
+  }
+  return best;
+}
+
 cudaError_t umma_gemm(const __nv_bfloat16* A, long long lda, bool a_mn_major,
                       const __nv_bfloat16* B, long long ldb, bool b_mn_major,
                       int m, int n, int k, const Epilogue& e, int* status, cudaStream_t stream) {
@@ -797,9 +909,12 @@ cudaError_t umma_gemm(const __nv_bfloat16* A, long long lda, bool a_mn_major,
   bool ok = true;
   tmC = CUtensorMap{};
   // output boxes of the staged epilogues: 32 rows x 32 columns, clipped to the [m, n] extent
+  const int ksplit = (e.kind == EPI_ACCUM_F32 && e.ksplit > 1) ? e.ksplit : 1;
+  if (ksplit > 1 && (ksplit > (k + BK - 1) / BK || e.ksplit_rows < umma_accum_slab_rows(m))) return cudaErrorInvalidValue;
   if (e.kind == EPI_ACCUM_F32 || e.kind == EPI_SUBSET_LOGP) {
     if ((e.ld % 4) || ((size_t)e.out & 15)) return cudaErrorInvalidValue;
-    ok = ok && make_map(&tmC, e.out, (unsigned long long)n, (unsigned long long)m, (unsigned long long)e.ld, 16, 32, true);
+    const unsigned long long out_rows = (unsigned long long)(ksplit - 1) * e.ksplit_rows + m;   // k-split slabs stacked
+    ok = ok && make_map(&tmC, e.out, (unsigned long long)n, out_rows, (unsigned long long)e.ld, 16, 32, true);
   } else if (e.kind == EPI_DLOGITS || e.kind == EPI_STORE_OUT) {
     if ((e.ld % 8) || ((size_t)e.out & 15)) return cudaErrorInvalidValue;
     ok = ok && make_map(&tmC, e.out, (unsigned long long)n, (unsigned long long)m, (unsigned long long)e.ld, 32, 32);
@@ -815,6 +930,8 @@ cudaError_t umma_gemm(const __nv_bfloat16* A, long long lda, bool a_mn_major,
   a.a_mn = a_mn_major ? 1 : 0;
   a.b_mn = b_mn_major ? 1 : 0;
   a.nsplit = e.nsplit;
+  a.ksplit = ksplit;
+  a.ksplit_rows = ksplit > 1 ? e.ksplit_rows : 0;
   a.status = status;
   a.e = e;
   const int m_tiles = (m + BM * CTAS_DEFAULT - 1) / (BM * CTAS_DEFAULT), n_tiles = (n + BN - 1) / BN;
@@ -830,7 +947,7 @@ cudaError_t umma_gemm(const __nv_bfloat16* A, long long lda, bool a_mn_major,
     const int bands = (int)((m_tiles + g - 1) / g);
     a.raster_g = (m_tiles + bands - 1) / bands;          // bands of equal height
   }
-  long long units = (long long)m_tiles * (walks ? e.nsplit : n_tiles);
+  long long units = (long long)m_tiles * (walks ? e.nsplit : n_tiles) * ksplit;
   if (walks && (e.nsplit < 1 || e.nsplit > n_tiles)) return cudaErrorInvalidValue;
   const int groups = sm_count() / CTAS_DEFAULT;
   const int grid = (int)(units < groups ? units : groups) * CTAS_DEFAULT;

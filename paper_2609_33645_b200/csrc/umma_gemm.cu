@@ -307,8 +307,20 @@ __device__ __forceinline__ unsigned long long make_smem_desc(unsigned addr, bool
   return d;
 }
 
+// x / d for 0 <= x < 2^22, 1 <= d: a float quotient and one correction step instead of the long
+// integer-division sequence (the tile decode runs in every warp for every tile).
+__device__ __forceinline__ int fast_div(int x, int d, int& rem) {
+  int q = __float2int_rz(__fdividef((float)x, (float)d));
+  int r = x - q * d;
+  if (r < 0) { --q; r += d; }
+  else if (r >= d) { ++q; r -= d; }
+  rem = r;
+  return q;
+}
+
 __device__ __forceinline__ void split_range(int n_tiles, int splits, int sp, int& start, int& cnt) {
-  const int base = n_tiles / splits, rem = n_tiles % splits;
+  int rem;
+  const int base = fast_div(n_tiles, splits, rem);
   cnt = base + (sp < rem ? 1 : 0);
   start = sp * base + min(sp, rem);
 }
@@ -322,15 +334,16 @@ __device__ __forceinline__ void split_range(int n_tiles, int splits, int sp, int
 __device__ __forceinline__ void decode_unit(int u, int m_tiles, int n_tiles, int splits, int ksplit, int g,
                                             int& mt, int& sp, int& ks, int& nt0, int& cnt) {
   const int cols = splits * ksplit;              // a column split may itself be cut along k
-  const int band_units = g * cols;
-  const int band = u / band_units, r = u - band * band_units;
+  int r, row;
+  const int band = fast_div(u, g * cols, r);
   const int rows = min(g, m_tiles - band * g);
-  int c = r / rows;
-  mt = band * g + (r - c * rows);
+  int c = fast_div(r, rows, row);
+  mt = band * g + row;
   if (band & 1) c = cols - 1 - c;
-  sp = c / ksplit;
-  ks = c - sp * ksplit;
-  split_range(n_tiles, splits, sp, nt0, cnt);
+  if (ksplit == 1) { sp = c; ks = 0; }
+  else sp = fast_div(c, ksplit, ks);
+  if (splits == n_tiles) { nt0 = sp; cnt = 1; }  // one tile per unit
+  else split_range(n_tiles, splits, sp, nt0, cnt);
 }
 
 // ---------------------------------------------------------------------------------------------

@@ -288,7 +288,7 @@ def test_random_small_shapes(lib, path, case):
     rng = np.random.default_rng(1000 + case)
     N = int(rng.integers(1, 7))
     D = int(rng.choice([8, 24, 64, 136, 200]))
-    V = int(rng.integers(2, 260)) * 8
+    V = int(rng.integers(9, 2100))                       # any vocabulary size, odd ones included
     T_hi = int(rng.integers(1, 70))
     U_hi = int(rng.integers(0, max(1, min(T_hi, 40)) + 1))
     dtype = "bf16" if (path == AUTO or case % 2) else "fp32"
@@ -307,6 +307,18 @@ def test_random_small_shapes(lib, path, case):
     ref = H.run_oracle(batch, beam=beam if beam > 0 else None)
     tol = (2e-3, 1e-2) if dtype == "bf16" else (2e-5, 5e-4)
     H.assert_parity(gpu, ref, batch, tol=tol)
+
+
+@pytest.mark.parametrize("path", [SIMT, AUTO])
+def test_zero_and_negative_utterance_weights(lib, path):
+    # c_n = 0 switches an utterance's gradient off without flagging it; a negative c_n flips its sign
+    cfg = small("c3", V=4096 + 77, D=128, N=5, T_div=8, U_div=4)
+    batch = wl.make_batch(cfg, with_bias=True, permute_ids=True)
+    c = np.array([0.0, -1.0, 1.0, 3.0, -0.5], dtype=np.float32)
+    gpu = H.run_gpu(lib, batch, gemm_path=path, utt_weights=c, chunk=1024)
+    ref = H.run_oracle(batch, utt_weights=c)
+    H.assert_parity(gpu, ref, batch)
+    assert np.all(gpu["dH"][0] == 0.0) and gpu["flags"][0] == 0 and gpu["loss"][0] > 0
 
 
 @pytest.mark.parametrize("V,D", [(8192 + 384, 256), (4 * 4096 + 1000, 64)])   # one upload / four segments of W

@@ -12,7 +12,10 @@
  * the call's later steps).  Every buffer is owned by the caller; the library
  * keeps no pointers between calls and, except where an entry point says
  * otherwise, allocates no device memory.  Calls on one device must not be issued
- * from several host threads at once.
+ * from several host threads at once.  pruned_ctc_fwd_bwd, its traced and host-buffer
+ * forms and pctc_greedy_decode upload small per-call index tables from temporary host
+ * memory and therefore cannot be part of a CUDA graph: on a stream that is being
+ * captured they return PCTC_ERR_UNSUPPORTED before enqueuing anything.
  * Functions return a status code and never throw or abort.
  */
 #ifndef PRUNEDCTC_H_

@@ -263,6 +263,14 @@ pctc_status_t pruned_ctc_fwd_bwd(const pctc_problem_t* p, const void* hidden, co
 }  // extern "C"
 
 namespace {
+// Every call uploads per-call index tables from temporary host memory.  A stream capture would record
+// those copies and read that memory again at every replay, long after it is gone, so a capturing
+// stream is refused before anything is enqueued.
+bool stream_is_capturing(cudaStream_t stream) {
+  cudaStreamCaptureStatus cs = cudaStreamCaptureStatusNone;
+  return cudaStreamIsCapturing(stream, &cs) == cudaSuccess && cs != cudaStreamCaptureStatusNone;
+}
+
 // The whole call.  `pipe` is non-null only for the host-buffer entry point.
 pctc_status_t run_call(const pctc_problem_t* p, const void* hidden, const void* W, const void* bias,
                        const int32_t* targets, const int32_t* input_lengths, const int32_t* target_lengths,
@@ -285,6 +293,7 @@ pctc_status_t run_call(const pctc_problem_t* p, const void* hidden, const void* 
     return PCTC_ERR_INVALID_ARG;   // (null dH / dW are aligned)
   if (pl.use_umma && !umma_available()) return PCTC_ERR_CUDA;
   cudaStream_t stream = (cudaStream_t)stream_v;
+  if (stream_is_capturing(stream)) return PCTC_ERR_UNSUPPORTED;
   Aux aux;
   if (get_aux(&aux) != cudaSuccess) return PCTC_ERR_CUDA;
   char* ws = (char*)workspace;
@@ -664,6 +673,7 @@ pctc_status_t pruned_ctc_fwd_bwd_host(const pctc_problem_t* p, const void* hidde
   if ((size_t)device_scratch & (ALIGN - 1)) return PCTC_ERR_INVALID_ARG;
   if (scratch_bytes < h.total) return PCTC_ERR_WORKSPACE_TOO_SMALL;
   cudaStream_t stream = (cudaStream_t)stream_v;
+  if (stream_is_capturing(stream)) return PCTC_ERR_UNSUPPORTED;
   char* d = (char*)device_scratch;
   const bool want_db = bias && dbias;
 #define PCTC_CUDA(call)                              \
@@ -736,6 +746,7 @@ pctc_status_t pctc_greedy_decode(const pctc_problem_t* p, const void* hidden, co
   if (((size_t)workspace & (ALIGN - 1)) || ((size_t)hidden & 15) || ((size_t)W & 15)) return PCTC_ERR_INVALID_ARG;
   if (g.use_umma && !umma_available()) return PCTC_ERR_CUDA;
   cudaStream_t stream = (cudaStream_t)stream_v;
+  if (stream_is_capturing(stream)) return PCTC_ERR_UNSUPPORTED;
   char* ws = (char*)workspace;
   const int N = g.N, M = g.M, D = g.D;
 #define PCTC_CUDA(call)                              \

@@ -415,3 +415,29 @@ def test_bf16_shapes_the_tensor_core_path_does_not_cover_fall_to_the_fma_kernels
     batch = wl.make_batch(cfg, with_bias=True, permute_ids=True)
     gpu = H.run_gpu(lib, batch, gemm_path=AUTO)
     H.assert_parity(gpu, H.run_oracle(batch), batch)
+
+
+def test_capturing_stream_is_refused_before_anything_is_enqueued(lib):
+    # the call uploads per-call index tables from temporary host memory, which a graph replay would
+    # read again after it is gone: a capturing stream gets "unsupported" and an empty capture
+    import torch
+    batch = wl.make_batch(small("c2", V=2048, D=64, N=3, T_div=10, U_div=4))
+    dev = torch.device("cuda:0")
+    hidden = torch.from_numpy(batch.hidden).to(dev).to(torch.bfloat16)
+    W = torch.from_numpy(batch.W).to(dev).to(torch.bfloat16)
+    targets = torch.from_numpy(batch.targets).to(dev)
+    args = (hidden, W, None, targets, batch.input_lengths, batch.target_lengths, batch.blank)
+    eager = lib.pruned_ctc_fwd_bwd(*args, check_status=True)
+    torch.cuda.synchronize()
+    loss0 = eager["loss"].clone()
+    s = torch.cuda.Stream()
+    s.wait_stream(torch.cuda.current_stream())
+    g = torch.cuda.CUDAGraph()
+    with pytest.raises(lib.PctcError) as ei:
+        with torch.cuda.graph(g, stream=s):
+            lib.pruned_ctc_fwd_bwd(*args, workspace=eager["workspace"], out=eager)
+    assert ei.value.status == 3
+    torch.cuda.synchronize()
+    again = lib.pruned_ctc_fwd_bwd(*args, workspace=eager["workspace"], out=eager, check_status=True)   # still usable
+    torch.cuda.synchronize()
+    assert torch.equal(again["loss"], loss0)

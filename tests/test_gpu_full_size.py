@@ -1,5 +1,6 @@
 """Parity at full size: the bf16 configurations c2-c5 exactly as bench.py launches them
-(default chunk; c4 is the bench default: D=4096, V=151,936, about 8,000 frames), checked on
+(default chunk; c4 is the bench default: D=4096, V=151,936, about 8,000 frames) and the smallest
+workload of the paper's own grid (g16k: 160 utterances of 100 frames, D=512, V=180,000), checked on
 outputs the oracle can compute one by one (integer outputs, every per-utterance loss, dH of
 two utterances, sampled rows of dW) and on identities that hold at any size.  c1 (fp32) is
 compared in full in test_gpu_parity.py."""
@@ -15,7 +16,7 @@ from tests import helpers as H
 pytestmark = pytest.mark.gpu
 
 
-@pytest.mark.parametrize("name", ["c2", "c3", "c4", "c5"])
+@pytest.mark.parametrize("name", ["c2", "c3", "c4", "c5", "g16k"])
 def test_full_size_sampled_parity(lib, name):
     import torch
     cfg = wl.CONFIGS[name]

@@ -18,9 +18,21 @@ pytestmark = pytest.mark.gpu
 
 @pytest.mark.parametrize("name", ["c2", "c3", "c4", "c5", "g16k"])
 def test_full_size_sampled_parity(lib, name):
+    check_sampled_parity(lib, wl.CONFIGS[name])
+
+
+def test_chunk_buffer_beyond_2_to_31_elements(lib):
+    # 64 utterances of about 4,200 frames: M x C = 268,000 x 8,192 > 2^31 elements in the dlogits chunk,
+    # so every index into it has to be 64-bit; narrow head and small vocabulary keep the oracle quick
+    cfg = wl.Config("bigM", N=64, T_lo=4150, T_hi=4250, D=256, V=8192 + 40, dtype="bf16", U_lo=5, U_hi=20,
+                    zipf_s=1.1, seed=1777)
+    check_sampled_parity(lib, cfg)
+
+
+def check_sampled_parity(lib, cfg):
     import torch
-    cfg = wl.CONFIGS[name]
     batch = wl.make_batch(cfg)
+    assert batch.M * min(cfg.V, 8192) > 2 ** 31 or cfg.name != "bigM"
     dev = torch.device("cuda:0")
     hidden = torch.from_numpy(batch.hidden).to(dev).to(torch.bfloat16)
     W = torch.from_numpy(batch.W).to(dev).to(torch.bfloat16)

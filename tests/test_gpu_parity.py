@@ -441,3 +441,14 @@ def test_capturing_stream_is_refused_before_anything_is_enqueued(lib):
     again = lib.pruned_ctc_fwd_bwd(*args, workspace=eager["workspace"], out=eager, check_status=True)   # still usable
     torch.cuda.synchronize()
     assert torch.equal(again["loss"], loss0)
+
+
+def test_million_class_vocabulary(lib):
+    # V = 1,000,003 (odd, 123 chunks of 8,192 on the tensor-core path): bitmap ranking over 31k words,
+    # class map of 4 MB, many column splits of the normaliser, a ragged last chunk of 579 classes
+    cfg = dataclasses.replace(wl.CONFIGS["c2"], name="v1m", N=3, T_lo=30, T_hi=48, D=32, V=1_000_003,
+                              U_lo=4, U_hi=12, zipf_s=1.05, seed=4242)
+    batch = wl.make_batch(cfg, permute_ids=True)
+    gpu = H.run_gpu(lib, batch, chunk=8192)
+    ref = H.run_oracle(batch)
+    H.assert_parity(gpu, ref, batch)

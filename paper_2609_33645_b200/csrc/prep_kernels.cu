@@ -115,6 +115,15 @@ __global__ void k_stack_frames(const char* __restrict__ hidden, char* __restrict
   copy_row(hidden + ((size_t)n * T + t) * row_bytes, X + (size_t)m * row_bytes, row_bytes);
 }
 
+__device__ __forceinline__ void store4(float* dst, float4 v) { *reinterpret_cast<float4*>(dst) = v; }
+__device__ __forceinline__ void store4(__nv_bfloat16* dst, float4 v) {
+  const __nv_bfloat162 lo = __floats2bfloat162_rn(v.x, v.y), hi = __floats2bfloat162_rn(v.z, v.w);
+  uint2 o;
+  o.x = *reinterpret_cast<const unsigned*>(&lo);
+  o.y = *reinterpret_cast<const unsigned*>(&hi);
+  *reinterpret_cast<uint2*>(dst) = o;
+}
+
 template <typename TOut>
 __global__ void k_unstack_cast(const float* __restrict__ acc, int nslab, size_t slab_stride, TOut* __restrict__ dH,
                                int T, int D, const int* __restrict__ T_n, const int* __restrict__ row0) {
@@ -125,6 +134,17 @@ __global__ void k_unstack_cast(const float* __restrict__ acc, int nslab, size_t 
     return;
   }
   const float* src = acc + ((size_t)row0[n] + t) * D;
+  if ((D & 3) == 0) {                          // four columns per thread: 16-byte loads, 8- or 16-byte stores
+    for (int d = threadIdx.x * 4; d < D; d += blockDim.x * 4) {
+      float4 v = *reinterpret_cast<const float4*>(src + d);
+      for (int s = 1; s < nslab; ++s) {        // k-split partial sums, fixed order
+        const float4 u = *reinterpret_cast<const float4*>(src + s * slab_stride + d);
+        v.x += u.x; v.y += u.y; v.z += u.z; v.w += u.w;
+      }
+      store4(dst + d, v);
+    }
+    return;
+  }
   for (int d = threadIdx.x; d < D; d += blockDim.x) {
     float v = src[d];
     for (int s = 1; s < nslab; ++s) v += src[s * slab_stride + d];     // k-split partial sums, fixed order

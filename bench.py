@@ -130,8 +130,8 @@ def reduce_over_ranks(ms: float, frames: float, flops: float, device=None):
     return float(t[0].item()), float(s[0].item()), float(s[1].item())
 
 
-def _traced_call(binding, hidden, W, targets, il, tl, batch, res, trace, call):
-    binding.pruned_ctc_fwd_bwd(hidden, W, None, targets, il, tl, batch.blank, workspace=res["workspace"], out=res,
+def _traced_call(binding, hidden, W, bias_dev, targets, il, tl, batch, res, trace, call):
+    binding.pruned_ctc_fwd_bwd(hidden, W, bias_dev, targets, il, tl, batch.blank, workspace=res["workspace"], out=res,
                                trace=trace, **call)
     return trace
 
@@ -219,6 +219,7 @@ def main():
                     help="data-parallel training step: dW of every step is summed over the ranks, one NCCL "
                          "all-reduce per vocabulary chunk on a communication stream (off by default: the "
                          "head-and-loss path itself has no exchange step)")
+    ap.add_argument("--bias", action="store_true", help="give the head a bias (dbias is then part of the step)")
     ap.add_argument("--e2e-steps", type=int, default=3)
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--cpu-frames", type=int, default=1024)
@@ -265,7 +266,7 @@ def main():
     peaks = load_peaks()
 
     # ---- the batch: every rank its own utterances, same shape distribution ----
-    batch = wl.make_batch(cfg, seed=rank_seed(cfg, rank))
+    batch = wl.make_batch(cfg, seed=rank_seed(cfg, rank), with_bias=args.bias)
     tdt = torch.bfloat16 if cfg.dtype == "bf16" else torch.float32
     h_hidden = torch.from_numpy(batch.hidden).to(tdt).pin_memory()
     h_W = torch.from_numpy(batch.W).to(tdt).pin_memory()
@@ -273,6 +274,8 @@ def main():
     hidden = h_hidden.to(dev, non_blocking=True)
     W = h_W.to(dev, non_blocking=True)
     targets = h_targets.to(dev, non_blocking=True)
+    h_bias = None if batch.bias is None else torch.from_numpy(batch.bias).to(tdt).pin_memory()
+    bias_dev = None if h_bias is None else h_bias.to(dev, non_blocking=True)
     il, tl = batch.input_lengths, batch.target_lengths
     M, D, V, N = batch.M, cfg.D, cfg.V, cfg.N
     flops_per_step = (6.0 if args.frozen_head else 8.0) * M * D * V
@@ -291,10 +294,10 @@ def main():
         max_K = 1 + int(np.unique(toks).size)
     dev_call = dict(call, skip_dW=args.frozen_head, max_K=max_K)
 
-    res = binding.pruned_ctc_fwd_bwd(hidden, W, None, targets, il, tl, batch.blank, check_status=True, **dev_call)
+    res = binding.pruned_ctc_fwd_bwd(hidden, W, bias_dev, targets, il, tl, batch.blank, check_status=True, **dev_call)
     torch.cuda.synchronize()
     for _ in range(max(0, args.warmup - 1)):
-        res = binding.pruned_ctc_fwd_bwd(hidden, W, None, targets, il, tl, batch.blank,
+        res = binding.pruned_ctc_fwd_bwd(hidden, W, bias_dev, targets, il, tl, batch.blank,
                                          workspace=res["workspace"], out=res, **dev_call)
     torch.cuda.synchronize()
 
@@ -306,7 +309,7 @@ def main():
         dw_rows = dp.chunk_rows(V, chunk)
         for _ in range(2):                       # NCCL sets up its channels at the first collective
             dp.allreduce_rows(res["dW"], dw_rows, dp.dw_ready_events(
-                _traced_call(binding, hidden, W, targets, il, tl, batch, res, traces[0], dev_call)), comm_stream=comm)
+                _traced_call(binding, hidden, W, bias_dev, targets, il, tl, batch, res, traces[0], dev_call)), comm_stream=comm)
         torch.cuda.synchronize()
     sampler = ClockSampler(local_dev)
     if rank == 0:
@@ -318,7 +321,7 @@ def main():
     torch.cuda.synchronize()
     ev0.record()
     for s in range(args.steps):
-        binding.pruned_ctc_fwd_bwd(hidden, W, None, targets, il, tl, batch.blank, workspace=res["workspace"],
+        binding.pruned_ctc_fwd_bwd(hidden, W, bias_dev, targets, il, tl, batch.blank, workspace=res["workspace"],
                                    out=res, trace=traces[s], **dev_call)
         if sum_dW:
             dp.allreduce_rows(res["dW"], dw_rows, dp.dw_ready_events(traces[s]), comm_stream=comm)
@@ -372,12 +375,13 @@ def main():
     # kernels launched by the library inside the timed region
     dp_launches = 4 if args.beam > 0 else 2      # sweeps (+ best-alignment sweeps, arc flags), occupancies
     # subset (3), stacking, gather + Z_U, DP, normaliser + combine, loss, row clean-up, chunks, un-stacking
-    launches_per_step = 3 + 1 + 2 + dp_launches + 2 + 1 + 1 + (2 if args.frozen_head else 3) * nchunks + 1
+    launches_per_step = (3 + 1 + 2 + dp_launches + 2 + 1 + 1 + (2 if args.frozen_head else 3) * nchunks + 1
+                        + (nchunks if args.bias else 0))          # + column sums for dbias
     gpu_launches = launches_per_step * args.steps
 
     # ---- end to end through the host-buffer entry point ----
     e2e = None
-    if args.e2e_steps > 0 and not args.frozen_head:
+    if args.e2e_steps > 0 and not args.frozen_head and not args.bias:
         h_res = binding.pruned_ctc_fwd_bwd_host(h_hidden, h_W, None, h_targets, il, tl, batch.blank,
                                                 device=dev, **call)
         torch.cuda.synchronize()
@@ -426,7 +430,7 @@ def main():
         ms_per_step=ms_per_step, higher_is_better=True, scaling="weak", vs_baseline=None,
         dtype=cfg.dtype, data="synthetic",
         config=dict(workload=cfg.name, N=N, T_range=[cfg.T_lo, cfg.T_hi], D=D, V=V, M_frames=M,
-                    K_selected=int(res["K"].item()), beam=args.beam, chunk=chunk, frozen_head=args.frozen_head, max_K=max_K,
+                    K_selected=int(res["K"].item()), beam=args.beam, chunk=chunk, frozen_head=args.frozen_head, bias=args.bias, max_K=max_K,
                     l2="inputs larger than L2 (W and dW are %.2f GB each)" % (W.numel() * 2 / 1e9),
                     parallelism=("utterance-sharded data parallel, dW all-reduced per vocabulary chunk (NCCL)"
                                  if sum_dW else "independent utterance batches per GPU, no collective")),

@@ -25,7 +25,7 @@ struct Plan {
   bool bf16, use_umma, beam;
   // byte offsets into the workspace
   size_t o_status, o_meta_i, o_cell0, o_bitmap, o_wrank, o_vmap, o_U, o_K, o_rel, o_flags, o_X, o_lambda,
-      o_partial, o_WU, o_S, o_G, o_roww, o_alpha, o_beta, o_va, o_vb, o_offa, o_offb, o_best, o_maskf, o_maskb, o_mcell0, o_chunk, o_dHacc;
+      o_partial, o_WU, o_S, o_G, o_roww, o_alpha, o_beta, o_va, o_vb, o_offa, o_offb, o_best, o_maskf, o_maskb, o_mcell0, o_chunk, o_colpart, o_dHacc;
   size_t total;
   size_t meta_ints;  // T_n[N] | U_n[N] | row0[N+1] | row_utt[M]
 };
@@ -116,6 +116,8 @@ pctc_status_t make_plan(const pctc_problem_t* p, const int32_t* Tn, const int32_
     pl->o_mcell0 = take((size_t)pl->N * 8);
   }
   pl->o_chunk = take((size_t)pl->M * pl->chunk * pl->elem);
+  // db_c on the tensor-core path: per block of 32 rows, the column sums the dlogits epilogue forms
+  pl->o_colpart = pl->use_umma ? take((size_t)((pl->M + 31) / 32) * pl->chunk * 4) : 0;
   // few output tiles (small M x D): the dX contraction of a chunk is cut along k into ksplit ranges, each
   // with its own fp32 accumulator, summed in a fixed order when dH is written (deterministic)
   pl->ksplit = pl->use_umma ? umma_accum_splits(pl->M, pl->D, pl->chunk, DH_SPLIT_EXTRA_BYTES) : 1;
@@ -496,6 +498,10 @@ pctc_status_t run_call(const pctc_problem_t* p, const void* hidden, const void* 
       e.gamma = d_G;
       e.ld_gamma = (long long)pl.ldS;
       e.roww = dp.roww;
+      if (pl.use_umma && bias && dbias) {
+        e.colpart = (float*)(ws + pl.o_colpart);
+        e.ld_colpart = pl.chunk;
+      }
       GemmCall c{d_X, D, false, Wc, D, false, M, Cc, D};
       PCTC_CUDA(run_gemm(pl.use_umma, pl.bf16, c, e, d_status, stream));
     }
@@ -531,7 +537,11 @@ pctc_status_t run_call(const pctc_problem_t* p, const void* hidden, const void* 
     }
     if (bias && dbias) {
       PCTC_MARK(PCTC_PHASE_DBIAS);
-      PCTC_CUDA(column_sums(d_chunk, pl.bf16, pl.chunk, M, Cc, dbias, pl.bf16, v0, p->accumulate_dW != 0, stream));
+      if (pl.use_umma)
+        PCTC_CUDA(colpart_sums((const float*)(ws + pl.o_colpart), pl.chunk, (M + 31) / 32, Cc, dbias, pl.bf16, v0,
+                               p->accumulate_dW != 0, stream));
+      else
+        PCTC_CUDA(column_sums(d_chunk, pl.bf16, pl.chunk, M, Cc, dbias, pl.bf16, v0, p->accumulate_dW != 0, stream));
     }
     if (pipe && pipe->dW_host && !p->skip_dW) {          // these rows of dW are final: send them home now
       cudaEvent_t ev = aux.chunk_done[ci & 1];

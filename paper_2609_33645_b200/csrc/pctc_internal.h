@@ -42,6 +42,8 @@ struct Epilogue {
   int partial_offset = 0;       // segment of B writes its splits at partial_offset .. +nsplit-1
   int accumulate = 0;           // EPI_ACCUM_F32 / EPI_STORE_OUT: add to the destination instead of overwriting
   int out_is_bf16 = 0;          // EPI_DLOGITS / EPI_STORE_OUT destination type
+  float* colpart = nullptr;     // EPI_DLOGITS on the tensor-core path: [ceil(m/32), ld_colpart] column sums of
+  long long ld_colpart = 0;     //   each block of 32 rows of the rounded output (db_c = dZ_c^T 1), or null
   int ksplit = 1;               // EPI_ACCUM_F32 on the tensor-core path: the contraction is cut into this many
   int ksplit_rows = 0;          //   ranges of k; range s accumulates into rows [s * ksplit_rows, ...) of `out`
 };
@@ -111,6 +113,10 @@ cudaError_t zero_nonfinite_rows(void* X, int M, int D, int elem_bytes, const int
 
 // dH[n,t,:] = T(sum over slabs s < nslab, in ascending s, of acc[s*slab_stride + (row0[n]+t)*D + :]) for
 // t < T_n, zero for padded frames.
+// db[v0 + j] (+)= sum over the nblocks row blocks, in ascending order, of colpart[b * ld + j], j < cols.
+cudaError_t colpart_sums(const float* colpart, long long ld, int nblocks, int cols, void* db, bool db_bf16,
+                         long long v0, bool accumulate, cudaStream_t stream);
+
 cudaError_t unstack_cast(const float* acc, int nslab, size_t slab_stride, void* dH, int N, int T, int D,
                          bool out_bf16, const int* T_n, const int* row0, cudaStream_t stream);
 

@@ -188,6 +188,27 @@ __global__ void k_column_sums(const TIn* __restrict__ chunk, long long ld, int M
   }
 }
 
+// --- second stage of db_c when the dlogits epilogue has already summed blocks of 32 rows: a fixed-order
+// sum over the row blocks (reads 1/16 of the bytes of the chunk itself) ---
+template <typename TOut>
+__global__ void k_colpart_sums(const float* __restrict__ colpart, long long ld, int nblocks, int cols,
+                               TOut* __restrict__ db, long long v0, bool accumulate) {
+  __shared__ float s_part[8][33];
+  const int cx = threadIdx.x, ry = threadIdx.y;          // 32 columns x 8 interleaved row-block lanes
+  const int j = blockIdx.x * 32 + cx;
+  float acc = 0.f;
+  if (j < cols)
+    for (int b = ry; b < nblocks; b += 8) acc += colpart[(size_t)b * ld + j];
+  s_part[ry][cx] = acc;
+  __syncthreads();
+  if (ry == 0 && j < cols) {
+    float tot = 0.f;
+    for (int r = 0; r < 8; ++r) tot += s_part[r][cx];
+    if (accumulate) tot += float(db[v0 + j]);
+    db[v0 + j] = TOut(tot);
+  }
+}
+
 __global__ void k_lse_combine(const float2* __restrict__ partial, int nsplit, int M, float* __restrict__ lambda) {
   int i = blockIdx.x * blockDim.x + threadIdx.x;
   if (i >= M) return;
@@ -310,6 +331,16 @@ cudaError_t column_sums(const void* chunk, bool chunk_bf16, long long ld, int M,
     k_column_sums<<<grid, block, 0, stream>>>((const float*)chunk, ld, M, cols, (float*)db, v0, accumulate);
   else
     return cudaErrorInvalidValue;
+  return cudaGetLastError();
+}
+
+cudaError_t colpart_sums(const float* colpart, long long ld, int nblocks, int cols, void* db, bool db_bf16,
+                         long long v0, bool accumulate, cudaStream_t stream) {
+  dim3 block(32, 8), grid((cols + 31) / 32);
+  if (db_bf16)
+    k_colpart_sums<<<grid, block, 0, stream>>>(colpart, ld, nblocks, cols, (__nv_bfloat16*)db, v0, accumulate);
+  else
+    k_colpart_sums<<<grid, block, 0, stream>>>(colpart, ld, nblocks, cols, (float*)db, v0, accumulate);
   return cudaGetLastError();
 }
 

@@ -669,6 +669,28 @@ k_umma_gemm(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
               }
               fence_async_smem();                      // staged data visible to the TMA engine
               __syncwarp();
+              if (EPI == EPI_DLOGITS && a.e.colpart != nullptr && row0_cta + q * 32 < a.m) {
+                // db_c = dZ_c^T 1, first stage: lane c sums column c of the staged box, i.e. the rounded
+                // values of this warp's 32 rows (rows past m hold exact zeros), into the row block's slot
+                // lanes 0-15 take rows 0-15, lanes 16-31 rows 16-31; each reads column pair (lane & 15)
+                // as one 32-bit word, widens both halves and adds them with one packed fp32 add
+                const int cp = lane & 15, rbase = lane & 16;
+                float s0 = 0.f, s1 = 0.f;
+#pragma unroll
+                for (int rr = 0; rr < 16; ++rr) {
+                  const int row = rbase + rr;
+                  const unsigned piece = (unsigned)(cp >> 2) ^ (unsigned)((row >> 1) & 3);
+                  const unsigned wv = *reinterpret_cast<const unsigned*>(box + row * 64 + (piece << 4) + (cp & 3) * 4);
+                  s0 += __uint_as_float(wv << 16);
+                  s1 += __uint_as_float(wv & 0xffff0000u);
+                }
+                s0 += __shfl_xor_sync(0xffffffffu, s0, 16);
+                s1 += __shfl_xor_sync(0xffffffffu, s1, 16);
+                const float cs = (lane & 16) ? s1 : s0;                    // lanes 0-15: even columns, 16-31: odd
+                const int col = 2 * cp + ((lane >> 4) & 1);
+                if (j0 + col < n_eff)
+                  a.e.colpart[(long long)((row0_cta + q * 32) >> 5) * a.e.ld_colpart + j0 + col] = cs;
+              }
               if (lane == 0) {
                 if ((EPI == EPI_ACCUM_F32 || EPI == EPI_STORE_OUT) && a.e.accumulate)
                   tma_reduce_add_2d(&tmC, box, j0 + b * 16, row0_out + q * 32);

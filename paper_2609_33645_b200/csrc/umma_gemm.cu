@@ -282,6 +282,14 @@ __device__ __forceinline__ void fmul2(float& d0, float& d1, float a0, float a1, 
       : "=f"(d0), "=f"(d1)
       : "f"(a0), "f"(a1), "f"(b0), "f"(b1));
 }
+// v[0..31] += b[0..31]: the staged bias of a column group, read as eight 16-byte words
+__device__ __forceinline__ void add_bias32(float (&v)[32], const float* b) {
+#pragma unroll
+  for (int c = 0; c < 32; c += 4) {
+    const float4 bb = *reinterpret_cast<const float4*>(b + c);
+    v[c] += bb.x; v[c + 1] += bb.y; v[c + 2] += bb.z; v[c + 3] += bb.w;
+  }
+}
 __device__ __forceinline__ float lg2(float x) {
   float y;
   asm("lg2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
@@ -608,10 +616,7 @@ k_umma_gemm(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
                 v[c] = (j0 + c < n_eff) ? v[c] + (has_bias ? sb[g0 + c] : 0.f) - lam : 0.f;
             }
             if (EPI == EPI_DLOGITS) {
-              if (has_bias) {
-#pragma unroll
-                for (int c = 0; c < 32; ++c) v[c] += sb[g0 + c];
-              }
+              if (has_bias) add_bias32(v, sb + g0);
               // w p = exp2(z log2(e) + off2), off2 = log2(w) - lambda log2(e): one packed FMA per two logits
 #pragma unroll
               for (int c = 0; c < 32; c += 2) {
@@ -723,9 +728,10 @@ k_umma_gemm(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
             }
           } else if (EPI == EPI_LSE_PARTIAL) {
             // running (max, sum of exp) in the base-2 domain: x = z * log2(e)
-            if (!has_bias && j0 + 32 <= n_eff) {
-              // whole group inside the matrix, no bias: max over the raw logits, then one packed FMA per
-              // two logits forms x - max and feeds the exponentials
+            if (j0 + 32 <= n_eff) {
+              // whole group inside the matrix: max over the logits, then one packed FMA per two logits
+              // forms x - max and feeds the exponentials
+              if (has_bias) add_bias32(v, sb + cg * 32);
               float gm = v[0];
 #pragma unroll
               for (int c = 1; c < 32; ++c) gm = fmaxf(gm, v[c]);

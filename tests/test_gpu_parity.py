@@ -143,10 +143,11 @@ def test_beam_bf16_reduced_c5_shape(lib):
 
 def test_two_calls_are_bitwise_identical_and_workspace_is_reusable(lib):
     import torch
-    batch = wl.make_batch(small("c2", V=4096, D=128, N=4, T_div=8, U_div=4))
+    # with a bias (two-stage column sums) and few output tiles (the dX contraction is cut along k)
+    batch = wl.make_batch(small("c2", V=4096, D=128, N=4, T_div=8, U_div=4), with_bias=True)
     a = H.run_gpu(lib, batch)
     b = H.run_gpu(lib, batch)
-    for k in ("loss", "dH", "dW", "subset", "relabeled"):
+    for k in ("loss", "dH", "dW", "dbias", "subset", "relabeled"):
         np.testing.assert_array_equal(a[k], b[k])
     torch.cuda.synchronize()
 

@@ -453,3 +453,36 @@ def test_million_class_vocabulary(lib):
     gpu = H.run_gpu(lib, batch, chunk=8192)
     ref = H.run_oracle(batch)
     H.assert_parity(gpu, ref, batch)
+
+
+@pytest.mark.parametrize("case", range(40))
+def test_random_wide_shapes(lib, case):
+    # a wider seeded sweep: head widths up to 1024 (including widths that are no multiple of 64), odd
+    # vocabularies up to 40,000, up to 500 frames, any chunk width, optional bias, beam, signed utterance
+    # weights and frozen head, mostly on the tensor-core path
+    rng = np.random.default_rng(77000 + case)
+    N = int(rng.integers(1, 9))
+    D = int(rng.choice([8, 16, 64, 72, 128, 256, 512, 520, 1024]))
+    V = int(rng.choice([rng.integers(2, 300), rng.integers(300, 5000), rng.integers(5000, 40000)]))
+    T_hi = int(rng.choice([rng.integers(1, 20), rng.integers(20, 200), rng.integers(200, 500)]))
+    U_hi = int(rng.integers(0, max(1, min(T_hi, 120)) + 1))
+    path = SIMT if int(rng.integers(0, 4)) == 0 else AUTO
+    dtype = "fp32" if (path == SIMT and rng.random() < 0.5) else "bf16"
+    cfg = dataclasses.replace(wl.CONFIGS["c1"], name=f"wide{case}", N=N, T_lo=max(1, T_hi // 3), T_hi=T_hi, D=D, V=V,
+                              dtype=dtype, U_lo=0, U_hi=U_hi, zipf_s=[None, 1.0, 1.3][case % 3],
+                              blank=int(rng.integers(0, V)), seed=9000 + case, rms_norm=bool(case % 2))
+    batch = wl.make_batch(cfg, with_bias=bool(rng.integers(0, 2)), poison_padding=True,
+                          permute_ids=bool(rng.integers(0, 2)))
+    for n in range(N):
+        u = int(batch.target_lengths[n])
+        if u >= 3 and rng.random() < 0.5:
+            s0 = int(rng.integers(0, u - 2))
+            batch.targets[n, s0:s0 + 3] = batch.targets[n, s0]
+    beam = float(rng.choice([0.0, 0.0, 3.0, 12.0, 40.0]))
+    chunk = int(rng.choice([0, 0, 64, 200, 1024, 2048, 4096, 8192]))
+    w = rng.choice([0.0, 0.5, 1.0, 2.0], size=N).astype(np.float32) if rng.random() < 0.3 else None
+    frozen = bool(rng.random() < 0.2)
+    gpu = H.run_gpu(lib, batch, gemm_path=path, beam=beam, chunk=chunk, utt_weights=w, skip_dW=frozen)
+    ref = H.run_oracle(batch, beam=beam if beam > 0 else None, utt_weights=w)
+    tol = (2e-3, 1e-2) if dtype == "bf16" else (2e-5, 5e-4)
+    H.assert_parity(gpu, ref, batch, tol=tol)

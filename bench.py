@@ -367,8 +367,8 @@ def main():
     # DRAM bytes of the dominant kernel's launches of one step, from the ncu capture summarised in
     # profiles/umma_gemm_c4_speed_of_light.md (default workload and chunk only)
     traffic = None
-    if args.config == "c4" and not args.vocab and chunk == 8192 and not args.frozen_head and args.beam == 0:
-        traffic = dict(bytes_per_step=38.3e9, launches_per_step=58, bytes_per_launch_avg=38.3e9 / 58,
+    if args.config == "c4" and not args.vocab and chunk == 16384 and not args.frozen_head and args.beam == 0 and not args.bias:
+        traffic = dict(bytes_per_step=36.1e9, launches_per_step=31, bytes_per_launch_avg=36.1e9 / 31,
                        source="ncu dram__bytes_read.sum + dram__bytes_write.sum: the LSE launch and chunks 0-1 of each "
                               "chunk kernel, chunk averages scaled by launches")
 
@@ -382,8 +382,9 @@ def main():
     # ---- end to end through the host-buffer entry point ----
     e2e = None
     if args.e2e_steps > 0 and not args.frozen_head and not args.bias:
+        host_call = dict(beam=args.beam, chunk=args.chunk)     # 0: the host entry point's own default width
         h_res = binding.pruned_ctc_fwd_bwd_host(h_hidden, h_W, None, h_targets, il, tl, batch.blank,
-                                                device=dev, **call)
+                                                device=dev, **host_call)
         torch.cuda.synchronize()
         e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
         if world > 1:
@@ -392,7 +393,7 @@ def main():
         e0.record()
         for _ in range(args.e2e_steps):
             binding.pruned_ctc_fwd_bwd_host(h_hidden, h_W, None, h_targets, il, tl, batch.blank,
-                                            scratch=h_res["scratch"], out=h_res, device=dev, **call)
+                                            scratch=h_res["scratch"], out=h_res, device=dev, **host_call)
         e1.record()
         torch.cuda.synchronize()
         ms_e2e = e0.elapsed_time(e1) / args.e2e_steps

@@ -101,8 +101,8 @@ pctc_status_t pctc_workspace_bytes(const pctc_problem_t* problem,
  * The vocabulary chunk width C a call on this problem will use, and the number of
  * chunks ceil(V / C) (host-only; touches no device).  With problem->chunk > 0 it
  * is that value rounded up to the tile width of the path that runs; with 0 it is
- * the library's choice: 4,096 for fp32; for bf16 32,768 (D <= 1,024), 16,384
- * (D <= 2,048) or 8,192 columns, halved down to no less than 8,192 while the
+ * the library's choice: 4,096 for fp32; for bf16 32,768 (D <= 1,024) or 16,384
+ * columns, halved down to no less than 8,192 while the
  * [M, C] chunk temporary of Algorithm 1 (lines 12-13) would exceed 512 MiB.  The
  * chunk width changes the order of summation only, never what is computed.
  * nchunks_out may be NULL.  Same argument checks as pctc_workspace_bytes.
@@ -211,7 +211,8 @@ pctc_status_t pruned_ctc_fwd_bwd_traced(const pctc_problem_t* problem,
  * segment starts as soon as that segment has landed (for V >= 16,384; the summation
  * order of lambda then differs from the device entry point in the last bits);
  * Algorithm 1; the rows of dW go back to the host chunk by chunk while later
- * chunks are still being computed; loss, dH, dbias and the optional integer
+ * chunks are still being computed (with problem->chunk == 0 a bf16 call uses
+ * 8,192-column chunks here, so that the first rows leave early); loss, dH, dbias and the optional integer
  * outputs at the end.  `stream` waits for all of it.  The call does not synchronise: the host outputs are valid once
  * `stream` has been synchronised, and the host inputs must stay unchanged until
  * then.  Same return codes as pruned_ctc_fwd_bwd.  skip_dW, accumulate_dW and utt_weights

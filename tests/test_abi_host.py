@@ -63,7 +63,8 @@ def test_workspace_has_no_M_times_V_term(lib):
     (dict(dtype=1, V=10000), [50, 40], (4096, 3)),
     (dict(dtype=0, D=512, V=180000), [50, 40], (32768, 6)),         # narrow head: wide chunks
     (dict(dtype=0, D=2048, V=180000), [50, 40], (16384, 11)),
-    (dict(dtype=0, D=4096, V=151936), [50, 40], (8192, 19)),
+    (dict(dtype=0, D=4096, V=151936), [50, 40], (16384, 10)),
+    (dict(dtype=0, D=4096, V=151936, N=2, T=20000), [20000, 1], (8192, 19)),     # 512 MiB rule
     (dict(dtype=0, D=512, V=180000, N=2, T=16000), [16000, 1], (16384, 11)),   # [M, C] temporary <= 512 MiB
     (dict(dtype=0, D=512, V=180000, N=2, T=64000), [64000, 1], (8192, 22)),
     (dict(dtype=0, D=512, V=180000, chunk=1000), [50, 40], (1024, 176)),       # rounded up to the tile width

@@ -220,6 +220,9 @@ def main():
                          "all-reduce per vocabulary chunk on a communication stream (off by default: the "
                          "head-and-loss path itself has no exchange step)")
     ap.add_argument("--bias", action="store_true", help="give the head a bias (dbias is then part of the step)")
+    ap.add_argument("--dense-head", action="store_true",
+                    help="also time the three library GEMMs of a dense bf16 head that holds its [M, V] logits "
+                         "(forward, dX, dW: 6 M D V FLOPs) on the same shapes, as a yardstick for the time ratio")
     ap.add_argument("--e2e-steps", type=int, default=3)
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--cpu-frames", type=int, default=1024)
@@ -417,6 +420,39 @@ def main():
                                      batch.targets.shape[1], max_K=max_K_pre)
     ws_half = binding.workspace_bytes(prob_half, il, tl)
 
+    # ---- yardstick: a dense head's three library GEMMs with materialised logits (no loss, no softmax) ----
+    dense = None
+    if args.dense_head and cfg.dtype == "bf16" and rank == 0:
+        need = 2 * M * V
+        free_b, _ = torch.cuda.mem_get_info(dev)
+        if need + (2 << 30) < free_b:
+            X2 = hidden.reshape(-1, D)[:M].contiguous()
+            Zl = torch.empty((M, V), dtype=torch.bfloat16, device=dev)
+            dX2 = torch.empty_like(X2)
+            dW2 = torch.empty_like(W)
+            def dense_step():
+                torch.matmul(X2, W.t(), out=Zl)          # logits, kept
+                torch.matmul(Zl, W, out=dX2)             # dX  (Zl stands in for dlogits: same shape and dtype)
+                torch.matmul(Zl.t(), X2, out=dW2)        # dW
+            for _ in range(3):
+                dense_step()
+            torch.cuda.synchronize()
+            d0, d1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            d0.record()
+            for _ in range(args.steps):
+                dense_step()
+            d1.record()
+            torch.cuda.synchronize()
+            dms = d0.elapsed_time(d1) / args.steps
+            dense = dict(ms_per_step=dms, tflops=6.0 * M * D * V / (dms * 1e-3) / 1e12, logits_bytes=need,
+                         ratio_this_over_dense=ms_per_step / dms,
+                         what="torch.matmul (cuBLAS) forward + dX + dW with a materialised bf16 [M, V] logits "
+                              "array; no softmax, no loss: a lower bound for a dense head-and-loss step")
+            del Zl, dX2, dW2, X2
+            torch.cuda.empty_cache()
+        else:
+            dense = dict(skipped="the [M, V] logits array does not fit next to the benchmark's buffers")
+
     # ---- the oracle on the host cores, on a bounded sample ----
     cpu = None
     if not args.no_cpu_baseline and world == 1:
@@ -451,6 +487,8 @@ def main():
                         one_fp32_MxV_array=4 * M * V),
         e2e=e2e, gpu_launches=gpu_launches, clocks=clocks, cpu_baseline=cpu,
     )
+    if dense is not None:
+        line["dense_head"] = dense
     print(json.dumps(line), flush=True)
     if world > 1 or args.allreduce_dw:
         dist.destroy_process_group()

@@ -42,6 +42,10 @@ namespace {
 #define PCTC_TUNE_WALK_MB 32      // MB of A rows that a band of the column-walking kernels keeps hot in L2
 #endif
 
+#ifndef PCTC_TUNE_L2_PROMOTION
+#define PCTC_TUNE_L2_PROMOTION CU_TENSOR_MAP_L2_PROMOTION_L2_256B   // L2 fetch granularity of the TMA loads
+#endif
+
 #ifndef PCTC_TUNE_CTAS
 #define PCTC_TUNE_CTAS 2          // CTAs per tile: 2 = tcgen05 cta_group::2 pairs, 1 = independent CTAs
 #endif
@@ -829,7 +833,7 @@ bool make_map(CUtensorMap* map, const void* base, unsigned long long inner, unsi
       (box_inner * (fp32 ? 4u : 2u) == 64u) ? CU_TENSOR_MAP_SWIZZLE_64B : CU_TENSOR_MAP_SWIZZLE_128B;
   return fn(map, fp32 ? CU_TENSOR_MAP_DATA_TYPE_FLOAT32 : CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2,
             const_cast<void*>(base), dims, strides, box, estr,
-            CU_TENSOR_MAP_INTERLEAVE_NONE, swizzle, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+            CU_TENSOR_MAP_INTERLEAVE_NONE, swizzle, PCTC_TUNE_L2_PROMOTION,
             CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 

@@ -46,6 +46,10 @@ namespace {
 #define PCTC_TUNE_L2_PROMOTION CU_TENSOR_MAP_L2_PROMOTION_L2_256B   // L2 fetch granularity of the TMA loads
 #endif
 
+#ifndef PCTC_TUNE_MT2
+#define PCTC_TUNE_MT2 1           // 1: the dW contraction may use 512 x 256 tiles (see k_umma_gemm, MT)
+#endif
+
 #ifndef PCTC_TUNE_CTAS
 #define PCTC_TUNE_CTAS 2          // CTAs per tile: 2 = tcgen05 cta_group::2 pairs, 1 = independent CTAs
 #endif
@@ -75,6 +79,7 @@ struct UmmaArgs {
   int a_mn, b_mn;
   int nsplit;          // EPI_LSE_PARTIAL: column splits per row tile
   int raster_g;        // tile order: row tiles per band (see decode_unit)
+  int tile_mt;         // host only: 2 = launch the 512-row tile form (store epilogue, long contractions)
   int ksplit;          // EPI_ACCUM_F32: units per output tile, each contracting its own range of k
   int ksplit_rows;     //   ... and writing its own accumulator slab, this many rows further down
   int* status;
@@ -108,23 +113,25 @@ constexpr bool epi_uses_bias(int epi) {
 }
 constexpr bool epi_walks_splits(int epi) { return epi == EPI_LSE_PARTIAL || epi == EPI_ARGMAX_PARTIAL; }
 // ring depth: what is left of the 227 KB after the epilogue's own buffers
-constexpr int stages_of(int ctas, int epi, int ew) {
-  return ctas == 2 ? ((epi_uses_tma_store(epi) && ew == 8) ? 5 : 6) : (epi_uses_tma_store(epi) ? 3 : 4);
+// (mt = 2: two 128-row sub-tiles of A per CTA and stage, both accumulators on one tile: 48 KB stages, four of them)
+constexpr int stages_of(int ctas, int epi, int ew, int mt = 1) {
+  return mt == 2 ? 4
+                 : (ctas == 2 ? ((epi_uses_tma_store(epi) && ew == 8) ? 5 : 6) : (epi_uses_tma_store(epi) ? 3 : 4));
 }
-constexpr size_t ring_bytes(int ctas, int epi, int ew) {
-  return (size_t)stages_of(ctas, epi, ew) * (A_STAGE_BYTES + b_stage_bytes(ctas));
+constexpr size_t ring_bytes(int ctas, int epi, int ew, int mt = 1) {
+  return (size_t)stages_of(ctas, epi, ew, mt) * (mt * A_STAGE_BYTES + b_stage_bytes(ctas));
 }
-constexpr size_t off_stage(int ctas, int epi, int ew) { return ring_bytes(ctas, epi, ew); }
-constexpr size_t off_tail(int ctas, int epi, int ew) {
-  return ring_bytes(ctas, epi, ew) + (epi_uses_tma_store(epi) ? ew * STAGE_WARP_BYTES : 0);
+constexpr size_t off_stage(int ctas, int epi, int ew, int mt = 1) { return ring_bytes(ctas, epi, ew, mt); }
+constexpr size_t off_tail(int ctas, int epi, int ew, int mt = 1) {
+  return ring_bytes(ctas, epi, ew, mt) + (epi_uses_tma_store(epi) ? ew * STAGE_WARP_BYTES : 0);
 }
-constexpr size_t off_bias(int ctas, int epi, int ew) { return off_tail(ctas, epi, ew) + 256; }
-constexpr size_t off_list(int ctas, int epi, int ew) {
-  return off_bias(ctas, epi, ew) + (epi_uses_bias(epi) ? ew * warp_cols(ew) * 4 : 0);
+constexpr size_t off_bias(int ctas, int epi, int ew, int mt = 1) { return off_tail(ctas, epi, ew, mt) + 256; }
+constexpr size_t off_list(int ctas, int epi, int ew, int mt = 1) {
+  return off_bias(ctas, epi, ew, mt) + (epi_uses_bias(epi) ? ew * warp_cols(ew) * 4 : 0);
 }
 constexpr int list_words(int ew) { return warp_cols(ew) + 32; }
-constexpr size_t smem_bytes(int ctas, int epi, int ew) {
-  return 1024 + off_list(ctas, epi, ew) + (epi == EPI_DLOGITS ? ew * list_words(ew) * 4 : 0);
+constexpr size_t smem_bytes(int ctas, int epi, int ew, int mt = 1) {
+  return 1024 + off_list(ctas, epi, ew, mt) + (epi == EPI_DLOGITS ? ew * list_words(ew) * 4 : 0);
 }
 static_assert(sizeof(SharedTail) <= 256, "tail layout");
 
@@ -361,20 +368,27 @@ __device__ __forceinline__ void decode_unit(int u, int m_tiles, int n_tiles, int
 // ---------------------------------------------------------------------------------------------
 // The kernel
 // ---------------------------------------------------------------------------------------------
-template <int EPI, int CTAS, int EW>
+// MT = 2 (store epilogues only, two-CTA form): a tile is 512 x 256; every CTA stages two 128-row
+// sub-tiles of A per k-block next to its half of B, the two accumulators hold the two sub-tiles of ONE
+// tile (25% fewer operand bytes per FLOP than two 256 x 256 tiles), and the epilogue is not
+// overlapped with the next tile's MMAs.
+template <int EPI, int CTAS, int EW, int MT = 1>
 __global__ void __launch_bounds__(num_threads(EW), 1)
 k_umma_gemm(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
             const __grid_constant__ CUtensorMap tmC, UmmaArgs a) {
-  constexpr int STAGES = stages_of(CTAS, EPI, EW);
+  static_assert(MT == 1 || (MT == 2 && CTAS == 2 && (EPI == EPI_STORE_OUT || EPI == EPI_ACCUM_F32)), "tile height");
+  constexpr int STAGES = stages_of(CTAS, EPI, EW, MT);
   constexpr int B_STAGE_BYTES = b_stage_bytes(CTAS);
+  constexpr int A_STAGE = MT * A_STAGE_BYTES;  // this CTA's rows of A per stage
   constexpr int WARP_COLS = warp_cols(EW);
   constexpr int LIST_WORDS = list_words(EW);
-  constexpr int TILE_M = BM * CTAS;            // rows of the tile a CTA (pair) works on
+  constexpr int SUB_M = BM * CTAS;             // rows one MMA covers
+  constexpr int TILE_M = SUB_M * MT;           // rows of the tile a CTA (pair) works on
   extern __shared__ unsigned char smem_raw[];
   unsigned char* smem = (unsigned char*)(((size_t)smem_raw + 1023) & ~(size_t)1023);
   unsigned char* sA = smem;
-  unsigned char* sB = smem + (size_t)STAGES * A_STAGE_BYTES;
-  SharedTail* st = (SharedTail*)(smem + off_tail(CTAS, EPI, EW));
+  unsigned char* sB = smem + (size_t)STAGES * A_STAGE;
+  SharedTail* st = (SharedTail*)(smem + off_tail(CTAS, EPI, EW, MT));
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int rank = (CTAS == 2) ? (int)cluster_ctarank() : 0;     // position inside the pair
@@ -439,15 +453,20 @@ k_umma_gemm(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
             const unsigned ph = (g / STAGES) & 1u;
             if (!mbar_wait(&st->empty[s], ph ^ 1u, abort_flag, a.status, 1)) { ok = false; break; }
             // the leader's barrier counts the bytes of both CTAs
-            if (rank == 0) mbar_expect_tx(&st->full[s], CTAS * (A_STAGE_BYTES + B_STAGE_BYTES));
-            unsigned char* dA = sA + (size_t)s * A_STAGE_BYTES;
+            if (rank == 0) mbar_expect_tx(&st->full[s], CTAS * (A_STAGE + B_STAGE_BYTES));
+            unsigned char* dA = sA + (size_t)s * A_STAGE;
             unsigned char* dB = sB + (size_t)s * B_STAGE_BYTES;
-            if (!a.a_mn) {
-              load(dA, &tmA, kb * BK, row_a, &st->full[s]);
-            } else {
 #pragma unroll
-              for (int q = 0; q < BM / 64; ++q)
-                load(dA + q * MN_GROUP_BYTES, &tmA, row_a + q * 64, kb * BK, &st->full[s]);
+            for (int h = 0; h < MT; ++h) {               // sub-tile h: this CTA's 128 rows of pair rows h*256..
+              unsigned char* dAh = dA + h * A_STAGE_BYTES;
+              const int row_ah = row_a + h * SUB_M;
+              if (!a.a_mn) {
+                load(dAh, &tmA, kb * BK, row_ah, &st->full[s]);
+              } else {
+#pragma unroll
+                for (int q = 0; q < BM / 64; ++q)
+                  load(dAh + q * MN_GROUP_BYTES, &tmA, row_ah + q * 64, kb * BK, &st->full[s]);
+              }
             }
             if (!a.b_mn) {
               load(dB, &tmB, kb * BK, row_b, &st->full[s]);
@@ -472,7 +491,7 @@ k_umma_gemm(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
     if (lane == 0 && rank == 0) {        // the leader issues the MMAs of the pair
       const unsigned idesc = (1u << 4) | (1u << 7) | (1u << 10) | ((unsigned)(a.a_mn ? 1 : 0) << 15) |
                              ((unsigned)(a.b_mn ? 1 : 0) << 16) | ((unsigned)(BN >> 3) << 17) |
-                             ((unsigned)(TILE_M >> 4) << 24);
+                             ((unsigned)(SUB_M >> 4) << 24);
       const unsigned a_step = a.a_mn ? (2048u >> 4) : (32u >> 4);   // descriptor advance per 16 k
       const unsigned b_step = a.b_mn ? (2048u >> 4) : (32u >> 4);
       unsigned g = 0, it = 0;
@@ -483,8 +502,11 @@ k_umma_gemm(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
         split_range(k_blocks, ksplit, ks, kb0, kcnt);
         (void)mt;
         for (int nt = nt0; nt < nt0 + cnt && ok; ++nt, ++it) {
-          const unsigned acc = it & 1u, aph = (it >> 1) & 1u;
+          // MT == 1: the two accumulators alternate between tiles.  MT == 2: both belong to this tile
+          // (sub-tile h in accumulator h), so both must have been drained, and each is used once per tile.
+          const unsigned acc = (MT == 2) ? 0u : (it & 1u), aph = (MT == 2) ? (it & 1u) : ((it >> 1) & 1u);
           if (!mbar_wait(&st->tmem_empty[acc], aph ^ 1u, abort_flag, a.status, 2)) { ok = false; break; }
+          if (MT == 2 && !mbar_wait(&st->tmem_empty[1], aph ^ 1u, abort_flag, a.status, 2)) { ok = false; break; }
           tc_fence_after();
           const unsigned d_tmem = tmem_base + acc * BN;
           for (int kb = kb0; kb < kb0 + kcnt; ++kb, ++g) {
@@ -492,19 +514,26 @@ k_umma_gemm(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
             const unsigned ph = (g / STAGES) & 1u;
             if (!mbar_wait(&st->full[s], ph, abort_flag, a.status, 3)) { ok = false; break; }
             tc_fence_after();
-            const unsigned long long adesc = make_smem_desc(smem_u32(sA + (size_t)s * A_STAGE_BYTES), a.a_mn);
+            const unsigned long long adesc = make_smem_desc(smem_u32(sA + (size_t)s * A_STAGE), a.a_mn);
             const unsigned long long bdesc = make_smem_desc(smem_u32(sB + (size_t)s * B_STAGE_BYTES), a.b_mn);
 #pragma unroll
             for (int kk = 0; kk < BK / 16; ++kk) {
-              const unsigned long long ad = adesc + (unsigned long long)(kk * a_step);
               const unsigned long long bd = bdesc + (unsigned long long)(kk * b_step);
-              if (CTAS == 2) tc_mma_bf16_pair(d_tmem, ad, bd, idesc, (kb != kb0 || kk != 0) ? 1u : 0u);
-              else tc_mma_bf16(d_tmem, ad, bd, idesc, (kb != kb0 || kk != 0) ? 1u : 0u);
+#pragma unroll
+              for (int h = 0; h < MT; ++h) {
+                const unsigned long long ad =
+                    adesc + (unsigned long long)(kk * a_step) + (unsigned long long)(h * (A_STAGE_BYTES >> 4));
+                if (CTAS == 2) tc_mma_bf16_pair(d_tmem + h * BN, ad, bd, idesc, (kb != kb0 || kk != 0) ? 1u : 0u);
+                else tc_mma_bf16(d_tmem + h * BN, ad, bd, idesc, (kb != kb0 || kk != 0) ? 1u : 0u);
+              }
             }
             // frees the stage (in both CTAs) once these MMAs have read it
             if (CTAS == 2) tc_commit_pair(&st->empty[s]); else tc_commit(&st->empty[s]);
           }
-          if (ok) { if (CTAS == 2) tc_commit_pair(&st->tmem_full[acc]); else tc_commit(&st->tmem_full[acc]); }
+          if (ok) {
+            if (CTAS == 2) tc_commit_pair(&st->tmem_full[acc]); else tc_commit(&st->tmem_full[acc]);
+            if (MT == 2) tc_commit_pair(&st->tmem_full[1]);
+          }
         }
       }
       // all MMAs issued by this thread have completed before tensor memory is freed
@@ -517,10 +546,10 @@ k_umma_gemm(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
     const int q = warp & 3;                  // tensor-memory lane quarter this warp may read
     const int r = q * 32 + lane;             // accumulator row of this thread
     const int c_base = (ew >> 2) * WARP_COLS;   // this warp's columns of the tile: [c_base, c_base + WARP_COLS)
-    float* sb = (float*)(smem + off_bias(CTAS, EPI, EW)) + ew * WARP_COLS;     // bias of the warp's columns
-    int* sj = (int*)(smem + off_list(CTAS, EPI, EW)) + ew * LIST_WORDS;         // index in U of each of them, or -1
+    float* sb = (float*)(smem + off_bias(CTAS, EPI, EW, MT)) + ew * WARP_COLS;     // bias of the warp's columns
+    int* sj = (int*)(smem + off_list(CTAS, EPI, EW, MT)) + ew * LIST_WORDS;         // index in U of each of them, or -1
     unsigned* sg = (unsigned*)sj + WARP_COLS;                              // one mask of selected columns per 32
-    unsigned char* stage = smem + off_stage(CTAS, EPI, EW) + ew * STAGE_WARP_BYTES;   // this warp's two staging boxes
+    unsigned char* stage = smem + off_stage(CTAS, EPI, EW, MT) + ew * STAGE_WARP_BYTES;   // this warp's two staging boxes
     const unsigned swz64 = (unsigned)((lane >> 1) & 3); // 64-byte swizzle of a staged 64-byte row
     unsigned nbox = 0;                                  // boxes stored so far by this warp (buffer parity)
     const int pstride = a.e.partial_stride ? a.e.partial_stride : a.nsplit;   // split slots per row
@@ -568,7 +597,6 @@ k_umma_gemm(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
       int best_j = -1;
 
       for (int nt = nt0; nt < nt0 + cnt && ok; ++nt, ++it) {
-        const unsigned acc = it & 1u, aph = (it >> 1) & 1u;
         const int n0 = nt * BN;
         // ---- warp-private staging of per-column data (overlaps the MMAs of this tile) ----
         const bool has_bias = a.e.bias != nullptr;        // without a bias the staged zeros are never read
@@ -596,6 +624,9 @@ k_umma_gemm(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
         }
         __syncwarp();
 
+#pragma unroll 1
+        for (int h = 0; h < MT && ok; ++h) {       // MT == 2: sub-tile h of this tile sits in accumulator h
+        const unsigned acc = (MT == 2) ? (unsigned)h : (it & 1u), aph = (MT == 2) ? (it & 1u) : ((it >> 1) & 1u);
         int got = 0;
         if (lane == 0) got = mbar_wait(&st->tmem_full[acc], aph, abort_flag, a.status, 4) ? 1 : 0;
         got = __shfl_sync(0xffffffffu, got, 0);
@@ -702,8 +733,8 @@ k_umma_gemm(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
               }
               if (lane == 0) {
                 if ((EPI == EPI_ACCUM_F32 || EPI == EPI_STORE_OUT) && a.e.accumulate)
-                  tma_reduce_add_2d(&tmC, box, j0 + b * 16, row0_out + q * 32);
-                else tma_store_2d(&tmC, box, j0 + b * 16, row0_out + q * 32);
+                  tma_reduce_add_2d(&tmC, box, j0 + b * 16, row0_out + h * SUB_M + q * 32);
+                else tma_store_2d(&tmC, box, j0 + b * 16, row0_out + h * SUB_M + q * 32);
                 bulk_commit();
               }
               ++nbox;
@@ -777,6 +808,7 @@ k_umma_gemm(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
         tc_fence_before();
         __syncwarp();
         if (lane == 0) { if (CTAS == 2) mbar_arrive_leader(&st->tmem_empty[acc]); else mbar_arrive(&st->tmem_empty[acc]); }
+        }
       }
 
       if (EPI == EPI_LSE_PARTIAL && ok && row_ok)
@@ -849,14 +881,14 @@ int sm_count() {
 
 constexpr int CTAS_DEFAULT = PCTC_TUNE_CTAS;
 
-template <int EPI, int EW>
+template <int EPI, int EW, int MT = 1>
 cudaError_t launch_ew(const CUtensorMap& tmA, const CUtensorMap& tmB, const CUtensorMap& tmC, const UmmaArgs& a,
                       int grid, cudaStream_t stream) {
   static bool configured = false;
   static int max_groups = 0;        // CTA groups (clusters) that can be resident at once
-  constexpr size_t SMEM = smem_bytes(CTAS_DEFAULT, EPI, EW);
+  constexpr size_t SMEM = smem_bytes(CTAS_DEFAULT, EPI, EW, MT);
   static_assert(SMEM <= 227 * 1024, "shared memory budget");
-  auto kern = k_umma_gemm<EPI, CTAS_DEFAULT, EW>;
+  auto kern = k_umma_gemm<EPI, CTAS_DEFAULT, EW, MT>;
   if (!configured) {
     cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)SMEM);
     if (e != cudaSuccess) return e;
@@ -894,6 +926,9 @@ inline int epi_warps_for(int k) {
 template <int EPI>
 cudaError_t launch(const CUtensorMap& tmA, const CUtensorMap& tmB, const CUtensorMap& tmC, const UmmaArgs& a,
                    int grid, cudaStream_t stream) {
+  if constexpr (EPI == EPI_STORE_OUT && CTAS_DEFAULT == 2) {
+    if (a.tile_mt == 2) return launch_ew<EPI, 4, 2>(tmA, tmB, tmC, a, grid, stream);
+  }
   return epi_warps_for(a.k) == 8 ? launch_ew<EPI, 8>(tmA, tmB, tmC, a, grid, stream)
                                  : launch_ew<EPI, 4>(tmA, tmB, tmC, a, grid, stream);
 }
@@ -979,13 +1014,24 @@ cudaError_t umma_gemm(const __nv_bfloat16* A, long long lda, bool a_mn_major,
   a.ksplit_rows = ksplit > 1 ? e.ksplit_rows : 0;
   a.status = status;
   a.e = e;
-  const int m_tiles = (m + BM * CTAS_DEFAULT - 1) / (BM * CTAS_DEFAULT), n_tiles = (n + BN - 1) / BN;
+  const int n_tiles = (n + BN - 1) / BN;
+  const int groups = sm_count() / CTAS_DEFAULT;
+  // 512-row tiles for the dW contraction when its main loop is long (the un-overlapped epilogue is then
+  // a small share) and whole waves of the taller tiles cost no more than whole waves of the usual ones
+  a.tile_mt = 1;
+  if (PCTC_TUNE_MT2 && CTAS_DEFAULT == 2 && e.kind == EPI_STORE_OUT && k > EW_SWITCH_K && m >= 2 * BM * CTAS_DEFAULT) {
+    const long long t1 = (long long)((m + 255) / 256) * n_tiles, t2 = (long long)((m + 511) / 512) * n_tiles;
+    const long long w1 = (t1 + groups - 1) / groups, w2 = 2 * ((t2 + groups - 1) / groups);
+    if (w2 <= w1) a.tile_mt = 2;
+  }
+  const int tile_m = BM * CTAS_DEFAULT * a.tile_mt;
+  const int m_tiles = (m + tile_m - 1) / tile_m;
   const bool walks = e.kind == EPI_LSE_PARTIAL || e.kind == EPI_ARGMAX_PARTIAL;
   {
     // a unit of the walking kernels re-reads its A rows for every column tile: the band's A rows must
     // stay in L2 (and leave room for the streaming B); the other kernels read each panel once per
     // unit, and a near-square patch of tiles per wave touches the fewest panels
-    long long g = PCTC_TUNE_RASTER_G;
+    long long g = PCTC_TUNE_RASTER_G / a.tile_mt;
     if (walks) g = ((long long)PCTC_TUNE_WALK_MB << 20) / ((long long)BM * CTAS_DEFAULT * k * 2);
     if (g < 1) g = 1;
     if (g > m_tiles) g = m_tiles;
@@ -994,7 +1040,6 @@ cudaError_t umma_gemm(const __nv_bfloat16* A, long long lda, bool a_mn_major,
   }
   long long units = (long long)m_tiles * (walks ? e.nsplit : n_tiles) * ksplit;
   if (walks && (e.nsplit < 1 || e.nsplit > n_tiles)) return cudaErrorInvalidValue;
-  const int groups = sm_count() / CTAS_DEFAULT;
   const int grid = (int)(units < groups ? units : groups) * CTAS_DEFAULT;
   switch (e.kind) {
     case EPI_STORE_F32: return launch<EPI_STORE_F32>(tmA, tmB, tmC, a, grid, stream);

@@ -371,7 +371,7 @@ def main():
     # profiles/umma_gemm_c4_speed_of_light.md (default workload and chunk only)
     traffic = None
     if args.config == "c4" and not args.vocab and chunk == 16384 and not args.frozen_head and args.beam == 0 and not args.bias:
-        traffic = dict(bytes_per_step=36.1e9, launches_per_step=31, bytes_per_launch_avg=36.1e9 / 31,
+        traffic = dict(bytes_per_step=33.7e9, launches_per_step=31, bytes_per_launch_avg=33.7e9 / 31,
                        source="ncu dram__bytes_read.sum + dram__bytes_write.sum: the LSE launch and chunks 0-1 of each "
                               "chunk kernel, chunk averages scaled by launches")
 

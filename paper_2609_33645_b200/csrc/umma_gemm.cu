@@ -7,6 +7,11 @@
 // tcgen05.mma.cta_group::2 for both, each keeps the accumulator of its 128 rows in its own tensor
 // memory and runs its own epilogue.  B then crosses L2 -> shared memory once per pair instead of
 // once per CTA, and the freed shared memory deepens the ring to six stages.
+// The dW contraction (template parameter MT = 2) instead puts both accumulators on one 512x256
+// tile: two 128-row sub-tiles of A per CTA and stage, four 48 KB stages, epilogue after the tile.
+// Tiles are handed out in bands of row tiles (decode_unit) so that the CTA pairs running at the
+// same time share operand panels in L2; a contraction with few output tiles can be cut along k
+// (EPI_ACCUM_F32, one accumulator slab per range).
 //
 // One persistent CTA per SM, 192 or 320 threads in three roles:
 //   warp 0      TMA producer: 128-byte-swizzled operand tiles into a 5- or 6-stage ring

@@ -486,3 +486,25 @@ def test_random_wide_shapes(lib, case):
     ref = H.run_oracle(batch, beam=beam if beam > 0 else None, utt_weights=w)
     tol = (2e-3, 1e-2) if dtype == "bf16" else (2e-5, 5e-4)
     H.assert_parity(gpu, ref, batch, tol=tol)
+
+
+def test_tall_dw_tiles_ragged_chunk_and_accumulation(lib):
+    # D = 512, about 2,400 frames, one 16,384-column chunk plus a ragged one: the dW contraction of the
+    # first chunk runs on 512 x 256 tiles (long contraction, 64 such tiles fill one wave); the rows of dW
+    # must match the oracle across the chunk boundary, and a second call with accumulate_dW doubles them
+    import torch
+    cfg = small("c2", V=16384 + 300, D=512, N=6, T_div=1, U_div=2)
+    batch = wl.make_batch(cfg, permute_ids=True)
+    assert batch.M > 2048
+    ref = H.run_oracle(batch)
+    gpu = H.run_gpu(lib, batch, chunk=16384)
+    H.assert_parity(gpu, ref, batch)
+    dev = torch.device("cuda:0")
+    hidden = torch.from_numpy(batch.hidden).to(dev).to(torch.bfloat16)
+    W = torch.from_numpy(batch.W).to(dev).to(torch.bfloat16)
+    targets = torch.from_numpy(batch.targets).to(dev)
+    args = (hidden, W, None, targets, batch.input_lengths, batch.target_lengths, batch.blank)
+    out = lib.pruned_ctc_fwd_bwd(*args, chunk=16384)
+    out = lib.pruned_ctc_fwd_bwd(*args, chunk=16384, accumulate_dW=True, workspace=out["workspace"], out=out)
+    torch.cuda.synchronize()
+    assert H.rel_fro(out["dW"].float().cpu().numpy(), 2.0 * ref["dW"]) <= 1e-2

@@ -382,12 +382,45 @@ __global__ void k_arc_flags(const float* __restrict__ va, const float* __restric
   }
 }
 
+// ---- positions that carry the same label ---------------------------------------------------------
+// The occupancy of a class is the sum over the positions that carry it (Section 3.2).  To add them
+// in a fixed order without atomics, every label position i of an utterance gets a link word: the low
+// 16 bits hold 1 + the next position with the same label (0: none), bit 16 says that an earlier
+// position carries the label too.  The first position of a label then sums its chain in ascending
+// order.  One CTA per utterance; depends on the relabelled targets only.
+constexpr int LINK_HAS_PREV = 1 << 16;
+constexpr int LINK_MAX_U = 2048;               // >= (dp_max_states() - 1) / 2
+
+__global__ void k_repeat_links(const int* __restrict__ rel_all, int stride, const int* __restrict__ U_n,
+                               const int* __restrict__ flags, int* __restrict__ links_all) {
+  __shared__ int s_rel[LINK_MAX_U];
+  __shared__ int s_prev[LINK_MAX_U];
+  const int n = blockIdx.x;
+  if (flags[n] & (4 | 8)) return;              // excluded utterance: its labels may be -1, nobody reads its links
+  const int U = min(U_n[n], LINK_MAX_U);
+  const int* rel = rel_all + (long long)n * stride;
+  int* links = links_all + (long long)n * stride;
+  for (int i = threadIdx.x; i < U; i += blockDim.x) { s_rel[i] = rel[i]; s_prev[i] = 0; }
+  __syncthreads();
+  for (int i = threadIdx.x; i < U; i += blockDim.x) {
+    const int c = s_rel[i];
+    int nxt = 0;
+    for (int j = i + 1; j < U; ++j)
+      if (s_rel[j] == c) { nxt = j + 1; break; }
+    links[i] = nxt;
+    if (nxt) s_prev[nxt - 1] = 1;              // a position has at most one predecessor in its chain
+  }
+  __syncthreads();
+  for (int i = threadIdx.x; i < U; i += blockDim.x)
+    if (s_prev[i]) links[i] |= LINK_HAS_PREV;
+}
+
 // ---- occupancies (Algorithm 1 line 10, G = -gamma): one warp per stacked frame ----
 __global__ void k_gamma(const float* __restrict__ alpha, const float* __restrict__ beta,
                         const float* __restrict__ S, long long ldS, const int* __restrict__ rel_all, int stride,
                         BatchMeta meta, int M, const int* __restrict__ flags,
                         float* __restrict__ gamma, long long ldg, float* __restrict__ roww,
-                        const float* __restrict__ utt_weights) {
+                        const float* __restrict__ utt_weights, const int* __restrict__ links_all) {
   const int m = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
   const int lane = threadIdx.x & 31;
   if (m >= M) return;
@@ -419,12 +452,25 @@ __global__ void k_gamma(const float* __restrict__ alpha, const float* __restrict
   const float inv = 1.f / sum;
   float gb = 0.f;
   float* grow = gamma + (long long)m * ldg;
+  const int* links = links_all + (long long)n * stride;
   for (int s = lane; s < L; s += 32) {
-    const int c = (s & 1) ? rel[(s - 1) >> 1] : 0;
-    const float e = (s & 1) ? Srow[c] * LOG2E : e_blank;
-    const float g = ex2f(a[s] + b[s] - e - mx) * inv;
-    if (s & 1) { if (g != 0.f) atomicAdd(grow + c, g); }
-    else gb += g;
+    if (s & 1) {
+      // label position i: the first position of a label adds up the positions that carry it, in
+      // ascending order (a fixed order: repeated calls give the same bits), and stores the sum
+      const int i = (s - 1) >> 1;
+      int link = links[i];
+      if (link & LINK_HAS_PREV) continue;
+      const int c = rel[i];
+      const float e = Srow[c] * LOG2E;
+      float g = ex2f(a[s] + b[s] - e - mx);
+      for (int j = (link & 0xffff) - 1; j >= 0; j = (links[j] & 0xffff) - 1) {
+        const int s2 = 2 * j + 1;
+        g += ex2f(a[s2] + b[s2] - e - mx);
+      }
+      grow[c] = g * inv;
+    } else {
+      gb += ex2f(a[s] + b[s] - e_blank - mx) * inv;
+    }
   }
 #pragma unroll
   for (int o = 16; o > 0; o >>= 1) gb += __shfl_xor_sync(0xffffffffu, gb, o);
@@ -525,10 +571,12 @@ cudaError_t alignment_dp(const float* S, long long ldS, const int* relabeled, in
     if ((e = dispatch_sweep<MODE_LOG>(a, N, Lmax, stream)) != cudaSuccess) return e;
   }
   if ((e = cudaMemsetAsync(gamma, 0, (size_t)M * ld_gamma * sizeof(float), stream)) != cudaSuccess) return e;
+  k_repeat_links<<<N, 256, 0, stream>>>(relabeled, target_stride, meta.U_n, utt_flags, buf.links);
+  if ((e = cudaGetLastError()) != cudaSuccess) return e;
   const int warps = 8;
   k_gamma<<<(M + warps - 1) / warps, warps * 32, 0, stream>>>(buf.alpha, buf.beta, S, ldS, relabeled,
                                                                 target_stride, meta, M, utt_flags, gamma,
-                                                                ld_gamma, buf.roww, buf.utt_weights);
+                                                                ld_gamma, buf.roww, buf.utt_weights, buf.links);
   return cudaGetLastError();
 }
 

@@ -6,7 +6,6 @@
 #include <cmath>
 #include <cstring>
 #include <mutex>
-#include <vector>
 
 namespace {
 
@@ -25,7 +24,7 @@ struct Plan {
   bool bf16, use_umma, beam;
   // byte offsets into the workspace
   size_t o_status, o_meta_i, o_cell0, o_bitmap, o_wrank, o_vmap, o_U, o_K, o_rel, o_flags, o_X, o_lambda,
-      o_partial, o_WU, o_S, o_G, o_roww, o_alpha, o_beta, o_va, o_vb, o_offa, o_offb, o_best, o_maskf, o_maskb, o_mcell0, o_chunk, o_colpart, o_dHacc;
+      o_partial, o_WU, o_S, o_G, o_roww, o_links, o_alpha, o_beta, o_va, o_vb, o_offa, o_offb, o_best, o_maskf, o_maskb, o_mcell0, o_chunk, o_colpart, o_dHacc;
   size_t total;
   size_t meta_ints;  // T_n[N] | U_n[N] | row0[N+1] | row_utt[M]
 };
@@ -97,6 +96,7 @@ pctc_status_t make_plan(const pctc_problem_t* p, const int32_t* Tn, const int32_
   pl->o_K = take(4);
   pl->o_rel = take((size_t)pl->N * (size_t)(p->target_stride > 0 ? p->target_stride : 1) * 4);
   pl->o_flags = take((size_t)pl->N * 4);
+  pl->o_links = take((size_t)pl->N * (size_t)(p->target_stride > 0 ? p->target_stride : 1) * 4);
   pl->o_X = take((size_t)pl->M * pl->D * pl->elem);
   pl->o_lambda = take((size_t)pl->M * 4);
   pl->o_partial = take((size_t)pl->M * pl->nsplit * 8);
@@ -267,9 +267,8 @@ pctc_status_t pruned_ctc_fwd_bwd(const pctc_problem_t* p, const void* hidden, co
 }  // extern "C"
 
 namespace {
-// Every call uploads per-call index tables from temporary host memory.  A stream capture would record
-// those copies and read that memory again at every replay, long after it is gone, so a capturing
-// stream is refused before anything is enqueued.
+// A call forks onto the library's own auxiliary streams and records its events there; none of that
+// has been arranged for stream capture, so a capturing stream is refused before anything is enqueued.
 bool stream_is_capturing(cudaStream_t stream) {
   cudaStreamCaptureStatus cs = cudaStreamCaptureStatusNone;
   return cudaStreamIsCapturing(stream, &cs) == cudaSuccess && cs != cudaStreamCaptureStatusNone;
@@ -320,34 +319,12 @@ pctc_status_t run_call(const pctc_problem_t* p, const void* hidden, const void* 
 
   PCTC_MARK(PCTC_PHASE_PREP);
   // ---- batch description: lengths, first stacked row, first trellis cell, row -> utterance ----
-  std::vector<int> meta(pl.meta_ints);
-  std::vector<long long> cell0(N), mcell0(N);
-  {
-    int* Tn = meta.data();
-    int* Un = Tn + N;
-    int* row0 = Un + N;
-    int* row_utt = row0 + N + 1;
-    long long cells = 0, mcells = 0;
-    int r = 0;
-    for (int n = 0; n < N; ++n) {
-      Tn[n] = input_lengths[n];
-      Un[n] = target_lengths[n];
-      row0[n] = r;
-      cell0[n] = cells;
-      mcell0[n] = mcells;
-      mcells += (long long)Tn[n] * ((2LL * Un[n] + 1 + 3) / 4 * 4);
-      for (int t = 0; t < Tn[n]; ++t) row_utt[r + t] = n;
-      r += Tn[n];
-      cells += (long long)Tn[n] * (2LL * Un[n] + 1);
-    }
-    row0[N] = r;
-  }
+  // (built on the device from the lengths, which travel as kernel parameters: no copy from
+  // pageable host memory, no wait for the stream)
   int* d_meta = (int*)(ws + pl.o_meta_i);
   long long* d_cell0 = (long long*)(ws + pl.o_cell0);
-  PCTC_CUDA(cudaMemcpyAsync(d_meta, meta.data(), pl.meta_ints * 4, cudaMemcpyHostToDevice, stream));
-  PCTC_CUDA(cudaMemcpyAsync(d_cell0, cell0.data(), (size_t)N * 8, cudaMemcpyHostToDevice, stream));
-  if (pl.beam)
-    PCTC_CUDA(cudaMemcpyAsync(ws + pl.o_mcell0, mcell0.data(), (size_t)N * 8, cudaMemcpyHostToDevice, stream));
+  PCTC_CUDA(batch_meta(input_lengths, target_lengths, N, d_meta, d_meta + N, d_meta + 2 * N, d_cell0,
+                       pl.beam ? (long long*)(ws + pl.o_mcell0) : nullptr, d_meta + 3 * N + 1, stream));
   PCTC_CUDA(cudaMemsetAsync(ws + pl.o_status, 0, 256, stream));
   BatchMeta bm;
   bm.T_n = d_meta;
@@ -377,6 +354,7 @@ pctc_status_t run_call(const pctc_problem_t* p, const void* hidden, const void* 
   dp.beta = (float*)(ws + pl.o_beta);
   dp.roww = (float*)(ws + pl.o_roww);
   dp.utt_weights = p->utt_weights;
+  dp.links = (int*)(ws + pl.o_links);
   if (pl.beam) {
     dp.va = (float*)(ws + pl.o_va);
     dp.vb = (float*)(ws + pl.o_vb);
@@ -778,22 +756,9 @@ pctc_status_t pctc_greedy_decode(const pctc_problem_t* p, const void* hidden, co
   do {                                               \
     if ((call) != cudaSuccess) return PCTC_ERR_CUDA; \
   } while (0)
-  std::vector<int> meta(g.meta_ints);
-  {
-    int* Tn = meta.data();
-    int* row0 = Tn + N;
-    int* row_utt = row0 + N + 1;
-    int r = 0;
-    for (int n = 0; n < N; ++n) {
-      Tn[n] = input_lengths[n];
-      row0[n] = r;
-      for (int t = 0; t < Tn[n]; ++t) row_utt[r + t] = n;
-      r += Tn[n];
-    }
-    row0[N] = r;
-  }
   int* d_meta = (int*)(ws + g.o_meta);
-  PCTC_CUDA(cudaMemcpyAsync(d_meta, meta.data(), g.meta_ints * 4, cudaMemcpyHostToDevice, stream));
+  PCTC_CUDA(batch_meta(input_lengths, nullptr, N, d_meta, nullptr, d_meta + N, nullptr, nullptr, d_meta + 2 * N + 1,
+                       stream));
   PCTC_CUDA(cudaMemsetAsync(ws + g.o_status, 0, 256, stream));
   const int* d_Tn = d_meta;
   const int* d_row0 = d_meta + N;

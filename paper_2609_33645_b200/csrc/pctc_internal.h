@@ -97,6 +97,13 @@ struct BatchMeta {              // device arrays describing the batch
   const int* row_utt;           // [M] utterance of each stacked row
 };
 
+// Batch description from the host length arrays (U_host may be null: no targets).  The lengths
+// travel as kernel parameters, so nothing is copied from pageable host memory and the host does
+// not wait for the stream.  Writes T_n [N], U_n [N], row0 [N+1], cell0 [N] and mcell0 [N] (either
+// may be null), row_utt [M].
+cudaError_t batch_meta(const int* T_host, const int* U_host, int N, int* T_n, int* U_n, int* row0,
+                       long long* cell0, long long* mcell0, int* row_utt, cudaStream_t stream);
+
 // Algorithm 1 lines 2-3.  bitmap: ceil(V/32) words (zeroed here), vmap: [V].
 cudaError_t subset_and_relabel(const int* targets, int target_stride, const int* U_n_dev, int N,
                                long long V, int blank, unsigned* bitmap, int* word_rank,
@@ -145,6 +152,7 @@ struct DpBuffers {
   const long long* mcell0;    // [N] first flag byte of each utterance
   float* roww;         // [M]
   const float* utt_weights;   // [N] upstream gradient of each utterance loss, or null (all 1)
+  int* links;          // [N, target_stride] chains of label positions with equal labels (see k_repeat_links)
 };
 
 // Largest trellis width the DP kernels cover.

@@ -87,6 +87,69 @@ __global__ void k_relabel(const int* __restrict__ targets, int stride, const int
   relabeled[idx] = out;
 }
 
+// --- batch description (Algorithm 1 line 4: which stacked row belongs to which frame) ------------
+// The lengths reach the device as kernel parameters, up to LEN_SLICE utterances per launch, so the
+// host never copies from pageable memory and never waits for the stream; everything derived from
+// them (first stacked row, first trellis cell, first arc-flag byte, row -> utterance) is computed
+// on the device.
+constexpr int LEN_SLICE = 1024;
+struct LengthSlice {
+  int T[LEN_SLICE];
+  int U[LEN_SLICE];
+};
+
+__global__ void k_put_lengths(const __grid_constant__ LengthSlice s, int n0, int cnt, int* __restrict__ T_n,
+                              int* __restrict__ U_n) {
+  for (int i = threadIdx.x; i < cnt; i += blockDim.x) {
+    T_n[n0 + i] = s.T[i];
+    if (U_n) U_n[n0 + i] = s.U[i];
+  }
+}
+
+// One CTA: exclusive prefix sums over the utterances of T_n (rows), T_n (2 U_n + 1) (trellis cells)
+// and T_n roundup4(2 U_n + 1) (arc-flag bytes).  Each thread owns a contiguous run of utterances.
+__global__ void k_batch_offsets(const int* __restrict__ T_n, const int* __restrict__ U_n, int N, int* __restrict__ row0,
+                                long long* __restrict__ cell0, long long* __restrict__ mcell0) {
+  __shared__ long long s_rows[1024], s_cells[1024], s_mcells[1024];
+  const int tid = threadIdx.x, nt = blockDim.x;
+  const int per = (N + nt - 1) / nt;
+  const int n0 = min(N, tid * per), n1 = min(N, n0 + per);
+  long long rows = 0, cells = 0, mcells = 0;
+  for (int n = n0; n < n1; ++n) {
+    const long long T = T_n[n], L = U_n ? 2LL * U_n[n] + 1 : 1;
+    rows += T;
+    cells += T * L;
+    mcells += T * ((L + 3) / 4 * 4);
+  }
+  s_rows[tid] = rows; s_cells[tid] = cells; s_mcells[tid] = mcells;
+  __syncthreads();
+  for (int off = 1; off < nt; off <<= 1) {       // inclusive Hillis-Steele scan of the three sums
+    long long a = 0, b = 0, c = 0;
+    if (tid >= off) { a = s_rows[tid - off]; b = s_cells[tid - off]; c = s_mcells[tid - off]; }
+    __syncthreads();
+    s_rows[tid] += a; s_cells[tid] += b; s_mcells[tid] += c;
+    __syncthreads();
+  }
+  long long r = s_rows[tid] - rows, c = s_cells[tid] - cells, mc = s_mcells[tid] - mcells;
+  for (int n = n0; n < n1; ++n) {
+    const long long T = T_n[n], L = U_n ? 2LL * U_n[n] + 1 : 1;
+    row0[n] = (int)r;
+    if (cell0) cell0[n] = c;
+    if (mcell0) mcell0[n] = mc;
+    r += T;
+    c += T * L;
+    mc += T * ((L + 3) / 4 * 4);
+  }
+  if (tid == nt - 1) row0[N] = (int)s_rows[nt - 1];
+}
+
+__global__ void k_row_utt(const int* __restrict__ T_n, const int* __restrict__ row0, int N, int* __restrict__ row_utt) {
+  for (int n = blockIdx.x; n < N; n += gridDim.x) {
+    const int r0 = row0[n], T = T_n[n];
+    for (int t = threadIdx.x; t < T; t += blockDim.x) row_utt[r0 + t] = n;
+  }
+}
+
 // --- row copies ---------------------------------------------------------------------------------
 __device__ __forceinline__ void copy_row(const char* __restrict__ src, char* __restrict__ dst, size_t bytes) {
   if ((((size_t)src | (size_t)dst | bytes) & 15) == 0) {
@@ -212,8 +275,13 @@ __global__ void k_colpart_sums(const float* __restrict__ colpart, long long ld, 
 __global__ void k_lse_combine(const float2* __restrict__ partial, int nsplit, int M, float* __restrict__ lambda) {
   int i = blockIdx.x * blockDim.x + threadIdx.x;
   if (i >= M) return;
+  // a slot nothing was written to holds (anything, 0): it must not take part in the maximum either,
+  // or a frame whose every logit lies far below the empty slot's value would lose its whole sum
   float mx = -CUDART_INF_F;
-  for (int s = 0; s < nsplit; ++s) mx = fmaxf(mx, partial[(size_t)i * nsplit + s].x);
+  for (int s = 0; s < nsplit; ++s) {
+    const float2 p = partial[(size_t)i * nsplit + s];
+    if (!(p.y <= 0.f)) mx = fmaxf(mx, p.x);
+  }
   float sum = 0.f;
   for (int s = 0; s < nsplit; ++s) {
     float2 p = partial[(size_t)i * nsplit + s];
@@ -291,6 +359,22 @@ cudaError_t subset_and_relabel(const int* targets, int target_stride, const int*
                                         status);
   if (total > 0)
     k_relabel<<<blocks, 256, 0, stream>>>(targets, target_stride, U_n_dev, N, V, blank, vmap, relabeled);
+  return cudaGetLastError();
+}
+
+cudaError_t batch_meta(const int* T_host, const int* U_host, int N, int* T_n, int* U_n, int* row0,
+                       long long* cell0, long long* mcell0, int* row_utt, cudaStream_t stream) {
+  LengthSlice s;
+  for (int n0 = 0; n0 < N; n0 += LEN_SLICE) {
+    const int cnt = (N - n0 < LEN_SLICE) ? (N - n0) : LEN_SLICE;
+    for (int i = 0; i < cnt; ++i) {
+      s.T[i] = T_host[n0 + i];
+      s.U[i] = U_host ? U_host[n0 + i] : 0;
+    }
+    k_put_lengths<<<1, 256, 0, stream>>>(s, n0, cnt, T_n, U_host ? U_n : nullptr);
+  }
+  k_batch_offsets<<<1, 1024, 0, stream>>>(T_n, U_host ? U_n : nullptr, N, row0, cell0, mcell0);
+  k_row_utt<<<(N < 1024 ? N : 1024), 256, 0, stream>>>(T_n, row0, N, row_utt);
   return cudaGetLastError();
 }
 

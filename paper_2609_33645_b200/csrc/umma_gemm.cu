@@ -28,11 +28,14 @@
 //
 // Every mbarrier wait is bounded: after about two seconds a wait stores a code
 // in the caller's status word, raises a CTA-wide abort flag and every role
-// leaves its loop; the CTA then drains its own copies, frees its tensor memory
-// and returns.
+// leaves its loop; the CTA then waits (bounded, whatever the abort flag says)
+// for the copies and MMAs it has issued, lingers a millisecond for what its
+// peer may still have in flight, frees its tensor memory and returns.
 #include "pctc_internal.h"
 
 #include <cuda.h>
+
+#include <atomic>
 #include <math_constants.h>
 
 namespace pctc {
@@ -75,7 +78,12 @@ constexpr int b_stage_bytes(int ctas) { return (BN / ctas) * BK * 2; }   // each
 constexpr int num_threads(int ew) { return 64 + ew * 32; }
 constexpr int TMEM_COLS = 512;
 constexpr int MN_GROUP_BYTES = 64 * BK * 2;          // one 64-wide MN group of an MN-major tile
-constexpr long long WAIT_LIMIT_CYCLES = 4000000000LL;
+#ifndef PCTC_WAIT_LIMIT_CYCLES
+#define PCTC_WAIT_LIMIT_CYCLES 4000000000LL   // about two seconds; a test build shortens it so that a wait runs out
+#endif
+constexpr long long WAIT_LIMIT_CYCLES = PCTC_WAIT_LIMIT_CYCLES;
+constexpr long long DRAIN_LIMIT_CYCLES = 200000000LL;   // the waits of an aborting CTA for its own copies and MMAs
+constexpr long long ABORT_LINGER_CYCLES = 2000000LL;    // an aborting CTA stays this long before it leaves (see the kernel's end)
 constexpr float LOG2E = 1.4426950408889634f;
 constexpr float LN2 = 0.6931471805599453f;
 
@@ -180,6 +188,16 @@ __device__ __forceinline__ bool mbar_wait(unsigned long long* bar, unsigned pari
         return false;
       }
     }
+  }
+}
+// The waits of the drain: for copies and MMAs this CTA has already issued.  They run when the CTA is
+// aborting too, so they ignore the abort flag and keep only their own limit.
+__device__ __forceinline__ bool mbar_wait_drain(unsigned long long* bar, unsigned parity) {
+  if (mbar_try(bar, parity)) return true;
+  const long long t0 = clock64();
+  for (unsigned it = 1;; ++it) {
+    if (mbar_try(bar, parity)) return true;
+    if ((it & 255u) == 0u && clock64() - t0 > DRAIN_LIMIT_CYCLES) return false;
   }
 }
 
@@ -488,7 +506,7 @@ k_umma_gemm(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
       if (rank == 0) {
         const unsigned issued = g;
         for (unsigned j = (issued > STAGES ? issued - STAGES : 0); j < issued; ++j)
-          mbar_wait(&st->full[j % STAGES], (j / STAGES) & 1u, abort_flag, nullptr, 0, 200000000LL);
+          mbar_wait_drain(&st->full[j % STAGES], (j / STAGES) & 1u);
       }
     }
   } else if (warp == 1) {
@@ -543,7 +561,7 @@ k_umma_gemm(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
       }
       // all MMAs issued by this thread have completed before tensor memory is freed
       if (CTAS == 2) tc_commit_pair_local(&st->done); else tc_commit(&st->done);
-      mbar_wait(&st->done, 0, abort_flag, nullptr, 0, 200000000LL);
+      mbar_wait_drain(&st->done, 0);
     }
   } else {
     // ===================== epilogue warps =====================
@@ -828,6 +846,15 @@ k_umma_gemm(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
 
   tc_fence_before();
   __syncthreads();
+  if (*abort_flag) {
+    // A wait gave up somewhere in this CTA.  The leader has waited above for the copies of the stages
+    // it issued itself (its barriers count the peer's bytes of those stages too) and for its MMAs.
+    // What that cannot cover is a copy the peer issued for a stage the leader never reached: such a
+    // copy lands within microseconds, so both CTAs simply stay for a fixed while before they leave.
+    const long long t0 = clock64();
+    while (clock64() - t0 < ABORT_LINGER_CYCLES) { }
+    __syncthreads();
+  }
   if (CTAS == 2) cluster_sync_all();     // no CTA of a pair leaves while the other may still signal it
   if (warp == 1) {
     tc_fence_after();
@@ -874,13 +901,26 @@ bool make_map(CUtensorMap* map, const void* base, unsigned long long inner, unsi
             CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
+// Per-device state: a process may drive several GPUs, and both the shared-memory opt-in of a kernel
+// and the SM count belong to one device.  Entries are filled on first use; the values are the same
+// whichever thread fills them.
+constexpr int MAX_DEVICES = 64;
+int current_device() {
+  int dev = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= MAX_DEVICES) return 0;
+  return dev;
+}
+
 int sm_count() {
-  static int n = [] {
-    int dev = 0, v = 0;
-    if (cudaGetDevice(&dev) != cudaSuccess) return 148;
-    if (cudaDeviceGetAttribute(&v, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || v <= 0) return 148;
-    return v;
-  }();
+  static std::atomic<int> table[MAX_DEVICES];
+  const int dev = current_device();
+  int n = table[dev].load(std::memory_order_relaxed);
+  if (n == 0) {
+    int v = 0;
+    if (cudaDeviceGetAttribute(&v, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || v <= 0) v = 148;
+    n = v;
+    table[dev].store(n, std::memory_order_relaxed);
+  }
   return n;
 }
 
@@ -889,15 +929,17 @@ constexpr int CTAS_DEFAULT = PCTC_TUNE_CTAS;
 template <int EPI, int EW, int MT = 1>
 cudaError_t launch_ew(const CUtensorMap& tmA, const CUtensorMap& tmB, const CUtensorMap& tmC, const UmmaArgs& a,
                       int grid, cudaStream_t stream) {
-  static bool configured = false;
-  static int max_groups = 0;        // CTA groups (clusters) that can be resident at once
+  // per device: 0 = this kernel has not been configured there yet, else the number of CTA groups
+  // (clusters) that can be resident at once
+  static std::atomic<int> groups_on[MAX_DEVICES];
   constexpr size_t SMEM = smem_bytes(CTAS_DEFAULT, EPI, EW, MT);
   static_assert(SMEM <= 227 * 1024, "shared memory budget");
   auto kern = k_umma_gemm<EPI, CTAS_DEFAULT, EW, MT>;
-  if (!configured) {
+  const int dev = current_device();
+  int max_groups = groups_on[dev].load(std::memory_order_acquire);
+  if (max_groups == 0) {
     cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)SMEM);
     if (e != cudaSuccess) return e;
-    configured = true;
   }
   cudaLaunchAttribute attr[1];
   attr[0].id = cudaLaunchAttributeClusterDimension;
@@ -915,6 +957,7 @@ cudaError_t launch_ew(const CUtensorMap& tmA, const CUtensorMap& tmB, const CUte
     int n = 0;
     if (cudaOccupancyMaxActiveClusters(&n, kern, &cfg) != cudaSuccess || n <= 0) n = sm_count() / CTAS_DEFAULT;
     max_groups = n;
+    groups_on[dev].store(n, std::memory_order_release);
   }
   if (grid > max_groups * CTAS_DEFAULT) grid = max_groups * CTAS_DEFAULT;
   cfg.gridDim = dim3((unsigned)grid);

@@ -29,7 +29,16 @@ def test_chunk_buffer_beyond_2_to_31_elements(lib):
     check_sampled_parity(lib, cfg)
 
 
-def check_sampled_parity(lib, cfg):
+@pytest.mark.parametrize("beam", [8.0, 16.0])
+def test_c5_full_size_gradients_under_a_beam(lib, beam):
+    """Section 3.3 at full size (T up to 3000, about 1,200 trellis positions): the gradients p - gamma^beta
+    against the oracle AT THE SAME BEAM.  At these beams gamma^beta differs strongly from the exact
+    occupancy (Appendix B.3: most of the exact lattice's mass is discarded), so this is a check of the
+    arc-masked sweeps, not of the unpruned ones."""
+    check_sampled_parity(lib, wl.CONFIGS["c5"], beam=beam, n_dH=1)
+
+
+def check_sampled_parity(lib, cfg, beam=0.0, n_dH=2):
     import torch
     batch = wl.make_batch(cfg)
     assert batch.M * min(cfg.V, 8192) > 2 ** 31 or cfg.name != "bigM"
@@ -38,7 +47,7 @@ def check_sampled_parity(lib, cfg):
     W = torch.from_numpy(batch.W).to(dev).to(torch.bfloat16)
     targets = torch.from_numpy(batch.targets).to(dev)
     res = lib.pruned_ctc_fwd_bwd(hidden, W, None, targets, batch.input_lengths, batch.target_lengths, batch.blank,
-                                 check_status=True)
+                                 beam=beam, check_status=True)
     torch.cuda.synchronize()
 
     # ---- identities that hold at any size (computed from the GPU outputs alone) ----
@@ -73,9 +82,9 @@ def check_sampled_parity(lib, cfg):
     del res
     torch.cuda.empty_cache()
     order = np.argsort(batch.input_lengths)
-    dH_for = [int(order[0]), int(order[1])]
+    dH_for = [int(order[k]) for k in range(n_dH)]
     t0 = time.time()
-    ref = H.run_oracle(batch, dW_rows=rows, dH_for=dH_for)
+    ref = H.run_oracle(batch, beam=beam if beam > 0 else None, dW_rows=rows, dH_for=dH_for)
     print(f"oracle (sampled) took {time.time() - t0:.1f} s")
     np.testing.assert_array_equal(flags_gpu, ref["flags"])
     assert np.all(np.abs(loss - ref["loss"]) <= 2e-3 * np.abs(ref["loss"])), (loss, ref["loss"])

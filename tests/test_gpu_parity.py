@@ -152,6 +152,26 @@ def test_two_calls_are_bitwise_identical_and_workspace_is_reusable(lib):
     torch.cuda.synchronize()
 
 
+def test_repeated_labels_pool_in_a_fixed_order(lib):
+    """The occupancy of a class sums over the positions that carry it (Section 3.2).  One utterance
+    whose labels are all the same token, one that cycles through three tokens (many scattered
+    repeats), one ordinary: parity with the oracle, and three calls must agree bit for bit."""
+    cfg = small("c2", V=2048, D=64, N=3, T_div=2, U_div=1)
+    batch = wl.make_batch(cfg, permute_ids=True)
+    U0 = min(int(batch.target_lengths[0]), int(batch.input_lengths[0]) // 2 - 1)
+    batch.target_lengths[0] = U0
+    batch.targets[0, :U0] = 777                                   # T >= 2 U - 1 keeps it feasible
+    U1 = int(batch.target_lengths[1])
+    batch.targets[1, :U1] = np.array([5, 1500, 31])[np.arange(U1) % 3]
+    runs = [H.run_gpu(lib, batch) for _ in range(3)]
+    ref = H.run_oracle(batch)
+    assert not ref["flags"].any()
+    H.assert_parity(runs[0], ref, batch)
+    for other in runs[1:]:
+        for k in ("loss", "dH", "dW"):
+            np.testing.assert_array_equal(runs[0][k], other[k])
+
+
 @pytest.mark.parametrize("path", [SIMT, AUTO])
 def test_frozen_head_utterance_weights_and_accumulation(lib, path):
     import torch
@@ -322,10 +342,15 @@ def test_zero_and_negative_utterance_weights(lib, path):
     assert np.all(gpu["dH"][0] == 0.0) and gpu["flags"][0] == 0 and gpu["loss"][0] > 0
 
 
-@pytest.mark.parametrize("V,D", [(8192 + 384, 256), (4 * 4096 + 1000, 64)])   # one upload / four segments of W
-def test_host_buffer_entry_point_matches_device_entry_point(lib, V, D):
+# one upload / four segments of W; and a strongly negative bias: every logit of a frame then lies far
+# below zero, so the normaliser must not be anchored at the value an unused partial slot holds
+@pytest.mark.parametrize("V,D,bias_shift", [(8192 + 384, 256, 0.0), (4 * 4096 + 1000, 64, 0.0),
+                                            (4 * 4096 + 1000, 64, -200.0)])
+def test_host_buffer_entry_point_matches_device_entry_point(lib, V, D, bias_shift):
     import torch
     batch = wl.make_batch(small("c3", V=V, D=D, N=4, T_div=4, U_div=2), with_bias=True, permute_ids=True)
+    if bias_shift:
+        batch.bias = wl.round_to_bf16(batch.bias + np.float32(bias_shift))
     dev_out = H.run_gpu(lib, batch, chunk=2048)
     tdt = torch.bfloat16
     hid = torch.from_numpy(batch.hidden).to(tdt).pin_memory()
@@ -416,6 +441,46 @@ def test_bf16_shapes_the_tensor_core_path_does_not_cover_fall_to_the_fma_kernels
     batch = wl.make_batch(cfg, with_bias=True, permute_ids=True)
     gpu = H.run_gpu(lib, batch, gemm_path=AUTO)
     H.assert_parity(gpu, H.run_oracle(batch), batch)
+
+
+def test_call_returns_to_the_host_while_the_stream_is_still_busy(lib):
+    """No hidden synchronisation: with tens of milliseconds of earlier work still queued on the stream,
+    a call on the paper-grid shape with the most frames (640 utterances of 100 frames, vocabulary
+    reduced) must hand control back to the host at once, and give the same bits as an idle-stream call."""
+    import time
+    import torch
+    cfg = wl.reduced(wl.CONFIGS["g64k"], V=4096, D=128, name="g64k-small")
+    batch = wl.make_batch(cfg)
+    assert batch.M == 64000
+    dev = torch.device("cuda:0")
+    hidden = torch.from_numpy(batch.hidden).to(dev).to(torch.bfloat16)
+    W = torch.from_numpy(batch.W).to(dev).to(torch.bfloat16)
+    targets = torch.from_numpy(batch.targets).to(dev)
+    args = (hidden, W, None, targets, batch.input_lengths, batch.target_lengths, batch.blank)
+    first = lib.pruned_ctc_fwd_bwd(*args, check_status=True)
+    torch.cuda.synchronize()
+    want = {k: first[k].clone() for k in ("loss", "dH", "dW", "subset", "relabeled", "flags")}
+    a = torch.randn(8192, 8192, device=dev, dtype=torch.bfloat16)
+    c = torch.empty_like(a)
+    torch.matmul(a, a, out=c)
+    torch.cuda.synchronize()
+    busy = torch.cuda.Event()
+    t_busy = time.perf_counter()
+    for _ in range(120):                               # about 0.1 s of queued work (0.7 ms or more each)
+        torch.matmul(a, a, out=c)
+    busy.record()
+    t0 = time.perf_counter()
+    res = lib.pruned_ctc_fwd_bwd(*args, workspace=first["workspace"], out=first)
+    t1 = time.perf_counter()
+    still_busy = not busy.query()
+    torch.cuda.synchronize()
+    t_done = time.perf_counter()
+    print(f"host time of the call {1e3 * (t1 - t0):.2f} ms; queued work took {1e3 * (t_done - t_busy):.1f} ms")
+    assert still_busy, "the earlier work had finished before the call returned: the call waited for the stream"
+    assert t1 - t0 < 0.010
+    for k, v in want.items():
+        assert torch.equal(res[k], v), k
+    assert lib.workspace_status(res["workspace"]) == 0
 
 
 def test_capturing_stream_is_refused_before_anything_is_enqueued(lib):

@@ -12,10 +12,12 @@
  * the call's later steps).  Every buffer is owned by the caller; the library
  * keeps no pointers between calls and, except where an entry point says
  * otherwise, allocates no device memory.  Calls on one device must not be issued
- * from several host threads at once.  pruned_ctc_fwd_bwd, its traced and host-buffer
- * forms and pctc_greedy_decode upload small per-call index tables from temporary host
- * memory and therefore cannot be part of a CUDA graph: on a stream that is being
- * captured they return PCTC_ERR_UNSUPPORTED before enqueuing anything.
+ * from several host threads at once; several devices may be driven from one process.
+ * No call waits for the stream or for the device: the host length arrays travel as kernel
+ * parameters and every table derived from them is built on the device.
+ * pruned_ctc_fwd_bwd, its traced and host-buffer forms and pctc_greedy_decode fork onto
+ * the library's auxiliary streams, which has not been arranged for stream capture: on a
+ * stream that is being captured they return PCTC_ERR_UNSUPPORTED before enqueuing anything.
  * Functions return a status code and never throw or abort.
  */
 #ifndef PRUNEDCTC_H_
@@ -309,10 +311,20 @@ pctc_status_t pctc_subset_relabel_noalloc(const int32_t* targets, const int32_t*
 /*
  * Device-side status word.  Every wait inside a kernel (on an mbarrier) is
  * bounded; a wait that gives up stores a non-zero code and the kernel returns
- * cleanly instead of hanging.  pruned_ctc_fwd_bwd keeps the word at the start of
- * its workspace (zeroed by each call); this function copies it to the host after
- * synchronising `stream`.  0 means no wait gave up.  PCTC_ERR_TIMEOUT is returned
- * when it is non-zero.
+ * cleanly instead of hanging: it waits (again bounded) for the copies and tensor-core
+ * operations it has in flight, frees its tensor memory and leaves.  pruned_ctc_fwd_bwd
+ * keeps the word at the start of its workspace (zeroed by each call); this function
+ * copies it to the host after synchronising `stream`.  Codes (the first event wins):
+ *   0            nothing to report                                     -> PCTC_OK
+ *   1 .. 4       a bounded wait gave up (1 producer waiting for a free stage, 2 MMA issuer
+ *                waiting for a drained accumulator, 3 MMA issuer waiting for operands,
+ *                4 epilogue waiting for an accumulator)                 -> PCTC_ERR_TIMEOUT
+ *   0x100        the batch has more selected classes than problem.max_K -> PCTC_ERR_INVALID_ARG
+ *   0x201 ..     only in a library built with -DPCTC_DEBUG_BOUNDS: an index that a kernel was
+ *                about to gather or scatter through was out of range (0x200 + checking site);
+ *                the access was skipped                                 -> PCTC_ERR_INVALID_ARG
+ * `workspace` may be any device word that received a status, e.g. the device_status of
+ * pctc_gemm_bf16.
  */
 pctc_status_t pctc_workspace_status(const void* workspace, void* stream, int32_t* status_host);
 

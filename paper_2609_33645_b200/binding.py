@@ -90,7 +90,19 @@ def load() -> ctypes.CDLL:
     if not os.path.exists(LIB_PATH):
         raise RuntimeError(f"{LIB_PATH} is missing: run paper_2609_33645_b200.build.build() first; "
                            "there is no fallback implementation")
-    lib = ctypes.CDLL(LIB_PATH)
+    _lib = _configure(ctypes.CDLL(LIB_PATH))
+    return _lib
+
+
+def load_variant(path: str) -> ctypes.CDLL:
+    """A test variant of the library (build.build_variant), loaded beside the regular one: call its
+    entry points directly, e.g. ``gemm_bf16(..., lib=load_variant(path))``."""
+    if not os.path.exists(path):
+        raise RuntimeError(f"{path} is missing: run paper_2609_33645_b200.build.build_variant() first")
+    return _configure(ctypes.CDLL(path))
+
+
+def _configure(lib: ctypes.CDLL) -> ctypes.CDLL:
     vp, i32p = ctypes.c_void_p, ctypes.POINTER(ctypes.c_int32)
     lib.pctc_workspace_bytes.restype = ctypes.c_int
     lib.pctc_workspace_bytes.argtypes = [ctypes.POINTER(Problem), i32p, i32p, ctypes.POINTER(ctypes.c_size_t)]
@@ -120,7 +132,6 @@ def load() -> ctypes.CDLL:
     lib.pctc_workspace_status.argtypes = [vp, vp, i32p]
     lib.pctc_status_string.restype = ctypes.c_char_p
     lib.pctc_status_string.argtypes = [ctypes.c_int]
-    _lib = lib
     return lib
 
 
@@ -169,7 +180,7 @@ def _dptr(t) -> Optional[int]:
 def pruned_ctc_fwd_bwd(hidden, W, bias, targets, input_lengths, target_lengths, blank_id, *, beam=0.0,
                        chunk=0, gemm_path=GEMM_AUTO, workspace=None, out=None, check_status=False,
                        trace: Optional[Trace] = None, skip_dW=False, accumulate_dW=False, utt_weights=None,
-                       max_K=0, forward_only=False):
+                       max_K=0, forward_only=False, lib_handle=None):
     """Algorithm 1 on CUDA tensors.
 
     hidden [N,T,D], W [V,D], bias [V] or None (bf16 or fp32, same dtype), targets
@@ -180,10 +191,11 @@ def pruned_ctc_fwd_bwd(hidden, W, bias, targets, input_lengths, target_lengths, 
     preallocated tensors from an earlier call with the same shapes.
     skip_dW: frozen head, dW is None.  accumulate_dW: add into out["dW"] / out["dbias"].
     utt_weights: fp32 CUDA tensor [N] of upstream gradients of the utterance losses.
+    lib_handle: a test variant of the library from load_variant() instead of the regular one.
     """
     import torch
 
-    lib = load()
+    lib = lib_handle or load()
     if not (hidden.is_cuda and W.is_cuda and hidden.is_contiguous() and W.is_contiguous()):
         raise ValueError("hidden and W must be contiguous CUDA tensors")
     if hidden.dtype != W.dtype or hidden.dtype not in (torch.bfloat16, torch.float32):
@@ -201,7 +213,7 @@ def pruned_ctc_fwd_bwd(hidden, W, bias, targets, input_lengths, target_lengths, 
         raise ValueError("utt_weights must be an fp32 CUDA tensor of shape [N]")
     prob = make_problem(N, T, D, V, dt, blank_id, beam, chunk, stride, gemm_path, skip_dW, accumulate_dW,
                         None if utt_weights is None else utt_weights.data_ptr(), max_K, forward_only)
-    need = workspace_bytes(prob, il, tl)
+    need = workspace_bytes(prob, il, tl)          # host-only arithmetic, the same in every variant
     dev = hidden.device
     if workspace is None or workspace.numel() < need:
         workspace = torch.empty(need, dtype=torch.uint8, device=dev)
@@ -239,20 +251,21 @@ def pruned_ctc_fwd_bwd(hidden, W, bias, targets, input_lengths, target_lengths, 
     if st != 0:
         raise PctcError(st, "pruned_ctc_fwd_bwd")
     if check_status:
-        code = workspace_status(workspace)
+        code = workspace_status(workspace, lib_handle=lib)
         if code != 0:
-            raise PctcError(6, f"device status word {code}")
+            raise PctcError(6 if code < 0x100 else 1, f"device status word {code:#x}")
     return res
 
 
-def workspace_status(workspace) -> int:
-    """Synchronise the current stream and return the device status word (0: no wait gave up)."""
+def workspace_status(workspace, lib_handle=None) -> int:
+    """Synchronise the current stream and return the device status word: 0 nothing to report, 1-4 a
+    bounded wait gave up, 0x100 more selected classes than max_K, 0x201.. (debug build) a bad index."""
     import torch
 
     host = ctypes.c_int32(0)
     stream = ctypes.c_void_p(torch.cuda.current_stream(workspace.device).cuda_stream)
-    st = load().pctc_workspace_status(_dptr(workspace), stream, ctypes.byref(host))
-    if st not in (0, 6):
+    st = (lib_handle or load()).pctc_workspace_status(_dptr(workspace), stream, ctypes.byref(host))
+    if st not in (0, 1, 6):
         raise PctcError(st, "pctc_workspace_status")
     return int(host.value)
 

@@ -3,6 +3,7 @@
 ``build()`` runs nvcc for sm_100a on every ``csrc/*.cu`` (in parallel), links
 ``libprunedctc.so`` next to this file and returns its path.  Objects are cached
 under ``build/`` and rebuilt only when a source or header is newer.
+``build_variant(tag)`` builds a test variant of the same sources (see VARIANTS).
 """
 
 from __future__ import annotations
@@ -48,15 +49,37 @@ def headers():
     return hs
 
 
-def build(verbose: bool = False, extra_flags=()) -> str:
-    os.makedirs(OBJ_DIR, exist_ok=True)
+# Variants of the library for tests: same sources, extra compile-time definitions, a file of their own.
+#   shortwait  every bounded device wait gives up after a few thousand cycles, so that an ordinary
+#              call exercises the give-up path (status word, drain, clean return)
+#   bounds     every index that a kernel gathers or scatters through (selected classes, relabelled
+#              targets, row tables) is range-checked first; a bad one is recorded in the status word
+#              and the access is skipped
+VARIANTS = {
+    "shortwait": ("-DPCTC_WAIT_LIMIT_CYCLES=3000LL", "-DPCTC_WAIT_POLL_MASK=0u"),
+    "bounds": ("-DPCTC_DEBUG_BOUNDS=1",),
+}
+
+
+def variant_path(tag: str) -> str:
+    return os.path.join(HERE, f"libprunedctc_{tag}.so")
+
+
+def build_variant(tag: str, verbose: bool = False) -> str:
+    return build(verbose=verbose, extra_flags=VARIANTS[tag], tag=tag)
+
+
+def build(verbose: bool = False, extra_flags=(), tag: str = "") -> str:
+    obj_dir = OBJ_DIR + ("_" + tag if tag else "")
+    lib_path = variant_path(tag) if tag else LIB_PATH
+    os.makedirs(obj_dir, exist_ok=True)
     nvcc = _nvcc()
     srcs = sources()
     hdr_time = _newest(headers() + [os.path.abspath(__file__)])
     jobs = []
     objs = []
     for src in srcs:
-        obj = os.path.join(OBJ_DIR, os.path.basename(src)[:-3] + ".o")
+        obj = os.path.join(obj_dir, os.path.basename(src)[:-3] + ".o")
         objs.append(obj)
         if os.path.exists(obj) and os.path.getmtime(obj) >= max(os.path.getmtime(src), hdr_time):
             continue
@@ -77,9 +100,9 @@ def build(verbose: bool = False, extra_flags=()) -> str:
             for out in ex.map(run, jobs):
                 if verbose and out:
                     sys.stderr.write(out)
-    if jobs or not os.path.exists(LIB_PATH) or os.path.getmtime(LIB_PATH) < _newest(objs):
-        run([nvcc, "-shared", "-o", LIB_PATH, *objs])   # static cudart (nvcc default)
-    return LIB_PATH
+    if jobs or not os.path.exists(lib_path) or os.path.getmtime(lib_path) < _newest(objs):
+        run([nvcc, "-shared", "-o", lib_path, *objs])   # static cudart (nvcc default)
+    return lib_path
 
 
 if __name__ == "__main__":

@@ -51,6 +51,7 @@ struct SweepArgs {
   double* off_a; double* off_b;            // MODE_MAX: per-frame offsets of the rows written
   double* best;                            // [N] best alignment score (base 2)
   float* loss; int* flags;
+  int* status;                             // status word (index checks of the debug build)
 };
 
 __device__ __forceinline__ void cp_async4(void* smem_dst, const void* gsrc) {
@@ -103,6 +104,15 @@ __global__ void __launch_bounds__(W * 32) k_ctc_sweep(SweepArgs a) {
     if (cnt) atomicAdd(&s_rep, cnt);
   }
   __syncthreads();
+  if (kCheckBounds) {                                              // every label indexes a column of Z_U
+    __shared__ int s_badidx;
+    if (tid == 0) s_badidx = 0;
+    __syncthreads();
+    for (int i = tid; i < U; i += NTH)
+      if (!index_ok(rel[i], 0, a.ldS, a.status, 5)) s_badidx = 1;
+    __syncthreads();
+    if (s_badidx) return;
+  }
   if (T < U + s_rep) {                                             // no alignment exists (Appendix B.1)
     if (dir == 0 && tid == 0 && MODE != MODE_MAX) { atomicOr(&a.flags[n], 1); a.loss[n] = 0.f; }
     return;
@@ -343,8 +353,10 @@ __global__ void k_arc_flags(const float* __restrict__ va, const float* __restric
                             unsigned char* __restrict__ mask_b) {
   const int m = blockIdx.x;
   const int n = meta.row_utt[m];
+  if (!index_ok(n, 0, meta.N, meta.status, 6)) return;
   if (flags[n] != 0) return;
   const int r0 = meta.row0[n], t = m - r0, T = meta.T_n[n];
+  if (!index_ok(t, 0, T, meta.status, 6)) return;
   const int L = 2 * meta.U_n[n] + 1, Lp4 = (L + 3) & ~3;
   const double best = best_all[n];
   const float* a_prev = va + meta.cell0[n] + (long long)(t - 1) * L;   // read for t >= 1 only
@@ -425,9 +437,21 @@ __global__ void k_gamma(const float* __restrict__ alpha, const float* __restrict
   const int lane = threadIdx.x & 31;
   if (m >= M) return;
   const int n = meta.row_utt[m];
+  if (!index_ok(n, 0, meta.N, meta.status, 7)) return;
   if (flags[n] != 0) { if (lane == 0) roww[m] = 0.f; return; }
   const int t = m - meta.row0[n];
   const int U = meta.U_n[n], L = 2 * U + 1;
+  if (!index_ok(t, 0, meta.T_n[n], meta.status, 7)) return;
+  if (kCheckBounds) {                          // labels index the row of Z_U and of gamma; links stay inside the utterance
+    bool bad = false;
+    for (int i = lane; i < U; i += 32) {
+      const int nxt = (links_all[(long long)n * stride + i] & 0xffff) - 1;
+      if (!index_ok(rel_all[(long long)n * stride + i], 0, ldg < ldS ? ldg : ldS, meta.status, 7) ||
+          !index_ok(nxt, -1, U, meta.status, 7) || (nxt >= 0 && nxt <= i && !index_ok(-1, 0, 1, meta.status, 7)))
+        bad = true;
+    }
+    if (__any_sync(0xffffffffu, bad)) return;
+  }
   const int* rel = rel_all + (long long)n * stride;
   const float* a = alpha + meta.cell0[n] + (long long)t * L;
   const float* b = beta + meta.cell0[n] + (long long)t * L;
@@ -484,6 +508,7 @@ __global__ void k_finalize_loss(const float* __restrict__ lambda, BatchMeta meta
   __shared__ int s_bad;
   const int n = blockIdx.x, tid = threadIdx.x;
   const int r0 = meta.row0[n], T = meta.T_n[n];
+  if (!index_ok((long long)r0 + T, 1, (long long)meta.M + 1, meta.status, 8)) return;
   if (flags[n] != 0) return;                 // excluded: loss is already 0, row weights already 0
   double acc = 0.0;
   for (int t = tid; t < T; t += blockDim.x) acc += (double)lambda[r0 + t];
@@ -553,7 +578,7 @@ cudaError_t alignment_dp(const float* S, long long ldS, const int* relabeled, in
   SweepArgs a{};
   a.S = S; a.ldS = ldS; a.rel = relabeled; a.stride = target_stride;
   a.T_n = meta.T_n; a.U_n = meta.U_n; a.row0 = meta.row0; a.cell0 = meta.cell0; a.mcell0 = buf.mcell0;
-  a.loss = loss; a.flags = utt_flags;
+  a.loss = loss; a.flags = utt_flags; a.status = meta.status;
   a.off_a = buf.off_a; a.off_b = buf.off_b; a.best = buf.best;
   const bool use_beam = (beam > 0.f) && isfinite(beam);
   cudaError_t e;

@@ -177,9 +177,11 @@ struct GemmCall {
   int m, n, k;
 };
 
-cudaError_t run_gemm(bool use_umma, bool bf16, const GemmCall& c, const Epilogue& e, int* status,
+cudaError_t run_gemm(bool use_umma, bool bf16, const GemmCall& c, const Epilogue& e_in, int* status,
                      cudaStream_t stream) {
   if (c.m <= 0 || c.n <= 0) return cudaSuccess;
+  Epilogue e = e_in;
+  e.status = status;
   if (use_umma)
     return umma_gemm((const __nv_bfloat16*)c.A, c.lda, c.a_mn, (const __nv_bfloat16*)c.B, c.ldb, c.b_mn,
                      c.m, c.n, c.k, e, status, stream);
@@ -233,7 +235,8 @@ pctc_status_t pctc_workspace_status(const void* workspace, void* stream, int32_t
   cudaStream_t s = (cudaStream_t)stream;
   if (cudaMemcpyAsync(status_host, workspace, 4, cudaMemcpyDeviceToHost, s) != cudaSuccess) return PCTC_ERR_CUDA;
   if (cudaStreamSynchronize(s) != cudaSuccess) return PCTC_ERR_CUDA;
-  return *status_host ? PCTC_ERR_TIMEOUT : PCTC_OK;
+  if (*status_host == 0) return PCTC_OK;
+  return *status_host < 0x100 ? PCTC_ERR_TIMEOUT : PCTC_ERR_INVALID_ARG;
 }
 
 pctc_status_t pctc_gemm_bf16(const void* A, const void* B, float* C, int32_t m, int32_t n, int32_t k,
@@ -332,6 +335,9 @@ pctc_status_t run_call(const pctc_problem_t* p, const void* hidden, const void* 
   bm.row0 = d_meta + 2 * N;
   bm.row_utt = d_meta + 3 * N + 1;
   bm.cell0 = d_cell0;
+  bm.N = N;
+  bm.M = M;
+  bm.status = (int*)(ws + pl.o_status);
 
   int* d_status = (int*)(ws + pl.o_status);
   unsigned* d_bitmap = (unsigned*)(ws + pl.o_bitmap);
@@ -371,7 +377,7 @@ pctc_status_t run_call(const pctc_problem_t* p, const void* hidden, const void* 
   PCTC_CUDA(subset_and_relabel(targets, p->target_stride, bm.U_n, N, V, p->blank_id, d_bitmap, d_wrank, d_vmap,
                                d_U, d_K, d_rel, d_flags, pl.Kcap, d_status, stream));
   // ---- line 4: stack the valid frames ----
-  PCTC_CUDA(stack_frames(hidden, d_X, N, pl.T, D, pl.elem, bm.row_utt, bm.row0, M, stream));
+  PCTC_CUDA(stack_frames(hidden, d_X, N, pl.T, D, pl.elem, bm.row_utt, bm.row0, M, d_status, stream));
 
   // ---- line 6: logits of the selected classes, Z_U = X W_U^T + b_U; lines 7-10: the DP ----
   // The alignment sum of Eq. "ctc-factorization" needs no normaliser, so the DP runs on Z_U (on the
@@ -380,9 +386,10 @@ pctc_status_t run_call(const pctc_problem_t* p, const void* hidden, const void* 
   auto subset_logits_and_dp = [&]() -> pctc_status_t {
     PCTC_MARK(PCTC_PHASE_SUBSET_LOGP);
     {
-      PCTC_CUDA(gather_rows(W, d_WU, d_U, d_K, pl.Kcap, D, pl.elem, stream));
+      PCTC_CUDA(gather_rows(W, d_WU, d_U, d_K, pl.Kcap, D, pl.elem, V, d_status, stream));
       Epilogue e;
       e.kind = EPI_SUBSET_LOGP;
+      e.vocab = V;
       e.out = d_S;
       e.ld = (long long)pl.ldS;
       e.lambda = nullptr;
@@ -456,7 +463,7 @@ pctc_status_t run_call(const pctc_problem_t* p, const void* hidden, const void* 
   }
   PCTC_CUDA(cudaStreamWaitEvent(stream, aux.join, 0));
   PCTC_CUDA(finalize_loss(d_lambda, bm, N, loss, d_flags, dp.roww, stream));
-  if (!p->forward_only) PCTC_CUDA(zero_nonfinite_rows(d_X, M, D, pl.elem, bm.row_utt, d_flags, stream));
+  if (!p->forward_only) PCTC_CUDA(zero_nonfinite_rows(d_X, M, D, pl.elem, bm.row_utt, d_flags, N, d_status, stream));
 
   // ---- lines 11-17: backward, one vocabulary chunk at a time ----
   int dh_slabs = 1;                  // dX accumulator slabs in use (k-split of the dX contraction)
@@ -468,6 +475,7 @@ pctc_status_t run_call(const pctc_problem_t* p, const void* hidden, const void* 
     {
       Epilogue e;                      // recompute Z_c and form Eq. "vjp"
       e.kind = EPI_DLOGITS;
+      e.vocab = V;
       e.out = d_chunk;
       e.ld = pl.chunk;
       e.out_is_bf16 = pl.bf16;
@@ -536,7 +544,9 @@ pctc_status_t run_call(const pctc_problem_t* p, const void* hidden, const void* 
     PCTC_CUDA(cudaStreamWaitEvent(stream, aux.copies_done, 0));
   }
   PCTC_MARK(PCTC_PHASE_FINISH);
-  if (!p->forward_only) PCTC_CUDA(unstack_cast(d_dHacc, dh_slabs, (size_t)pl.slab_rows * D, dH, N, pl.T, D, pl.bf16, bm.T_n, bm.row0, stream));
+  if (!p->forward_only)
+    PCTC_CUDA(unstack_cast(d_dHacc, dh_slabs, (size_t)pl.slab_rows * D, dH, N, pl.T, D, pl.bf16, bm.T_n, bm.row0, M,
+                           d_status, stream));
 
   // ---- optional integer outputs ----
   if (subset_out)
@@ -766,7 +776,7 @@ pctc_status_t pctc_greedy_decode(const pctc_problem_t* p, const void* hidden, co
   void* d_X = ws + g.o_X;
   float2* d_partial = (float2*)(ws + g.o_partial);
   int* d_labels = (int*)(ws + g.o_labels);
-  PCTC_CUDA(stack_frames(hidden, d_X, N, g.T, D, g.elem, d_row_utt, d_row0, M, stream));
+  PCTC_CUDA(stack_frames(hidden, d_X, N, g.T, D, g.elem, d_row_utt, d_row0, M, (int*)(ws + g.o_status), stream));
   Epilogue e;
   e.kind = EPI_ARGMAX_PARTIAL;
   e.bias = bias;

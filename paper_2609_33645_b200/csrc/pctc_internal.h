@@ -10,6 +10,28 @@
 namespace pctc {
 
 // ---------------------------------------------------------------------------
+// Index checks of the debug build (-DPCTC_DEBUG_BOUNDS): every index a kernel gathers or scatters
+// through (row tables, selected classes, relabelled targets, label chains) is range-checked before
+// use.  A bad index stores 0x200 + the number of the checking site in the status word (the first
+// one wins) and the access is skipped; nothing faults.  In the regular build the check is compiled
+// out.  Status word codes: 1-4 a bounded wait gave up (which wait), 0x100 more selected classes than
+// problem.max_K, 0x201.. an index out of range.
+// ---------------------------------------------------------------------------
+#ifdef PCTC_DEBUG_BOUNDS
+constexpr bool kCheckBounds = true;
+#else
+constexpr bool kCheckBounds = false;
+#endif
+#ifdef __CUDACC__
+__device__ __forceinline__ bool index_ok(long long idx, long long lo, long long hi, int* status, int site) {
+  if (!kCheckBounds) return true;
+  if (idx >= lo && idx < hi) return true;
+  if (status) atomicCAS(status, 0, 0x200 + site);
+  return false;
+}
+#endif
+
+// ---------------------------------------------------------------------------
 // Contractions:  acc(i,j) = sum_k A(i,k) * B(j,k),  then an epilogue.
 // ---------------------------------------------------------------------------
 
@@ -46,6 +68,8 @@ struct Epilogue {
   long long ld_colpart = 0;     //   each block of 32 rows of the rounded output (db_c = dZ_c^T 1), or null
   int ksplit = 1;               // EPI_ACCUM_F32 on the tensor-core path: the contraction is cut into this many
   int ksplit_rows = 0;          //   ranges of k; range s accumulates into rows [s * ksplit_rows, ...) of `out`
+  long long vocab = 0;          // V, for the index checks of the debug build
+  int* status = nullptr;        //   ... and the status word they report to
 };
 
 struct GemmShape {
@@ -95,6 +119,8 @@ struct BatchMeta {              // device arrays describing the batch
   const int* row0;              // [N+1] first stacked row of each utterance
   const long long* cell0;       // [N] first trellis cell of each utterance
   const int* row_utt;           // [M] utterance of each stacked row
+  int N = 0, M = 0;             // extents, for the index checks of the debug build
+  int* status = nullptr;        // status word
 };
 
 // Batch description from the host length arrays (U_host may be null: no targets).  The lengths
@@ -112,11 +138,11 @@ cudaError_t subset_and_relabel(const int* targets, int target_stride, const int*
 
 // Algorithm 1 line 4: X[row0[n] + t] = hidden[n, t], t < T_n.
 cudaError_t stack_frames(const void* hidden, void* X, int N, int T, int D, int elem_bytes,
-                         const int* row_utt, const int* row0, int M, cudaStream_t stream);
+                         const int* row_utt, const int* row0, int M, int* status, cudaStream_t stream);
 
 // Zero the stacked frames of utterances flagged non-finite (flag 2), before the backward pass.
 cudaError_t zero_nonfinite_rows(void* X, int M, int D, int elem_bytes, const int* row_utt, const int* utt_flags,
-                                cudaStream_t stream);
+                                int N, int* status, cudaStream_t stream);
 
 // dH[n,t,:] = T(sum over slabs s < nslab, in ascending s, of acc[s*slab_stride + (row0[n]+t)*D + :]) for
 // t < T_n, zero for padded frames.
@@ -125,11 +151,11 @@ cudaError_t colpart_sums(const float* colpart, long long ld, int nblocks, int co
                          long long v0, bool accumulate, cudaStream_t stream);
 
 cudaError_t unstack_cast(const float* acc, int nslab, size_t slab_stride, void* dH, int N, int T, int D,
-                         bool out_bf16, const int* T_n, const int* row0, cudaStream_t stream);
+                         bool out_bf16, const int* T_n, const int* row0, int M, int* status, cudaStream_t stream);
 
 // W_U[j,:] = W[U[j],:] for j < K (rows K.. of the [Kcap, D] buffer are zeroed).
 cudaError_t gather_rows(const void* W, void* W_U, const int* U, const int* Kdev, int Kcap, int D,
-                        int elem_bytes, cudaStream_t stream);
+                        int elem_bytes, long long V, int* status, cudaStream_t stream);
 
 // db[v0 + j] = sum_i chunk[i*ld + j]
 cudaError_t column_sums(const void* chunk, bool chunk_bf16, long long ld, int M, int cols,

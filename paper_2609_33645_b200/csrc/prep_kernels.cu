@@ -171,10 +171,12 @@ __device__ __forceinline__ void zero_row(char* __restrict__ dst, size_t bytes) {
 }
 
 __global__ void k_stack_frames(const char* __restrict__ hidden, char* __restrict__ X, int T, size_t row_bytes,
-                               const int* __restrict__ row_utt, const int* __restrict__ row0) {
+                               const int* __restrict__ row_utt, const int* __restrict__ row0, int N, int* status) {
   const int m = blockIdx.x;
   const int n = row_utt[m];
+  if (!index_ok(n, 0, N, status, 1)) return;
   const int t = m - row0[n];
+  if (!index_ok(t, 0, T, status, 1)) return;
   copy_row(hidden + ((size_t)n * T + t) * row_bytes, X + (size_t)m * row_bytes, row_bytes);
 }
 
@@ -189,13 +191,15 @@ __device__ __forceinline__ void store4(__nv_bfloat16* dst, float4 v) {
 
 template <typename TOut>
 __global__ void k_unstack_cast(const float* __restrict__ acc, int nslab, size_t slab_stride, TOut* __restrict__ dH,
-                               int T, int D, const int* __restrict__ T_n, const int* __restrict__ row0) {
+                               int T, int D, const int* __restrict__ T_n, const int* __restrict__ row0, int M,
+                               int* status) {
   const int n = blockIdx.x / T, t = blockIdx.x - n * T;
   TOut* dst = dH + ((size_t)n * T + t) * D;
   if (t >= T_n[n]) {
     zero_row(reinterpret_cast<char*>(dst), (size_t)D * sizeof(TOut));
     return;
   }
+  if (!index_ok((long long)row0[n] + t, 0, M, status, 3)) return;
   const float* src = acc + ((size_t)row0[n] + t) * D;
   if ((D & 3) == 0) {                          // four columns per thread: 16-byte loads, 8- or 16-byte stores
     for (int d = threadIdx.x * 4; d < D; d += blockDim.x * 4) {
@@ -216,18 +220,19 @@ __global__ void k_unstack_cast(const float* __restrict__ acc, int nslab, size_t 
 }
 
 __global__ void k_gather_rows(const char* __restrict__ W, char* __restrict__ W_U, const int* __restrict__ U,
-                              const int* __restrict__ Kdev, size_t row_bytes) {
+                              const int* __restrict__ Kdev, size_t row_bytes, long long V, int* status) {
   const int j = blockIdx.x;
   char* dst = W_U + (size_t)j * row_bytes;
-  if (j < *Kdev) copy_row(W + (size_t)U[j] * row_bytes, dst, row_bytes);
+  if (j < *Kdev && index_ok(U[j], 0, V, status, 4)) copy_row(W + (size_t)U[j] * row_bytes, dst, row_bytes);
   else zero_row(dst, row_bytes);
 }
 
 // --- frames of an utterance with a non-finite loss (NaN/Inf in its states): the stacked copy is
 // zeroed before the backward pass, so that 0 * NaN cannot leak into dW through dZ^T X ---
 __global__ void k_zero_nonfinite_rows(char* __restrict__ X, size_t row_bytes, const int* __restrict__ row_utt,
-                                      const int* __restrict__ flags) {
+                                      const int* __restrict__ flags, int N, int* status) {
   const int m = blockIdx.x;
+  if (!index_ok(row_utt[m], 0, N, status, 2)) return;
   if (flags[row_utt[m]] & 2) zero_row(X + (size_t)m * row_bytes, row_bytes);
 }
 
@@ -379,30 +384,31 @@ cudaError_t batch_meta(const int* T_host, const int* U_host, int N, int* T_n, in
 }
 
 cudaError_t stack_frames(const void* hidden, void* X, int N, int T, int D, int elem_bytes,
-                         const int* row_utt, const int* row0, int M, cudaStream_t stream) {
-  (void)N;
-  k_stack_frames<<<M, 128, 0, stream>>>((const char*)hidden, (char*)X, T, (size_t)D * elem_bytes, row_utt, row0);
+                         const int* row_utt, const int* row0, int M, int* status, cudaStream_t stream) {
+  k_stack_frames<<<M, 128, 0, stream>>>((const char*)hidden, (char*)X, T, (size_t)D * elem_bytes, row_utt, row0, N,
+                                        status);
   return cudaGetLastError();
 }
 
 cudaError_t zero_nonfinite_rows(void* X, int M, int D, int elem_bytes, const int* row_utt, const int* utt_flags,
-                                cudaStream_t stream) {
-  k_zero_nonfinite_rows<<<M, 64, 0, stream>>>((char*)X, (size_t)D * elem_bytes, row_utt, utt_flags);
+                                int N, int* status, cudaStream_t stream) {
+  k_zero_nonfinite_rows<<<M, 64, 0, stream>>>((char*)X, (size_t)D * elem_bytes, row_utt, utt_flags, N, status);
   return cudaGetLastError();
 }
 
 cudaError_t unstack_cast(const float* acc, int nslab, size_t slab_stride, void* dH, int N, int T, int D,
-                         bool out_bf16, const int* T_n, const int* row0, cudaStream_t stream) {
+                         bool out_bf16, const int* T_n, const int* row0, int M, int* status, cudaStream_t stream) {
   if (out_bf16)
-    k_unstack_cast<__nv_bfloat16><<<N * T, 128, 0, stream>>>(acc, nslab, slab_stride, (__nv_bfloat16*)dH, T, D, T_n, row0);
+    k_unstack_cast<__nv_bfloat16><<<N * T, 128, 0, stream>>>(acc, nslab, slab_stride, (__nv_bfloat16*)dH, T, D, T_n,
+                                                             row0, M, status);
   else
-    k_unstack_cast<float><<<N * T, 128, 0, stream>>>(acc, nslab, slab_stride, (float*)dH, T, D, T_n, row0);
+    k_unstack_cast<float><<<N * T, 128, 0, stream>>>(acc, nslab, slab_stride, (float*)dH, T, D, T_n, row0, M, status);
   return cudaGetLastError();
 }
 
 cudaError_t gather_rows(const void* W, void* W_U, const int* U, const int* Kdev, int Kcap, int D,
-                        int elem_bytes, cudaStream_t stream) {
-  k_gather_rows<<<Kcap, 128, 0, stream>>>((const char*)W, (char*)W_U, U, Kdev, (size_t)D * elem_bytes);
+                        int elem_bytes, long long V, int* status, cudaStream_t stream) {
+  k_gather_rows<<<Kcap, 128, 0, stream>>>((const char*)W, (char*)W_U, U, Kdev, (size_t)D * elem_bytes, V, status);
   return cudaGetLastError();
 }
 

@@ -140,12 +140,13 @@ __global__ void __launch_bounds__(NT, TS == 64 ? 3 : PCTC_TUNE_SIMT_CTAS) k_simt
           const float z = a + bias_at<T>(e.bias, e.v0 + j);
           if (z > run_max[r]) { run_max[r] = z; run_idx[r] = j; }     // ascending j: first maximum wins
         } else if (EPI == EPI_SUBSET_LOGP) {
-          if (j < Kdev)
+          if (j < Kdev && index_ok(e.U[j], 0, e.vocab, e.status, 10))
             reinterpret_cast<float*>(e.out)[(long long)i * e.ld + j] = a + bias_at<T>(e.bias, e.U[j]) - lam;
         } else if (EPI == EPI_DLOGITS) {
           const long long v = e.v0 + j;
           const float p = __expf(a + bias_at<T>(e.bias, v) - lam);
-          const int jj = e.vmap[v];
+          int jj = e.vmap[v];
+          if (!index_ok(jj, -1, e.ld_gamma, e.status, 9)) jj = -1;
           const float gam = (jj >= 0) ? e.gamma[(long long)i * e.ld_gamma + jj] : 0.f;
           reinterpret_cast<T*>(e.out)[(long long)i * e.ld + j] = T(w == 0.f ? 0.f : w * (p - gam));
         } else if (EPI == EPI_ACCUM_F32) {

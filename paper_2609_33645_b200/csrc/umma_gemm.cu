@@ -81,6 +81,9 @@ constexpr int MN_GROUP_BYTES = 64 * BK * 2;          // one 64-wide MN group of 
 #ifndef PCTC_WAIT_LIMIT_CYCLES
 #define PCTC_WAIT_LIMIT_CYCLES 4000000000LL   // about two seconds; a test build shortens it so that a wait runs out
 #endif
+#ifndef PCTC_WAIT_POLL_MASK
+#define PCTC_WAIT_POLL_MASK 255u              // the clock and the abort flag are looked at every 256th poll
+#endif
 constexpr long long WAIT_LIMIT_CYCLES = PCTC_WAIT_LIMIT_CYCLES;
 constexpr long long DRAIN_LIMIT_CYCLES = 200000000LL;   // the waits of an aborting CTA for its own copies and MMAs
 constexpr long long ABORT_LINGER_CYCLES = 2000000LL;    // an aborting CTA stays this long before it leaves (see the kernel's end)
@@ -180,7 +183,7 @@ __device__ __forceinline__ bool mbar_wait(unsigned long long* bar, unsigned pari
   const long long t0 = clock64();
   for (unsigned it = 1;; ++it) {
     if (mbar_try(bar, parity)) return true;
-    if ((it & 255u) == 0u) {
+    if ((it & PCTC_WAIT_POLL_MASK) == 0u) {
       if (*abort_flag) return false;
       if (clock64() - t0 > limit) {
         *abort_flag = 1;
@@ -592,7 +595,9 @@ k_umma_gemm(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
 #pragma unroll
       for (int gq = 0; gq < NGRP; ++gq) {
         const int j = nt2 * BN + c_base + gq * 32 + lane;
-        pre_jj[gq] = (j < n_eff) ? a.e.vmap[a.e.v0 + j] : -1;
+        int jj = (j < n_eff) ? a.e.vmap[a.e.v0 + j] : -1;
+        if (!index_ok(jj, -1, a.e.ld_gamma, a.status, 9)) jj = -1;      // the class map indexes a row of gamma
+        pre_jj[gq] = jj;
       }
     };
     if (EPI == EPI_DLOGITS && group < units) prefetch(group);
@@ -630,7 +635,10 @@ k_umma_gemm(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
             const int j = n0 + c_base + c;
             float b = 0.f;
             if (bias && j < n_eff) {
-              if (EPI == EPI_SUBSET_LOGP) b = __bfloat162float(bias[a.e.U[j]]);
+              if (EPI == EPI_SUBSET_LOGP) {
+                const int cls = a.e.U[j];
+                if (index_ok(cls, 0, a.e.vocab, a.status, 10)) b = __bfloat162float(bias[cls]);
+              }
               else b = __bfloat162float(bias[a.e.v0 + j]);
             }
             sb[c] = b;

@@ -22,6 +22,7 @@ def rel_fro(x, ref):
 
 
 def run_gpu(binding, batch, *, beam=0.0, chunk=0, gemm_path=0, check_status=True, utt_weights=None, **kw):
+    """kw goes to binding.pruned_ctc_fwd_bwd (skip_dW, max_K, lib_handle, ...)."""
     import torch
 
     dev = torch.device("cuda:0")

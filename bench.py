@@ -136,6 +136,74 @@ def _traced_call(binding, hidden, W, bias_dev, targets, il, tl, batch, res, trac
     return trace
 
 
+def time_config(binding, torch, dev, cfg, beam, steps, warmup, peaks):
+    """Device-resident timing of one configuration with the protocol of the headline run: inputs in HBM,
+    `warmup` untimed calls, `steps` timed calls between two CUDA events on the launching stream."""
+    batch = wl.make_batch(cfg)
+    tdt = torch.bfloat16 if cfg.dtype == "bf16" else torch.float32
+    hidden = torch.from_numpy(batch.hidden).to(tdt).to(dev)
+    W = torch.from_numpy(batch.W).to(tdt).to(dev)
+    targets = torch.from_numpy(batch.targets).to(dev)
+    il, tl = batch.input_lengths, batch.target_lengths
+    M, D, V, N = batch.M, cfg.D, cfg.V, cfg.N
+    dt = binding.PCTC_BF16 if cfg.dtype == "bf16" else binding.PCTC_FP32
+    prob = binding.make_problem(N, batch.T, D, V, dt, batch.blank, beam, 0, batch.targets.shape[1])
+    ws_bytes = binding.workspace_bytes(prob, il, tl)
+    chunk, nchunks = binding.chunk_width(prob, il, tl)
+    half = binding.make_problem(N, batch.T, D, max(8, V // 2 // 8 * 8), dt, batch.blank, beam, chunk,
+                                batch.targets.shape[1])
+    ws_half = binding.workspace_bytes(half, il, tl)
+    res = binding.pruned_ctc_fwd_bwd(hidden, W, None, targets, il, tl, batch.blank, beam=beam, check_status=True)
+    for _ in range(max(0, warmup - 1)):
+        binding.pruned_ctc_fwd_bwd(hidden, W, None, targets, il, tl, batch.blank, beam=beam,
+                                   workspace=res["workspace"], out=res)
+    trace = binding.Trace(binding.Trace.capacity_for(V, chunk))
+    ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    torch.cuda.synchronize()
+    ev0.record()
+    for s in range(steps):
+        binding.pruned_ctc_fwd_bwd(hidden, W, None, targets, il, tl, batch.blank, beam=beam,
+                                   workspace=res["workspace"], out=res, trace=trace if s == steps - 1 else None)
+    ev1.record()
+    torch.cuda.synchronize()
+    if binding.workspace_status(res["workspace"]) != 0:
+        raise SystemExit("device status word set while timing " + cfg.name)
+    ms = ev0.elapsed_time(ev1) / steps
+    dp_ms = sum(t for kind, t in trace.spans() if kind >= 0 and binding.PHASES[kind] == "dp")
+    flops = 8.0 * M * D * V
+    tfl = flops / (ms * 1e-3) / 1e12
+    out = dict(workload=cfg.name, dtype=cfg.dtype, beam=beam, M_frames=M, K_selected=int(res["K"].item()), D=D, V=V,
+               chunk=chunk, steps=steps, warmup=warmup, ms_per_step=round(ms, 4), frames_per_s=round(M / (ms * 1e-3), 1),
+               tflops=round(tfl, 2),
+               frac_of_bf16_peak=(dict(burst=round(tfl / peaks["bf16_tflops"], 4),
+                                       sustained=round(tfl / peaks["bf16_tflops_sustained"], 4))
+                                  if cfg.dtype == "bf16" else None),
+               dp_ms=round(dp_ms, 4), workspace_bytes=ws_bytes, workspace_bytes_at_half_V=ws_half,
+               one_fp32_MxV_array=4 * M * V,
+               l2=("inputs larger than L2" if W.numel() * W.element_size() > (126 << 20) else
+                   "inputs smaller than L2: L2 flushed by nothing, latency-bound case"))
+    del res, hidden, W, targets, trace
+    torch.cuda.empty_cache()
+    return out
+
+
+def load_traffic(cfg_name: str, chunk: int):
+    """DRAM bytes of the dominant kernel per step for this workload and chunk width, if a capture of it is
+    on record (a small JSON written beside the summary of that ncu capture)."""
+    path = os.path.join(ROOT, "profiles", "umma_gemm_dram_traffic.json")
+    try:
+        with open(path) as f:
+            table = json.load(f)
+    except (OSError, ValueError):
+        return None
+    for row in table.get("captures", []):
+        if row.get("workload") == cfg_name and int(row.get("chunk", -1)) == int(chunk):
+            return dict(bytes_per_step=row["bytes_per_step"], launches_per_step=row["launches_per_step"],
+                        bytes_per_launch_avg=row["bytes_per_step"] / row["launches_per_step"],
+                        source=row.get("source", "ncu dram__bytes_read.sum + dram__bytes_write.sum"))
+    return None
+
+
 def oracle_sample(batch, frames: int):
     """The first `frames` frames of utterance 0 with a proportional prefix of its labels."""
     n = 0
@@ -223,6 +291,12 @@ def main():
     ap.add_argument("--dense-head", action="store_true",
                     help="also time the three library GEMMs of a dense bf16 head that holds its [M, V] logits "
                          "(forward, dX, dW: 6 M D V FLOPs) on the same shapes, as a yardstick for the time ratio")
+    ap.add_argument("--all-configs", dest="all_configs", action="store_true", default=None,
+                    help="after the headline region, time every configuration (c1, c2, c3, c4, c5 without a beam "
+                         "and at beams 8 and 16) with the same protocol and fewer steps, and report them in an "
+                         "`all_configs` block (default: on for the default workload on one GPU)")
+    ap.add_argument("--no-all-configs", dest="all_configs", action="store_false")
+    ap.add_argument("--all-steps", type=int, default=10, help="timed steps per configuration of --all-configs")
     ap.add_argument("--e2e-steps", type=int, default=3)
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--cpu-frames", type=int, default=1024)
@@ -367,13 +441,11 @@ def main():
         per_kernel[k] = dict(ms=round(phase_ms[k], 4), launches=phase_cnt[k] // args.steps,
                              tflops=round(split_flops[k] / (phase_ms[k] * 1e-3) / 1e12, 2))
 
-    # DRAM bytes of the dominant kernel's launches of one step, from the ncu capture summarised in
-    # profiles/umma_gemm_c4_speed_of_light.md (default workload and chunk only)
+    # DRAM bytes of the dominant kernel's launches of one step: from the record of an ncu capture of this
+    # workload at this chunk width, if there is one (null otherwise)
     traffic = None
-    if args.config == "c4" and not args.vocab and chunk == 16384 and not args.frozen_head and args.beam == 0 and not args.bias:
-        traffic = dict(bytes_per_step=33.7e9, launches_per_step=31, bytes_per_launch_avg=33.7e9 / 31,
-                       source="ncu dram__bytes_read.sum + dram__bytes_write.sum: the LSE launch and chunks 0-1 of each "
-                              "chunk kernel, chunk averages scaled by launches")
+    if not args.vocab and not args.frozen_head and args.beam == 0 and not args.bias:
+        traffic = load_traffic(cfg.name, chunk)
 
     # kernels launched by the library inside the timed region
     dp_launches = 4 if args.beam > 0 else 2      # sweeps (+ best-alignment sweeps, arc flags), occupancies
@@ -462,13 +534,29 @@ def main():
                    sample=(f"oracle fwd+bwd (float64, full V, full dW) on the first {frames} frames of "
                            f"utterance 0 of {cfg.name}"))
 
+    # ---- every configuration, same protocol, fewer steps (the headline stays the default workload) ----
+    all_cfg = None
+    want_all = args.all_configs
+    if want_all is None:
+        want_all = (args.config == "c4" and world == 1 and not (args.vocab or args.frozen_head or args.bias
+                                                                 or args.allreduce_dw or args.chunk or args.beam))
+    K_selected = int(res["K"].item())
+    w_gb = W.numel() * W.element_size() / 1e9
+    if want_all and world == 1:
+        del res, hidden, W, targets, traces
+        torch.cuda.empty_cache()
+        all_cfg = []
+        for name, beams in (("c1", (0.0,)), ("c2", (0.0,)), ("c3", (0.0,)), ("c4", (0.0,)), ("c5", (0.0, 16.0, 8.0))):
+            for b in beams:
+                all_cfg.append(time_config(binding, torch, dev, wl.CONFIGS[name], b, args.all_steps, 3, peaks))
+
     line = dict(
         metric=METRIC, value=value, unit=UNIT, n_gpus=world, steps=args.steps, warmup=args.warmup,
         ms_per_step=ms_per_step, higher_is_better=True, scaling="weak", vs_baseline=None,
         dtype=cfg.dtype, data="synthetic",
         config=dict(workload=cfg.name, N=N, T_range=[cfg.T_lo, cfg.T_hi], D=D, V=V, M_frames=M,
-                    K_selected=int(res["K"].item()), beam=args.beam, chunk=chunk, frozen_head=args.frozen_head, bias=args.bias, max_K=max_K,
-                    l2="inputs larger than L2 (W and dW are %.2f GB each)" % (W.numel() * 2 / 1e9),
+                    K_selected=K_selected, beam=args.beam, chunk=chunk, frozen_head=args.frozen_head, bias=args.bias, max_K=max_K,
+                    l2="inputs larger than L2 (W and dW are %.2f GB each)" % w_gb,
                     parallelism=("utterance-sharded data parallel, dW all-reduced per vocabulary chunk (NCCL)"
                                  if sum_dW else "independent utterance batches per GPU, no collective")),
         tflops=flops_all / (ms_per_step * 1e-3) / 1e12,
@@ -487,6 +575,8 @@ def main():
                         one_fp32_MxV_array=4 * M * V),
         e2e=e2e, gpu_launches=gpu_launches, clocks=clocks, cpu_baseline=cpu,
     )
+    if all_cfg is not None:
+        line["all_configs"] = all_cfg
     if dense is not None:
         line["dense_head"] = dense
     print(json.dumps(line), flush=True)

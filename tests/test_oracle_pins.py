@@ -425,3 +425,22 @@ def test_collapse_map_and_greedy_decode():
         Z = H[n, :Tn] @ W.T
         assert list(frames[n]) == [int(np.argmax(z)) for z in Z]
         assert hyps[n] == collapse(list(frames[n]), 2)
+    # a planted answer: orthonormal class vectors, every frame a multiple of its class's vector plus a
+    # little noise, so the top class of each frame is known without taking any arg-max
+    V = D = 9
+    Q, _ = np.linalg.qr(rng.standard_normal((D, D)))
+    planted = [[3, 3, 0, 0, 3, 7, 7, 0, 1, 1, 1, 8], [0, 0, 5, 0, 5, 5, 2]]
+    Hp = np.zeros((2, 12, D))
+    for n, labs in enumerate(planted):
+        for t, v in enumerate(labs):
+            Hp[n, t] = 4.0 * Q[v] + 0.05 * rng.standard_normal(D)
+    frames, hyps, _ = O.greedy_decode(Hp, Q, None, [12, 7], 0)
+    assert [list(f) for f in frames] == planted
+    assert hyps == [[3, 3, 7, 1, 8], [5, 5, 2]]                  # worked by hand from the planted frames
+    # equal logits: the smallest class index wins (two identical head rows)
+    W2 = np.array([[0.0, 1.0], [1.0, 0.0], [1.0, 0.0], [0.5, 0.5]])
+    frames, _, _ = O.greedy_decode(np.array([[[2.0, 0.0], [0.0, 3.0]]]), W2, None, [2], 0)
+    assert list(frames[0]) == [1, 0]
+    # a bias can overturn the projection's winner
+    frames, _, _ = O.greedy_decode(np.array([[[2.0, 0.0]]]), W2, np.array([0.0, 0.0, 0.0, 1.5]), [1], 0)
+    assert list(frames[0]) == [3]

@@ -53,15 +53,16 @@ class ClockSampler:
          "clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
          "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
 
-    def __init__(self, gpu_index: int):
+    def __init__(self, gpu_index: int, period_ms: int = 200):
         self.gpu = gpu_index
+        self.period_ms = int(period_ms)
         self.proc = None
         self.lines = []
 
     def start(self):
         try:
             self.proc = subprocess.Popen(
-                ["nvidia-smi", f"--query-gpu={self.Q}", "--format=csv,noheader,nounits", "-lms", "200",
+                ["nvidia-smi", f"--query-gpu={self.Q}", "--format=csv,noheader,nounits", "-lms", str(self.period_ms),
                  "-i", str(self.gpu)], stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
             self.thread = threading.Thread(target=self._read, daemon=True)
             self.thread.start()
@@ -297,6 +298,11 @@ def main():
                          "`all_configs` block (default: on for the default workload on one GPU)")
     ap.add_argument("--no-all-configs", dest="all_configs", action="store_false")
     ap.add_argument("--all-steps", type=int, default=10, help="timed steps per configuration of --all-configs")
+    ap.add_argument("--lib-variant", default="",
+                    help="time a measurement build of the library (build.VARIANTS, probe_*): one part of the "
+                         "tensor-core kernel is knocked out, so the results are wrong on purpose and the line "
+                         "is marked invalid; it shows what the step is bound by")
+    ap.add_argument("--clock-ms", type=int, default=200, help="sampling period of the clock record")
     ap.add_argument("--e2e-steps", type=int, default=3)
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--cpu-frames", type=int, default=1024)
@@ -337,8 +343,13 @@ def main():
             dist.init_process_group(backend)
     if rank == 0:
         build.build()
+        if args.lib_variant:
+            build.build_variant(args.lib_variant)
     if world > 1:
         dist.barrier()
+    if args.lib_variant:
+        binding.LIB_PATH = build.variant_path(args.lib_variant)
+        args.e2e_steps, args.all_configs, args.no_cpu_baseline = 0, False, True
     binding.load()
     peaks = load_peaks()
 
@@ -388,7 +399,7 @@ def main():
             dp.allreduce_rows(res["dW"], dw_rows, dp.dw_ready_events(
                 _traced_call(binding, hidden, W, bias_dev, targets, il, tl, batch, res, traces[0], dev_call)), comm_stream=comm)
         torch.cuda.synchronize()
-    sampler = ClockSampler(local_dev)
+    sampler = ClockSampler(local_dev, args.clock_ms)
     if rank == 0:
         sampler.start()
         time.sleep(0.25)
@@ -575,6 +586,8 @@ def main():
                         one_fp32_MxV_array=4 * M * V),
         e2e=e2e, gpu_launches=gpu_launches, clocks=clocks, cpu_baseline=cpu,
     )
+    if args.lib_variant:
+        line["invalid"] = "measurement build %s: part of the kernel is knocked out, results are wrong" % args.lib_variant
     if all_cfg is not None:
         line["all_configs"] = all_cfg
     if dense is not None:

@@ -103,9 +103,11 @@ pctc_status_t pctc_workspace_bytes(const pctc_problem_t* problem,
  * The vocabulary chunk width C a call on this problem will use, and the number of
  * chunks ceil(V / C) (host-only; touches no device).  With problem->chunk > 0 it
  * is that value rounded up to the tile width of the path that runs; with 0 it is
- * the library's choice: 4,096 for fp32; for bf16 32,768 (D <= 1,024) or 16,384
- * columns, halved down to no less than 8,192 while the
- * [M, C] chunk temporary of Algorithm 1 (lines 12-13) would exceed 512 MiB.  The
+ * the library's choice: 4,096 for fp32; for bf16 and D <= 1,024 the largest of 56,832,
+ * 37,888 and 18,944 columns (multiples of 74 x 256: whole waves of the 74 CTA pairs of a
+ * B200) whose [M, C] chunk temporary of Algorithm 1 (lines 12-13) stays within 512 MiB;
+ * otherwise 16,384 columns, halved down to no less than 8,192 while that temporary would
+ * exceed 512 MiB.  The
  * chunk width changes the order of summation only, never what is computed.
  * nchunks_out may be NULL.  Same argument checks as pctc_workspace_bytes.
  */

@@ -55,10 +55,16 @@ def headers():
 #   bounds     every index that a kernel gathers or scatters through (selected classes, relabelled
 #              targets, row tables) is range-checked first; a bad one is recorded in the status word
 #              and the access is skipped
+#   probe_*    measurement probes for `bench.py --lib-variant`: one part of the tensor-core kernel is
+#              knocked out (results are wrong on purpose) to show what a launch is bound by
 VARIANTS = {
     "shortwait": ("-DPCTC_WAIT_LIMIT_CYCLES=3000LL", "-DPCTC_WAIT_POLL_MASK=0u"),
     "bounds": ("-DPCTC_DEBUG_BOUNDS=1",),
+    "probe_noepilogue": ("-DPCTC_PROBE=7",),      # no tensor-memory loads, no epilogue arithmetic, no chunk store
+    "probe_nostore": ("-DPCTC_PROBE=4",),         # the dlogits chunk is computed but not written
+    "probe_skipa": ("-DPCTC_PROBE=8",),           # the normaliser kernel reloads only its B operand per tile
 }
+TEST_VARIANTS = ("shortwait", "bounds")           # the ones the test-suite loads
 
 
 def variant_path(tag: str) -> str:

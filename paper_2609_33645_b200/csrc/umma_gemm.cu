@@ -62,6 +62,20 @@ namespace {
 #define PCTC_TUNE_CTAS 2          // CTAs per tile: 2 = tcgen05 cta_group::2 pairs, 1 = independent CTAs
 #endif
 
+// Measurement probes (never set in the regular build; results are then wrong on purpose).  They knock
+// out one part of the kernel at a time to show what a launch is bound by:
+//   bit 0  the LSE and dlogits epilogues do not read tensor memory (they work on constants)
+//   bit 1  ... do no arithmetic (no exponentials, no maxima)
+//   bit 2  the dlogits epilogue does not stage or store the chunk
+//   bit 3  the column-walking kernels load their A rows only for the first tile of a unit
+#ifndef PCTC_PROBE
+#define PCTC_PROBE 0
+#endif
+constexpr bool PROBE_NO_TMEM_LD = (PCTC_PROBE & 1) != 0;
+constexpr bool PROBE_NO_MATH = (PCTC_PROBE & 2) != 0;
+constexpr bool PROBE_NO_STORE = (PCTC_PROBE & 4) != 0;
+constexpr bool PROBE_SKIP_A = (PCTC_PROBE & 8) != 0;
+
 #ifndef PCTC_TUNE_EPI_WARPS
 #define PCTC_TUNE_EPI_WARPS 0     // 0: by the contraction depth; 4 or 8: forced
 #endif
@@ -479,11 +493,13 @@ k_umma_gemm(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
             const unsigned ph = (g / STAGES) & 1u;
             if (!mbar_wait(&st->empty[s], ph ^ 1u, abort_flag, a.status, 1)) { ok = false; break; }
             // the leader's barrier counts the bytes of both CTAs
-            if (rank == 0) mbar_expect_tx(&st->full[s], CTAS * (A_STAGE + B_STAGE_BYTES));
+            const bool skip_a = PROBE_SKIP_A && epi_walks_splits(EPI) && nt != nt0;
+            if (rank == 0) mbar_expect_tx(&st->full[s], CTAS * ((skip_a ? 0 : A_STAGE) + B_STAGE_BYTES));
             unsigned char* dA = sA + (size_t)s * A_STAGE;
             unsigned char* dB = sB + (size_t)s * B_STAGE_BYTES;
 #pragma unroll
             for (int h = 0; h < MT; ++h) {               // sub-tile h: this CTA's 128 rows of pair rows h*256..
+              if (skip_a) break;
               unsigned char* dAh = dA + h * A_STAGE_BYTES;
               const int row_ah = row_a + h * SUB_M;
               if (!a.a_mn) {
@@ -675,7 +691,12 @@ k_umma_gemm(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
             const int j0 = n0 + c_base + g0;
             if (j0 >= n_eff) break;                   // warp-uniform
             float v[32];
-            tmem_ld32(taddr + g0, v);
+            if (PROBE_NO_TMEM_LD && EPI == EPI_DLOGITS) {
+#pragma unroll
+              for (int c = 0; c < 32; ++c) v[c] = (float)(lane + c) * 1e-3f;
+            } else {
+              tmem_ld32(taddr + g0, v);
+            }
             if (EPI == EPI_SUBSET_LOGP) {               // Z_U (or S = Z_U - lambda); columns past K are written as 0
 #pragma unroll
               for (int c = 0; c < 32; ++c)
@@ -684,12 +705,14 @@ k_umma_gemm(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
             if (EPI == EPI_DLOGITS) {
               if (has_bias) add_bias32(v, sb + g0);
               // w p = exp2(z log2(e) + off2), off2 = log2(w) - lambda log2(e): one packed FMA per two logits
+              if (!PROBE_NO_MATH) {
 #pragma unroll
-              for (int c = 0; c < 32; c += 2) {
-                float x0, x1;
-                ffma2(x0, x1, v[c], v[c + 1], LOG2E, LOG2E, off2, off2);
-                v[c] = ex2(x0);
-                v[c + 1] = ex2(x1);
+                for (int c = 0; c < 32; c += 2) {
+                  float x0, x1;
+                  ffma2(x0, x1, v[c], v[c + 1], LOG2E, LOG2E, off2, off2);
+                  v[c] = ex2(x0);
+                  v[c + 1] = ex2(x1);
+                }
               }
               if (sg[cg] != 0u) {
                 // the group holds selected classes: subtract their weighted occupancy in fp32, before
@@ -714,6 +737,13 @@ k_umma_gemm(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
               }
             }
             constexpr int NBOX = epi_fp32_boxes(EPI) ? 2 : 1;        // boxes per group
+            if (PROBE_NO_STORE && EPI == EPI_DLOGITS) {              // keep the values alive, store nothing
+              float t = 0.f;
+#pragma unroll
+              for (int c = 0; c < 32; ++c) t += v[c];
+              if (t == 12345.678f) a.status[1] = 1;
+              continue;
+            }
 #pragma unroll
             for (int b = 0; b < NBOX; ++b) {
               if (NBOX == 2 && j0 + b * 16 >= n_eff) break;          // warp-uniform
@@ -778,7 +808,19 @@ k_umma_gemm(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
           const int j0 = n0 + c_base + cg * 32;
           if (j0 >= n_eff) break;                    // warp-uniform
           float v[32];
-          tmem_ld32(taddr + cg * 32, v);
+          if (PROBE_NO_TMEM_LD && EPI == EPI_LSE_PARTIAL) {
+#pragma unroll
+            for (int c = 0; c < 32; ++c) v[c] = (float)(lane + c) * 1e-3f;
+          } else {
+            tmem_ld32(taddr + cg * 32, v);
+          }
+          if (PROBE_NO_MATH && EPI == EPI_LSE_PARTIAL) {
+            float t = 0.f;
+#pragma unroll
+            for (int c = 0; c < 32; ++c) t += v[c];
+            run_sum += t;
+            continue;
+          }
           if (EPI == EPI_STORE_F32) {
             if (row_ok) {
               float* dst = (float*)a.e.out + (long long)i * a.e.ld + j0;

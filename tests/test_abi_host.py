@@ -61,7 +61,10 @@ def test_workspace_has_no_M_times_V_term(lib):
 @pytest.mark.parametrize("kw,il,want", [
     (dict(dtype=1), [50, 40], (1000, 1)),                           # fp32: 4,096, capped by V
     (dict(dtype=1, V=10000), [50, 40], (4096, 3)),
-    (dict(dtype=0, D=512, V=180000), [50, 40], (32768, 6)),         # narrow head: wide chunks
+    (dict(dtype=0, D=512, V=180000), [50, 40], (56832, 4)),         # narrow head: 3 x 74 x 256 columns
+    (dict(dtype=0, D=512, V=180000, N=2, T=6400), [6399, 1], (37888, 5)),      # c2's frame count: 2 x 74 x 256
+    (dict(dtype=0, D=1024, V=151936, N=2, T=4470), [4469, 1], (56832, 3)),     # c3's
+    (dict(dtype=0, D=512, V=180000, N=2, T=14000), [13999, 1], (18944, 10)),
     (dict(dtype=0, D=2048, V=180000), [50, 40], (16384, 11)),
     (dict(dtype=0, D=4096, V=151936), [50, 40], (16384, 10)),
     (dict(dtype=0, D=4096, V=151936, N=2, T=20000), [20000, 1], (8192, 19)),     # 512 MiB rule

@@ -76,6 +76,10 @@ constexpr bool PROBE_NO_MATH = (PCTC_PROBE & 2) != 0;
 constexpr bool PROBE_NO_STORE = (PCTC_PROBE & 4) != 0;
 constexpr bool PROBE_SKIP_A = (PCTC_PROBE & 8) != 0;
 
+#ifndef PCTC_TUNE_CHUNK_HINT
+#define PCTC_TUNE_CHUNK_HINT 0    // L2 eviction priority for the bf16 dlogits chunk: bit 0 evict-first on its stores
+#endif                            // (dlogits), bit 1 evict-first on its loads (A operand of the dX and dW kernels)
+
 #ifndef PCTC_TUNE_EPI_WARPS
 #define PCTC_TUNE_EPI_WARPS 0     // 0: by the contraction depth; 4 or 8: forced
 #endif
@@ -232,6 +236,18 @@ __device__ __forceinline__ void tma_store_2d(const CUtensorMap* map, const void*
                ::"l"(map), "r"(c0), "r"(c1), "r"(smem_u32(smem_src))
                : "memory");
 }
+// The same copies with an L2 eviction-priority hint (a policy word from make_evict_first_policy).
+__device__ __forceinline__ unsigned long long make_evict_first_policy() {
+  unsigned long long p;
+  asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(p));
+  return p;
+}
+__device__ __forceinline__ void tma_store_2d_hint(const CUtensorMap* map, const void* smem_src, int c0, int c1,
+                                                  unsigned long long policy) {
+  asm volatile("cp.async.bulk.tensor.2d.global.shared::cta.tile.bulk_group.L2::cache_hint [%0, {%1, %2}], [%3], %4;"
+               ::"l"(map), "r"(c0), "r"(c1), "r"(smem_u32(smem_src)), "l"(policy)
+               : "memory");
+}
 __device__ __forceinline__ void tma_reduce_add_2d(const CUtensorMap* map, const void* smem_src, int c0, int c1) {
   asm volatile("cp.reduce.async.bulk.tensor.2d.global.shared::cta.add.tile.bulk_group [%0, {%1, %2}], [%3];"
                ::"l"(map), "r"(c0), "r"(c1), "r"(smem_u32(smem_src))
@@ -259,6 +275,13 @@ __device__ __forceinline__ void tma_load_2d_pair(void* smem_dst, const CUtensorM
   asm volatile(
       "cp.async.bulk.tensor.2d.cta_group::2.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
       ::"r"(smem_u32(smem_dst)), "l"(map), "r"(c0), "r"(c1), "r"(smem_u32(bar) & PEER_MASK)
+      : "memory");
+}
+__device__ __forceinline__ void tma_load_2d_pair_hint(void* smem_dst, const CUtensorMap* map, int c0, int c1,
+                                                      unsigned long long* bar, unsigned long long policy) {
+  asm volatile(
+      "cp.async.bulk.tensor.2d.cta_group::2.shared::cluster.global.tile.mbarrier::complete_tx::bytes.L2::cache_hint [%0], [%1, {%2, %3}], [%4], %5;"
+      ::"r"(smem_u32(smem_dst)), "l"(map), "r"(c0), "r"(c1), "r"(smem_u32(bar) & PEER_MASK), "l"(policy)
       : "memory");
 }
 __device__ __forceinline__ void mbar_arrive_leader(unsigned long long* bar) {
@@ -481,6 +504,13 @@ k_umma_gemm(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
         if (CTAS == 2) tma_load_2d_pair(dst, map, c0, c1, bar);
         else tma_load_2d(dst, map, c0, c1, bar);
       };
+      // the A operand of the dX and dW contractions is the dlogits chunk
+      constexpr bool HINT_A = (PCTC_TUNE_CHUNK_HINT & 2) && CTAS == 2 && (EPI == EPI_ACCUM_F32 || EPI == EPI_STORE_OUT);
+      const unsigned long long a_policy = HINT_A ? make_evict_first_policy() : 0ull;
+      auto load_a = [&](void* dst, const CUtensorMap* map, int c0, int c1, unsigned long long* bar) {
+        if (HINT_A) tma_load_2d_pair_hint(dst, map, c0, c1, bar, a_policy);
+        else load(dst, map, c0, c1, bar);
+      };
       for (int u = group; u < units && ok; u += ngroups) {
         int mt, sp, ks, nt0, cnt, kb0, kcnt;
         decode_unit(u, m_tiles, n_tiles, splits, ksplit, a.raster_g, mt, sp, ks, nt0, cnt);
@@ -503,11 +533,11 @@ k_umma_gemm(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
               unsigned char* dAh = dA + h * A_STAGE_BYTES;
               const int row_ah = row_a + h * SUB_M;
               if (!a.a_mn) {
-                load(dAh, &tmA, kb * BK, row_ah, &st->full[s]);
+                load_a(dAh, &tmA, kb * BK, row_ah, &st->full[s]);
               } else {
 #pragma unroll
                 for (int q = 0; q < BM / 64; ++q)
-                  load(dAh + q * MN_GROUP_BYTES, &tmA, row_ah + q * 64, kb * BK, &st->full[s]);
+                  load_a(dAh + q * MN_GROUP_BYTES, &tmA, row_ah + q * 64, kb * BK, &st->full[s]);
               }
             }
             if (!a.b_mn) {
@@ -795,6 +825,8 @@ k_umma_gemm(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
               if (lane == 0) {
                 if ((EPI == EPI_ACCUM_F32 || EPI == EPI_STORE_OUT) && a.e.accumulate)
                   tma_reduce_add_2d(&tmC, box, j0 + b * 16, row0_out + h * SUB_M + q * 32);
+                else if ((PCTC_TUNE_CHUNK_HINT & 1) && EPI == EPI_DLOGITS)
+                  tma_store_2d_hint(&tmC, box, j0 + b * 16, row0_out + h * SUB_M + q * 32, make_evict_first_policy());
                 else tma_store_2d(&tmC, box, j0 + b * 16, row0_out + h * SUB_M + q * 32);
                 bulk_commit();
               }

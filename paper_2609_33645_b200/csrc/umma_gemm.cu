@@ -349,6 +349,19 @@ __device__ __forceinline__ void ffma2(float& d0, float& d1, float a0, float a1, 
       : "=f"(d0), "=f"(d1)
       : "f"(a0), "f"(a1), "f"(b0), "f"(b1), "f"(c0), "f"(c1));
 }
+__device__ __forceinline__ void fadd2(float& d0, float& d1, float a0, float a1, float b0, float b1) {
+  asm("{\n\t.reg .b64 ra, rb, rd;\n\t"
+      "mov.b64 ra, {%2, %3};\n\tmov.b64 rb, {%4, %5};\n\t"
+      "add.rn.f32x2 rd, ra, rb;\n\tmov.b64 {%0, %1}, rd;\n\t}"
+      : "=f"(d0), "=f"(d1)
+      : "f"(a0), "f"(a1), "f"(b0), "f"(b1));
+}
+// max of three (one instruction on sm_100)
+__device__ __forceinline__ float fmax3(float a, float b, float c) {
+  float d;
+  asm("max.f32 %0, %1, %2, %3;" : "=f"(d) : "f"(a), "f"(b), "f"(c));
+  return d;
+}
 __device__ __forceinline__ void fmul2(float& d0, float& d1, float a0, float a1, float b0, float b1) {
   asm("{\n\t.reg .b64 ra, rb, rd;\n\t"
       "mov.b64 ra, {%2, %3};\n\tmov.b64 rb, {%4, %5};\n\t"
@@ -872,9 +885,14 @@ k_umma_gemm(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
               // whole group inside the matrix: max over the logits, then one packed FMA per two logits
               // forms x - max and feeds the exponentials
               if (has_bias) add_bias32(v, sb + cg * 32);
-              float gm = v[0];
+              // two chains of three-input maxima (a NaN logit is caught by the sum below, not here)
+              float gm0 = fmax3(v[0], v[1], v[2]), gm1 = fmax3(v[3], v[4], v[5]);
 #pragma unroll
-              for (int c = 1; c < 32; ++c) gm = fmaxf(gm, v[c]);
+              for (int c = 6; c + 3 < 32; c += 4) {
+                gm0 = fmax3(gm0, v[c], v[c + 1]);
+                gm1 = fmax3(gm1, v[c + 2], v[c + 3]);
+              }
+              const float gm = fmax3(gm0, gm1, fmaxf(v[30], v[31]));
               const float gmax = gm * LOG2E;
               if (gmax > run_max2) {
                 run_sum *= ex2(run_max2 - gmax);     // ex2(-inf) = 0 on the first group
@@ -886,8 +904,7 @@ k_umma_gemm(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
               for (int c = 0; c < 32; c += 2) {
                 float x0, x1;
                 ffma2(x0, x1, v[c], v[c + 1], LOG2E, LOG2E, nm, nm);
-                s0 += ex2(x0);
-                s1 += ex2(x1);
+                fadd2(s0, s1, s0, s1, ex2(x0), ex2(x1));   // one packed add per two exponentials
               }
               run_sum += s0 + s1;                    // a NaN logit makes the sum NaN
             } else {

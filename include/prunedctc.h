@@ -260,6 +260,29 @@ pctc_status_t pctc_greedy_decode(const pctc_problem_t* problem,
                                  void* workspace, size_t workspace_bytes, void* stream);
 
 /*
+ * The k best classes of every frame with their log-probabilities under the full-vocabulary
+ * softmax: what a CTC prefix beam search (the paper's decoder, Section 5.1: beam 4; the search
+ * itself is not part of this library) consumes per frame.  The head is applied in vocabulary
+ * chunks of problem->chunk columns (0: 4,096) as in the paper's recognition path (Appendix D);
+ * a chunk's logits live in the workspace only until the frame's running k best and its running
+ * log-sum-exp (Eq. "lognorm") have been updated, so no frames-by-vocabulary array exists.
+ *
+ * Uses N, T, D, V, dtype, chunk, gemm_path of `problem`.  hidden [N,T,D], W [V,D], bias [V] or
+ * NULL (device); input_lengths HOST [N]; k is 1, 2, 4 or 8.  Outputs (device):
+ *   topk_classes  [N,T,k] int32: classes by descending logit, the smaller class first among
+ *                 equal logits; -1 on padded frames and for ranks beyond V;
+ *   topk_logprobs [N,T,k] fp32 or NULL: log p of those classes; -inf where the class is -1.
+ * workspace: at least pctc_topk_workspace_bytes(), 256-byte aligned.
+ */
+pctc_status_t pctc_topk_workspace_bytes(const pctc_problem_t* problem, const int32_t* input_lengths_host,
+                                        int32_t k, size_t* bytes_out);
+pctc_status_t pctc_topk_decode(const pctc_problem_t* problem,
+                               const void* hidden, const void* W, const void* bias,
+                               const int32_t* input_lengths, int32_t k,
+                               int32_t* topk_classes, float* topk_logprobs,
+                               void* workspace, size_t workspace_bytes, void* stream);
+
+/*
  * Contraction kernel on its own, for validation of the tensor-core path:
  *   C[i,j] = sum_k A(i,k) B(j,k),  i < m, j < n, k < k,  C fp32 [m, n] row-major.
  * a_mn_major == 0: A is stored [m, k] (k contiguous); else A is stored [k, m].

@@ -438,6 +438,29 @@ def greedy_decode(hidden, W, bias, input_lengths, blank):
     return frames, hyps, logits
 
 
+def topk_decode(hidden, W, bias, input_lengths, k):
+    """Per utterance: the k classes with the largest logits of every valid frame (descending; the
+    smaller class index first among equal logits) and their log-probabilities under the
+    full-vocabulary softmax (Eq. "lognorm"): what a prefix beam search (Section 5.1) reads per frame."""
+    hidden = np.asarray(hidden, dtype=np.float64)
+    W64 = np.asarray(W, dtype=np.float64)
+    b64 = None if bias is None else np.asarray(bias, dtype=np.float64)
+    classes, logprobs = [], []
+    for n in range(hidden.shape[0]):
+        Z = head_logits(hidden[n, : int(input_lengths[n])], W64, b64)
+        logp = Z - log_normalizer(Z)[:, None]
+        V = Z.shape[1]
+        cls = np.full((Z.shape[0], k), -1, dtype=np.int64)
+        lp = np.full((Z.shape[0], k), -np.inf)
+        for t in range(Z.shape[0]):
+            order = np.lexsort((np.arange(V), -Z[t]))[:k]      # by logit, descending; ties by class index
+            cls[t, : len(order)] = order
+            lp[t, : len(order)] = logp[t, order]
+        classes.append(cls)
+        logprobs.append(lp)
+    return classes, logprobs
+
+
 def discarded_mass(loss_beam, loss_exact):
     """Delta_n = L_beta,n - L_n and delta_n = 1 - exp(-Delta_n)  (Appendix B.3)."""
     delta_big = np.asarray(loss_beam, dtype=np.float64) - np.asarray(loss_exact, dtype=np.float64)

@@ -23,7 +23,7 @@ UTT_INFEASIBLE, UTT_NONFINITE, UTT_BAD_TARGET, UTT_SUBSET_OVERFLOW = 1, 2, 4, 8
 EXPORTS = ("pctc_workspace_bytes", "pctc_chunk_width", "pruned_ctc_fwd_bwd", "pruned_ctc_fwd_bwd_traced", "pctc_gemm_bf16",
            "pctc_workspace_status", "pctc_status_string", "pctc_host_call_scratch_bytes",
            "pruned_ctc_fwd_bwd_host", "pctc_subset_relabel_noalloc", "pctc_greedy_workspace_bytes",
-           "pctc_greedy_decode")
+           "pctc_greedy_decode", "pctc_topk_workspace_bytes", "pctc_topk_decode")
 NOALLOC_MAX_V = 262144
 
 PHASES = ("prep", "lse", "subset_logp", "dp", "dlogits", "dh", "dw", "dbias", "finish")
@@ -125,6 +125,12 @@ def _configure(lib: ctypes.CDLL) -> ctypes.CDLL:
     lib.pctc_greedy_workspace_bytes.argtypes = [ctypes.POINTER(Problem), i32p, ctypes.POINTER(ctypes.c_size_t)]
     lib.pctc_greedy_decode.restype = ctypes.c_int
     lib.pctc_greedy_decode.argtypes = [ctypes.POINTER(Problem), vp, vp, vp, i32p, vp, vp, vp, vp, ctypes.c_size_t, vp]
+    lib.pctc_topk_workspace_bytes.restype = ctypes.c_int
+    lib.pctc_topk_workspace_bytes.argtypes = [ctypes.POINTER(Problem), i32p, ctypes.c_int32,
+                                              ctypes.POINTER(ctypes.c_size_t)]
+    lib.pctc_topk_decode.restype = ctypes.c_int
+    lib.pctc_topk_decode.argtypes = [ctypes.POINTER(Problem), vp, vp, vp, i32p, ctypes.c_int32, vp, vp, vp,
+                                     ctypes.c_size_t, vp]
     lib.pctc_gemm_bf16.restype = ctypes.c_int
     lib.pctc_gemm_bf16.argtypes = [vp, vp, vp, ctypes.c_int32, ctypes.c_int32, ctypes.c_int32,
                                    ctypes.c_int32, ctypes.c_int32, ctypes.c_int32, vp, vp]
@@ -392,3 +398,33 @@ def greedy_decode(hidden, W, bias, input_lengths, blank_id, *, gemm_path=GEMM_AU
     if st != 0:
         raise PctcError(st, "pctc_greedy_decode")
     return dict(frame_labels=frame_labels, tokens=tokens, token_lengths=token_lengths, workspace=workspace)
+
+
+def topk_decode(hidden, W, bias, input_lengths, k, *, chunk=0, gemm_path=GEMM_AUTO, workspace=None):
+    """The k best classes of every frame (k in 1, 2, 4, 8) and their log-probabilities under the
+    full-vocabulary softmax: device tensors classes [N,T,k] int32 (-1 on padded frames) and logprobs
+    [N,T,k] fp32 (-inf there), plus the reusable workspace."""
+    import torch
+
+    lib = load()
+    dt = PCTC_BF16 if hidden.dtype == torch.bfloat16 else PCTC_FP32
+    N, T, D = hidden.shape
+    V = W.shape[0]
+    il = _i32(input_lengths)
+    prob = make_problem(N, T, D, V, dt, 0, chunk=chunk, gemm_path=gemm_path)
+    need = ctypes.c_size_t(0)
+    st = lib.pctc_topk_workspace_bytes(ctypes.byref(prob), _ptr_i32(il), int(k), ctypes.byref(need))
+    if st != 0:
+        raise PctcError(st, "pctc_topk_workspace_bytes")
+    dev = hidden.device
+    if workspace is None or workspace.numel() < need.value:
+        workspace = torch.empty(need.value, dtype=torch.uint8, device=dev)
+    classes = torch.empty((N, T, k), dtype=torch.int32, device=dev)
+    logprobs = torch.empty((N, T, k), dtype=torch.float32, device=dev)
+    stream = ctypes.c_void_p(torch.cuda.current_stream(dev).cuda_stream)
+    st = lib.pctc_topk_decode(ctypes.byref(prob), _dptr(hidden), _dptr(W), _dptr(bias), _ptr_i32(il), int(k),
+                              _dptr(classes), _dptr(logprobs), _dptr(workspace), ctypes.c_size_t(workspace.numel()),
+                              stream)
+    if st != 0:
+        raise PctcError(st, "pctc_topk_decode")
+    return dict(classes=classes, logprobs=logprobs, workspace=workspace)

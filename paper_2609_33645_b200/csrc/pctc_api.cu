@@ -749,6 +749,87 @@ pctc_status_t pruned_ctc_fwd_bwd_host(const pctc_problem_t* p, const void* hidde
   return PCTC_OK;
 }
 
+namespace {
+struct TopkPlan {
+  GreedyPlan g;
+  int k, chunk;
+  size_t o_logits, o_val, o_idx, o_ms, total;
+};
+pctc_status_t topk_plan(const pctc_problem_t* p, const int32_t* Tn, int32_t k, TopkPlan* t) {
+  pctc_status_t st = greedy_plan(p, Tn, &t->g);
+  if (st != PCTC_OK) return st;
+  if (k != 1 && k != 2 && k != 4 && k != 8) return PCTC_ERR_INVALID_ARG;
+  if (p->chunk < 0) return PCTC_ERR_INVALID_ARG;
+  t->k = k;
+  long long chunk = p->chunk > 0 ? p->chunk : 4096;
+  if (chunk > t->g.V) chunk = t->g.V;
+  t->chunk = (int)((chunk + 3) / 4 * 4);                      // row pitch of the fp32 block: 16-byte rows
+  size_t o = t->g.o_partial;                                  // the arg-max partials are not needed here
+  auto take = [&](size_t bytes) { size_t r = o; o = up(o + bytes); return r; };
+  t->o_logits = take((size_t)t->g.M * t->chunk * 4);
+  t->o_val = take((size_t)t->g.M * k * 4);
+  t->o_idx = take((size_t)t->g.M * k * 4);
+  t->o_ms = take((size_t)t->g.M * 8);
+  t->total = o;
+  return PCTC_OK;
+}
+}  // namespace
+
+pctc_status_t pctc_topk_workspace_bytes(const pctc_problem_t* problem, const int32_t* input_lengths_host, int32_t k,
+                                        size_t* bytes_out) {
+  if (!bytes_out) return PCTC_ERR_INVALID_ARG;
+  TopkPlan t;
+  pctc_status_t st = topk_plan(problem, input_lengths_host, k, &t);
+  if (st != PCTC_OK) return st;
+  *bytes_out = t.total;
+  return PCTC_OK;
+}
+
+pctc_status_t pctc_topk_decode(const pctc_problem_t* p, const void* hidden, const void* W, const void* bias,
+                               const int32_t* input_lengths, int32_t k, int32_t* topk_classes, float* topk_logprobs,
+                               void* workspace, size_t workspace_bytes, void* stream_v) {
+  TopkPlan t;
+  pctc_status_t st = topk_plan(p, input_lengths, k, &t);
+  if (st != PCTC_OK) return st;
+  const GreedyPlan& g = t.g;
+  if (!hidden || !W || !topk_classes || !workspace) return PCTC_ERR_INVALID_ARG;
+  if (workspace_bytes < t.total) return PCTC_ERR_WORKSPACE_TOO_SMALL;
+  if (((size_t)workspace & (ALIGN - 1)) || ((size_t)hidden & 15) || ((size_t)W & 15)) return PCTC_ERR_INVALID_ARG;
+  if (g.use_umma && !umma_available()) return PCTC_ERR_CUDA;
+  cudaStream_t stream = (cudaStream_t)stream_v;
+  if (stream_is_capturing(stream)) return PCTC_ERR_UNSUPPORTED;
+  char* ws = (char*)workspace;
+  const int N = g.N, M = g.M, D = g.D;
+#define PCTC_CUDA(call)                              \
+  do {                                               \
+    if ((call) != cudaSuccess) return PCTC_ERR_CUDA; \
+  } while (0)
+  int* d_meta = (int*)(ws + g.o_meta);
+  int* d_status = (int*)(ws + g.o_status);
+  PCTC_CUDA(batch_meta(input_lengths, nullptr, N, d_meta, nullptr, d_meta + N, nullptr, nullptr, d_meta + 2 * N + 1,
+                       stream));
+  PCTC_CUDA(cudaMemsetAsync(d_status, 0, 256, stream));
+  void* d_X = ws + g.o_X;
+  float* d_logits = (float*)(ws + t.o_logits);
+  float* d_val = (float*)(ws + t.o_val);
+  int* d_idx = (int*)(ws + t.o_idx);
+  float2* d_ms = (float2*)(ws + t.o_ms);
+  PCTC_CUDA(stack_frames(hidden, d_X, N, g.T, D, g.elem, d_meta + 2 * N + 1, d_meta + N, M, d_status, stream));
+  for (long long v0 = 0; v0 < g.V; v0 += t.chunk) {          // the head in vocabulary chunks, logits never kept
+    const int Cc = (int)((g.V - v0 < t.chunk) ? (g.V - v0) : t.chunk);
+    Epilogue e;
+    e.kind = EPI_STORE_F32;
+    e.out = d_logits;
+    e.ld = t.chunk;
+    GemmCall c{d_X, D, false, (const char*)W + (size_t)v0 * D * g.elem, D, false, M, Cc, D};
+    PCTC_CUDA(run_gemm(g.use_umma, g.bf16, c, e, d_status, stream));
+    PCTC_CUDA(topk_update(k, d_logits, t.chunk, M, Cc, v0, bias, g.bf16, d_val, d_idx, d_ms, v0 == 0, stream));
+  }
+  PCTC_CUDA(topk_finish(k, d_val, d_idx, d_ms, d_meta + N, d_meta, N, g.T, topk_classes, topk_logprobs, stream));
+#undef PCTC_CUDA
+  return PCTC_OK;
+}
+
 pctc_status_t pctc_greedy_workspace_bytes(const pctc_problem_t* problem, const int32_t* input_lengths_host,
                                           size_t* bytes_out) {
   if (!bytes_out) return PCTC_ERR_INVALID_ARG;

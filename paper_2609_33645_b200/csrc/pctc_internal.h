@@ -106,6 +106,16 @@ cudaError_t argmax_combine(const float2* partial, int nparts, int M, int* labels
 cudaError_t greedy_collapse(const int* labels, const int* row0, const int* T_n, int N, int T, int blank,
                             int* frame_labels, int* tokens, int* token_lengths, cudaStream_t stream);
 
+// The k best classes per stacked frame (k in {1, 2, 4, 8}), chunk by chunk: `logits` is an fp32
+// [M, ld] block holding columns v0 .. v0+cols-1 of X W^T (bias, if any, is added here); run_val/run_idx
+// [M, k] and run_ms [M] (max, sum of exponentials) carry the state between chunks (first: start afresh).
+// Order: larger logit first, smaller class index among equals.
+cudaError_t topk_update(int k, const float* logits, long long ld, int M, int cols, long long v0, const void* bias,
+                        bool bias_bf16, float* run_val, int* run_idx, float2* run_ms, bool first, cudaStream_t stream);
+// classes [N,T,k] (-1 on padded frames) and log-probabilities [N,T,k] (may be null) from that state
+cudaError_t topk_finish(int k, const float* run_val, const int* run_idx, const float2* run_ms, const int* row0,
+                        const int* T_n, int N, int T, int* classes, float* logprobs, cudaStream_t stream);
+
 // Combine LSE partials: lambda[i] = log sum over splits.
 cudaError_t lse_combine(const float2* partial, int nsplit, int M, float* lambda, cudaStream_t stream);
 

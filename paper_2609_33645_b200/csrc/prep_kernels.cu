@@ -310,6 +310,115 @@ __global__ void k_argmax_combine(const float2* __restrict__ partial, int nparts,
   labels[i] = (idx == 0x7fffffff) ? 0 : idx;
 }
 
+// --- recognition: the k best classes of every frame with their log-probabilities ------------------
+// One warp per stacked frame and vocabulary chunk.  Every lane scans its share of the chunk's logits
+// keeping its own k best (sorted, in registers) and a running (max, sum of exponentials); the lanes'
+// lists, seeded with the frame's k best of the earlier chunks, are then merged by k rounds of a warp-wide
+// arg-max.  Order: larger logit first, among equal logits the smaller class index (the rule of the
+// frame arg-max above), so the result does not depend on the chunk width.
+__device__ __forceinline__ bool topk_before(float av, int ai, float bv, int bi) {
+  return av > bv || (av == bv && ai < bi);
+}
+
+template <int K, typename TB>
+__global__ void k_topk_update(const float* __restrict__ logits, long long ld, int M, int cols, long long v0,
+                              const TB* __restrict__ bias, float* __restrict__ run_val, int* __restrict__ run_idx,
+                              float2* __restrict__ run_ms, int first) {
+  const int m = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
+  const int lane = threadIdx.x & 31;
+  if (m >= M) return;
+  float val[K];
+  int idx[K];
+#pragma unroll
+  for (int r = 0; r < K; ++r) { val[r] = -CUDART_INF_F; idx[r] = 0x7fffffff; }
+  auto insert = [&](float z, int j) {
+    if (!topk_before(z, j, val[K - 1], idx[K - 1])) return;
+    val[K - 1] = z; idx[K - 1] = j;
+#pragma unroll
+    for (int r = K - 1; r > 0; --r) {
+      if (topk_before(val[r], idx[r], val[r - 1], idx[r - 1])) {
+        const float tv = val[r]; val[r] = val[r - 1]; val[r - 1] = tv;
+        const int ti = idx[r]; idx[r] = idx[r - 1]; idx[r - 1] = ti;
+      }
+    }
+  };
+  if (!first && lane < K) insert(run_val[(size_t)m * K + lane], run_idx[(size_t)m * K + lane]);
+  float mx = -CUDART_INF_F, sum = 0.f;
+  const float* row = logits + (size_t)m * ld;
+  for (int j = lane; j < cols; j += 32) {
+    float z = row[j];
+    if (bias) z += float(bias[v0 + j]);
+    if (z > mx) { sum = sum * __expf(mx - z) + 1.f; mx = z; }      // exp(-inf) = 0 at the first logit
+    else sum += __expf(z - mx);                                   // a NaN logit makes the sum NaN
+    insert(z, (int)(v0 + j));
+  }
+  // merge the 32 sorted lists: K rounds, each takes the best head and pops it in the lane that held it
+  float out_v = -CUDART_INF_F;
+  int out_i = 0x7fffffff;
+#pragma unroll
+  for (int r = 0; r < K; ++r) {
+    float bv = val[0];
+    int bi = idx[0];
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) {
+      const float ov = __shfl_xor_sync(0xffffffffu, bv, o);
+      const int oi = __shfl_xor_sync(0xffffffffu, bi, o);
+      if (topk_before(ov, oi, bv, bi)) { bv = ov; bi = oi; }
+    }
+    if (lane == r) { out_v = bv; out_i = bi; }
+    if (idx[0] == bi && bi != 0x7fffffff) {        // class indices are distinct across lanes: one lane pops
+#pragma unroll
+      for (int q = 0; q + 1 < K; ++q) { val[q] = val[q + 1]; idx[q] = idx[q + 1]; }
+      val[K - 1] = -CUDART_INF_F; idx[K - 1] = 0x7fffffff;
+    }
+  }
+  if (lane < K) { run_val[(size_t)m * K + lane] = out_v; run_idx[(size_t)m * K + lane] = out_i; }
+  // running normaliser: combine the lanes' (max, sum) pairs, then the earlier chunks'
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) {
+    const float om = __shfl_xor_sync(0xffffffffu, mx, o), os = __shfl_xor_sync(0xffffffffu, sum, o);
+    const float nm = fmaxf(mx, om);
+    if (nm == -CUDART_INF_F) { sum = sum + os; }                   // both empty (or NaN sums pass through)
+    else { sum = sum * __expf(mx - nm) + os * __expf(om - nm); }
+    mx = nm;
+  }
+  if (lane == 0) {
+    if (!first) {
+      const float2 p = run_ms[m];
+      const float nm = fmaxf(mx, p.x);
+      if (nm != -CUDART_INF_F) sum = sum * __expf(mx - nm) + p.y * __expf(p.x - nm);
+      else sum += p.y;
+      mx = nm;
+    }
+    run_ms[m] = make_float2(mx, sum);
+  }
+}
+
+// classes [N,T,K] and log-probabilities [N,T,K] of the padded layout; padded frames and ranks beyond V
+// read class -1 and log-probability -inf
+template <int K>
+__global__ void k_topk_finish(const float* __restrict__ run_val, const int* __restrict__ run_idx,
+                              const float2* __restrict__ run_ms, const int* __restrict__ row0,
+                              const int* __restrict__ T_n, int N, int T, int* __restrict__ classes,
+                              float* __restrict__ logprobs) {
+  const int i = blockIdx.x * blockDim.x + threadIdx.x;          // (n, t, r)
+  if (i >= N * T * K) return;
+  const int r = i % K, nt = i / K, t = nt % T, n = nt / T;
+  int cls = -1;
+  float lp = -CUDART_INF_F;
+  if (t < T_n[n]) {
+    const size_t m = (size_t)row0[n] + t;
+    const int j = run_idx[m * K + r];
+    if (j != 0x7fffffff) {
+      const float2 p = run_ms[m];
+      cls = j;
+      lp = run_val[m * K + r] - (p.x + logf(p.y));
+    }
+  }
+  classes[i] = cls;
+  if (logprobs) logprobs[i] = lp;
+}
+
 // One warp per utterance, 32 frames at a time: a frame emits its label iff the label is not blank
 // and differs from the previous frame's label.
 __global__ void k_greedy_collapse(const int* __restrict__ labels, const int* __restrict__ row0,
@@ -338,6 +447,47 @@ __global__ void k_greedy_collapse(const int* __restrict__ labels, const int* __r
 
 cudaError_t argmax_combine(const float2* partial, int nparts, int M, int* labels, cudaStream_t stream) {
   k_argmax_combine<<<(M + 127) / 128, 128, 0, stream>>>(partial, nparts, M, labels);
+  return cudaGetLastError();
+}
+
+namespace {
+template <int K>
+cudaError_t topk_update_k(const float* logits, long long ld, int M, int cols, long long v0, const void* bias,
+                          bool bias_bf16, float* run_val, int* run_idx, float2* run_ms, bool first, cudaStream_t stream) {
+  const int warps = 8;
+  const dim3 grid((M + warps - 1) / warps), block(warps * 32);
+  if (bias_bf16)
+    k_topk_update<K, __nv_bfloat16><<<grid, block, 0, stream>>>(logits, ld, M, cols, v0, (const __nv_bfloat16*)bias,
+                                                               run_val, run_idx, run_ms, first ? 1 : 0);
+  else
+    k_topk_update<K, float><<<grid, block, 0, stream>>>(logits, ld, M, cols, v0, (const float*)bias, run_val, run_idx,
+                                                       run_ms, first ? 1 : 0);
+  return cudaGetLastError();
+}
+}  // namespace
+
+cudaError_t topk_update(int k, const float* logits, long long ld, int M, int cols, long long v0, const void* bias,
+                        bool bias_bf16, float* run_val, int* run_idx, float2* run_ms, bool first, cudaStream_t stream) {
+  switch (k) {
+    case 1: return topk_update_k<1>(logits, ld, M, cols, v0, bias, bias_bf16, run_val, run_idx, run_ms, first, stream);
+    case 2: return topk_update_k<2>(logits, ld, M, cols, v0, bias, bias_bf16, run_val, run_idx, run_ms, first, stream);
+    case 4: return topk_update_k<4>(logits, ld, M, cols, v0, bias, bias_bf16, run_val, run_idx, run_ms, first, stream);
+    case 8: return topk_update_k<8>(logits, ld, M, cols, v0, bias, bias_bf16, run_val, run_idx, run_ms, first, stream);
+  }
+  return cudaErrorInvalidValue;
+}
+
+cudaError_t topk_finish(int k, const float* run_val, const int* run_idx, const float2* run_ms, const int* row0,
+                        const int* T_n, int N, int T, int* classes, float* logprobs, cudaStream_t stream) {
+  const long long total = (long long)N * T * k;
+  const int blocks = (int)((total + 255) / 256);
+  switch (k) {
+    case 1: k_topk_finish<1><<<blocks, 256, 0, stream>>>(run_val, run_idx, run_ms, row0, T_n, N, T, classes, logprobs); break;
+    case 2: k_topk_finish<2><<<blocks, 256, 0, stream>>>(run_val, run_idx, run_ms, row0, T_n, N, T, classes, logprobs); break;
+    case 4: k_topk_finish<4><<<blocks, 256, 0, stream>>>(run_val, run_idx, run_ms, row0, T_n, N, T, classes, logprobs); break;
+    case 8: k_topk_finish<8><<<blocks, 256, 0, stream>>>(run_val, run_idx, run_ms, row0, T_n, N, T, classes, logprobs); break;
+    default: return cudaErrorInvalidValue;
+  }
   return cudaGetLastError();
 }
 

@@ -110,3 +110,19 @@ def test_fwd_bwd_rejects_null_and_short_workspace_before_any_launch(lib):
     args[1] = None
     assert cdll.pruned_ctc_fwd_bwd(*args) == 1          # null hidden
     assert cdll.pctc_gemm_bf16(None, fake, fake, 8, 8, 8, 0, 0, 0, None, None) == 1
+
+
+def test_topk_workspace_query_validates_k_and_has_no_frames_by_vocabulary_term(lib):
+    il = np.array([50, 40], dtype=np.int32)
+    ptr = il.ctypes.data_as(ctypes.POINTER(ctypes.c_int32))
+    out = ctypes.c_size_t(0)
+    cdll = lib.load()
+    prob = _prob(lib, dtype=0, D=512, V=180000)
+    for k in (0, 3, 5, 16, -1):
+        assert cdll.pctc_topk_workspace_bytes(ctypes.byref(prob), ptr, k, ctypes.byref(out)) == 1
+    sizes = []
+    for V in (180000, 90000):
+        p = _prob(lib, dtype=0, D=512, V=V)
+        assert cdll.pctc_topk_workspace_bytes(ctypes.byref(p), ptr, 8, ctypes.byref(out)) == 0
+        sizes.append(out.value)
+    assert sizes[0] == sizes[1] < 90 * 180000          # one 4,096-column block of logits, whatever V

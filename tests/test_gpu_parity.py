@@ -573,3 +573,51 @@ def test_tall_dw_tiles_ragged_chunk_and_accumulation(lib):
     out = lib.pruned_ctc_fwd_bwd(*args, chunk=16384, accumulate_dW=True, workspace=out["workspace"], out=out)
     torch.cuda.synchronize()
     assert H.rel_fro(out["dW"].float().cpu().numpy(), 2.0 * ref["dW"]) <= 1e-2
+
+
+@pytest.mark.parametrize("path,dtype,k,chunk", [(SIMT, "fp32", 4, 300), (SIMT, "bf16", 8, 0), (AUTO, "bf16", 8, 1024),
+                                                (AUTO, "bf16", 1, 0), (AUTO, "bf16", 2, 4096)])
+def test_topk_recognition_matches_oracle(lib, path, dtype, k, chunk):
+    """The k best classes of every frame and their log-probabilities (the per-frame input of a prefix beam
+    search): classes must agree with the oracle wherever the oracle's neighbouring ranks are not near-ties,
+    log-probabilities rank by rank."""
+    import torch
+    from oracle import pruned_ctc_oracle as O
+    if dtype == "fp32":
+        cfg = dataclasses.replace(wl.CONFIGS["c1"], name="tk32", N=3, T_lo=10, T_hi=40, V=1531, D=72, seed=21)
+    else:
+        cfg = small("c3", V=9000 + 37, D=256, N=3, T_div=6)
+    batch = wl.make_batch(cfg, with_bias=True, poison_padding=True)
+    dev = torch.device("cuda:0")
+    tdt = torch.bfloat16 if dtype == "bf16" else torch.float32
+    hidden = torch.from_numpy(batch.hidden).to(dev).to(tdt)
+    W = torch.from_numpy(batch.W).to(dev).to(tdt)
+    bias = torch.from_numpy(batch.bias).to(dev).to(tdt)
+    res = lib.topk_decode(hidden, W, bias, batch.input_lengths, k, chunk=chunk, gemm_path=path)
+    torch.cuda.synchronize()
+    cls_g = res["classes"].cpu().numpy()
+    lp_g = res["logprobs"].cpu().numpy().astype(np.float64)
+    cls_r, lp_r = O.topk_decode(batch.hidden, batch.W, batch.bias, batch.input_lengths, k)
+    # full top-(k+1) of the oracle gives the gap below the last rank too
+    _, lp_r1 = O.topk_decode(batch.hidden, batch.W, batch.bias, batch.input_lengths, k + 1)
+    tol = 1e-4 if dtype == "fp32" else 2e-3
+    checked = 0
+    for n in range(cfg.N):
+        Tn = int(batch.input_lengths[n])
+        assert np.all(cls_g[n, Tn:] == -1) and np.all(np.isneginf(lp_g[n, Tn:]))
+        np.testing.assert_allclose(lp_g[n, :Tn], lp_r[n], atol=tol, rtol=0)      # rank by rank
+        gaps = -np.diff(lp_r1[n], axis=1)                                        # [Tn, k]: rank r to rank r+1
+        for t in range(Tn):
+            for r in range(k):
+                clear = gaps[t, r] > 4 * tol and (r == 0 or gaps[t, r - 1] > 4 * tol)
+                if clear:
+                    assert cls_g[n, t, r] == cls_r[n][t, r], (n, t, r)
+                    checked += 1
+    assert checked > 0.9 * k * batch.M
+    # rank one is the greedy decoder's label
+    greedy = lib.greedy_decode(hidden, W, bias, batch.input_lengths, 0, gemm_path=path)
+    fl = greedy["frame_labels"].cpu().numpy()
+    for n in range(cfg.N):
+        Tn = int(batch.input_lengths[n])
+        same = fl[n, :Tn] == cls_g[n, :Tn, 0]
+        assert same.mean() > 0.98          # the two take their maxima over different chunkings of V: near-ties may differ

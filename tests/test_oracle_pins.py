@@ -444,3 +444,35 @@ def test_collapse_map_and_greedy_decode():
     # a bias can overturn the projection's winner
     frames, _, _ = O.greedy_decode(np.array([[[2.0, 0.0]]]), W2, np.array([0.0, 0.0, 0.0, 1.5]), [1], 0)
     assert list(frames[0]) == [3]
+
+
+def test_topk_decode_against_planted_answers():
+    # orthonormal class vectors; a frame is 4 q_a + 2 q_b + 1 q_c + noise, so its three best classes are
+    # a, b, c in that order by construction, with logits close to 4, 2, 1 and all others close to 0
+    rng = np.random.default_rng(11)
+    V = D = 12
+    Q, _ = np.linalg.qr(rng.standard_normal((D, D)))
+    triples = [[(3, 7, 1), (0, 2, 11), (5, 4, 9), (9, 0, 3)], [(8, 1, 2), (6, 10, 0)]]
+    Hp = np.zeros((2, 4, D))
+    for n, frames in enumerate(triples):
+        for t, (a, b, c) in enumerate(frames):
+            Hp[n, t] = 4.0 * Q[a] + 2.0 * Q[b] + 1.0 * Q[c] + 0.01 * rng.standard_normal(D)
+    cls, lp = O.topk_decode(Hp, Q, None, [4, 2], 4)
+    for n, frames in enumerate(triples):
+        assert [tuple(r[:3]) for r in cls[n]] == frames
+        # log-probabilities: decreasing, differences equal to the planted logit gaps, and consistent with
+        # a softmax that sums to one over all classes
+        assert np.all(np.diff(lp[n], axis=1) <= 0)
+        np.testing.assert_allclose(lp[n][:, 0] - lp[n][:, 1], 2.0, atol=0.05)
+        np.testing.assert_allclose(lp[n][:, 1] - lp[n][:, 2], 1.0, atol=0.05)
+        full_cls, full_lp = O.topk_decode(Hp[n:n + 1], Q, None, [len(frames)], V)
+        np.testing.assert_allclose(np.exp(full_lp[0]).sum(axis=1), 1.0, rtol=1e-12)
+        assert sorted(full_cls[0][0]) == list(range(V))
+    # rank one is the greedy decoder's frame label
+    frames_greedy, _, _ = O.greedy_decode(Hp, Q, None, [4, 2], 0)
+    for n in range(2):
+        assert list(cls[n][:, 0]) == list(frames_greedy[n])
+    # equal logits: the smaller class index first; more ranks than classes: -1 and -inf
+    W2 = np.array([[1.0, 0.0], [1.0, 0.0], [0.0, 1.0]])
+    cls, lp = O.topk_decode(np.array([[[2.0, 1.0]]]), W2, None, [1], 4)
+    assert list(cls[0][0]) == [0, 1, 2, -1] and lp[0][0, 3] == -np.inf and lp[0][0, 0] == lp[0][0, 1]

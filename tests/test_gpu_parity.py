@@ -621,3 +621,23 @@ def test_topk_recognition_matches_oracle(lib, path, dtype, k, chunk):
         Tn = int(batch.input_lengths[n])
         same = fl[n, :Tn] == cls_g[n, :Tn, 0]
         assert same.mean() > 0.98          # the two take their maxima over different chunkings of V: near-ties may differ
+
+
+@pytest.mark.parametrize("path", [SIMT, AUTO])
+def test_more_utterances_than_one_length_slice(lib, path):
+    """2,100 very short utterances: the lengths reach the device in three kernel-parameter slices of 1,024,
+    and the prefix sums over the utterances run over more than one utterance per thread."""
+    cfg = wl.Config("manyutt", N=2100, T_lo=2, T_hi=6, D=16, V=96, dtype="bf16", U_lo=0, U_hi=3, zipf_s=1.1, seed=4242)
+    batch = wl.make_batch(cfg, poison_padding=True)
+    gpu = H.run_gpu(lib, batch, gemm_path=path)
+    ref = H.run_oracle(batch)
+    assert (ref["flags"] == 1).any() and (ref["flags"] == 0).any()      # some utterances have too few frames
+    H.assert_parity(gpu, ref, batch)
+    import torch
+    dev = torch.device("cuda:0")
+    greedy = lib.greedy_decode(torch.from_numpy(batch.hidden).to(dev).to(torch.bfloat16),
+                               torch.from_numpy(batch.W).to(dev).to(torch.bfloat16), None, batch.input_lengths, 0,
+                               gemm_path=path)
+    fl = greedy["frame_labels"].cpu().numpy()
+    for n in (0, 1023, 1024, 2047, 2048, 2099):
+        assert np.all(fl[n, : batch.input_lengths[n]] >= 0) and np.all(fl[n, batch.input_lengths[n]:] == -1)

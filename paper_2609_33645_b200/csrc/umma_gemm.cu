@@ -80,6 +80,10 @@ constexpr bool PROBE_SKIP_A = (PCTC_PROBE & 8) != 0;
 #define PCTC_TUNE_CHUNK_HINT 0    // L2 eviction priority for the bf16 dlogits chunk: bit 0 evict-first on its stores
 #endif                            // (dlogits), bit 1 evict-first on its loads (A operand of the dX and dW kernels)
 
+#ifndef PCTC_TUNE_PDL
+#define PCTC_TUNE_PDL 0           // 1: programmatic dependent launch: a contraction kernel's CTAs may start and set up
+#endif                            // (barriers, tensor memory) while the kernel before it in the stream drains
+
 #ifndef PCTC_TUNE_EPI_WARPS
 #define PCTC_TUNE_EPI_WARPS 0     // 0: by the contraction depth; 4 or 8: forced
 #endif
@@ -470,6 +474,11 @@ k_umma_gemm(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
   const int rank = (CTAS == 2) ? (int)cluster_ctarank() : 0;     // position inside the pair
   const int group = blockIdx.x / CTAS, ngroups = gridDim.x / CTAS;
 
+  // With programmatic dependent launch this CTA may be running before the kernel ahead of it in the
+  // stream has finished: nothing that kernel wrote may be read, and nothing it reads may be overwritten,
+  // before griddepcontrol.wait.  The set-up below touches shared and tensor memory only, except for the
+  // selected-class count, which the kernel ahead may still be writing.
+  if (PCTC_TUNE_PDL && EPI == EPI_SUBSET_LOGP) asm volatile("griddepcontrol.wait;" ::: "memory");
   // problem decomposition, identical in every role
   int n_eff = a.n;
   if (EPI == EPI_SUBSET_LOGP) n_eff = min(a.n, *a.e.Kdev);
@@ -507,6 +516,10 @@ k_umma_gemm(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
   tc_fence_after();
   const unsigned tmem_base = st->tmem_base;
   volatile int* abort_flag = &st->abort;
+  if (PCTC_TUNE_PDL) {
+    asm volatile("griddepcontrol.wait;" ::: "memory");                 // the kernels ahead are complete and visible
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");    // the next one may set up as SMs free up
+  }
 
   if (warp == 0) {
     // ===================== TMA producer =====================
@@ -1040,17 +1053,19 @@ cudaError_t launch_ew(const CUtensorMap& tmA, const CUtensorMap& tmB, const CUte
     cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)SMEM);
     if (e != cudaSuccess) return e;
   }
-  cudaLaunchAttribute attr[1];
+  cudaLaunchAttribute attr[2];
   attr[0].id = cudaLaunchAttributeClusterDimension;
   attr[0].val.clusterDim.x = CTAS_DEFAULT;
   attr[0].val.clusterDim.y = 1;
   attr[0].val.clusterDim.z = 1;
+  attr[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[1].val.programmaticStreamSerializationAllowed = 1;
   cudaLaunchConfig_t cfg = {};
   cfg.blockDim = dim3(num_threads(EW));
   cfg.dynamicSmemBytes = SMEM;
   cfg.stream = stream;
   cfg.attrs = attr;
-  cfg.numAttrs = 1;
+  cfg.numAttrs = PCTC_TUNE_PDL ? 2 : 1;
   if (max_groups == 0) {
     cfg.gridDim = dim3((unsigned)(sm_count() / CTAS_DEFAULT * CTAS_DEFAULT));
     int n = 0;

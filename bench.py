@@ -492,9 +492,10 @@ def main():
         traffic = load_traffic(cfg.name, chunk)
 
     # kernels launched by the library inside the timed region
-    dp_launches = 4 if args.beam > 0 else 2      # sweeps (+ best-alignment sweeps, arc flags), occupancies
-    # subset (3), stacking, gather + Z_U, DP, normaliser + combine, loss, row clean-up, chunks, un-stacking
-    launches_per_step = (3 + 1 + 2 + dp_launches + 2 + 1 + 1 + (2 if args.frozen_head else 3) * nchunks + 1
+    dp_launches = 5 if args.beam > 0 else 3      # sweeps (+ best-alignment sweeps, arc flags), label chains, occupancies
+    # batch tables (3), subset (3), stacking, gather + Z_U, DP, normaliser + combine, loss, row clean-up, chunks,
+    # un-stacking
+    launches_per_step = (3 + 3 + 1 + 2 + dp_launches + 2 + 1 + 1 + (2 if args.frozen_head else 3) * nchunks + 1
                         + (nchunks if args.bias else 0))          # + column sums for dbias
     gpu_launches = launches_per_step * args.steps
 

@@ -189,7 +189,7 @@ def time_config(binding, torch, dev, cfg, beam, steps, warmup, peaks):
 
 
 def print_table(path: str) -> int:
-    """Markdown rows of the `all_configs` block of a saved bench line (the results table of the design notes)."""
+    """Markdown rows of the `all_configs` block of a saved bench line."""
     line = None
     with open(path) as f:
         for x in f:

@@ -12,14 +12,12 @@ namespace {
 using namespace pctc;
 
 constexpr size_t ALIGN = 256;
-constexpr size_t DH_SPLIT_EXTRA_BYTES = 128u << 20;   // most that extra dX accumulators may take (narrow heads: k-split)
-constexpr size_t DH_STREAMK_EXTRA_BYTES = 256u << 20;  // ... and the one extra slab of the stream-K form (wide heads)
+constexpr size_t DH_SPLIT_EXTRA_BYTES = 128u << 20;   // most that extra dX accumulators may take
 inline size_t up(size_t x, size_t a = ALIGN) { return (x + a - 1) / a * a; }
 
 struct Plan {
   int N, T, D, M, Usum, Kcap, Lmax, chunk, nsplit, nchunks;
   int ksplit, slab_rows;   // dX accumulator: k-split slabs of slab_rows rows each (1 slab of M rows without)
-  bool streamk;            // dX contraction in stream-K form: two slabs, the second one zeroed per call
   long long V, cells, mcells;
   size_t ldS;
   int elem;          // bytes per element of hidden/W
@@ -135,17 +133,8 @@ pctc_status_t make_plan(const pctc_problem_t* p, const int32_t* Tn, const int32_
   pl->o_colpart = pl->use_umma ? take((size_t)((pl->M + 31) / 32) * pl->chunk * 4) : 0;
   // few output tiles (small M x D): the dX contraction of a chunk is cut along k into ksplit ranges, each
   // with its own fp32 accumulator, summed in a fixed order when dH is written (deterministic)
-  pl->streamk = pl->use_umma && umma_accum_streamk(pl->M, pl->D, pl->chunk) &&
-                (size_t)umma_accum_streamk_slab_rows(pl->M) * pl->D * 4 <= DH_STREAMK_EXTRA_BYTES;
-  if (pl->streamk) {
-    // wide heads: tall tiles, equal shares of k-blocks per CTA pair; a tile is shared by at most two pairs, the
-    // second one's part goes to a second slab
-    pl->ksplit = 2;
-    pl->slab_rows = umma_accum_streamk_slab_rows(pl->M);
-  } else {
-    pl->ksplit = pl->use_umma ? umma_accum_splits(pl->M, pl->D, pl->chunk, DH_SPLIT_EXTRA_BYTES) : 1;
-    pl->slab_rows = pl->ksplit > 1 ? umma_accum_slab_rows(pl->M) : pl->M;
-  }
+  pl->ksplit = pl->use_umma ? umma_accum_splits(pl->M, pl->D, pl->chunk, DH_SPLIT_EXTRA_BYTES) : 1;
+  pl->slab_rows = pl->ksplit > 1 ? umma_accum_slab_rows(pl->M) : pl->M;
   pl->o_dHacc = take((size_t)pl->ksplit * pl->slab_rows * pl->D * 4);
   pl->total = o;
   return PCTC_OK;
@@ -424,8 +413,6 @@ pctc_status_t run_call(const pctc_problem_t* p, const void* hidden, const void* 
     PCTC_MARK(-2);
     PCTC_CUDA(cudaEventRecord(aux.fork, stream));
     PCTC_CUDA(cudaStreamWaitEvent(aux.side, aux.fork, 0));
-    if (pl.streamk && !p->forward_only)          // the second dX slab starts at zero: parts of tiles are added to it
-      PCTC_CUDA(cudaMemsetAsync(d_dHacc + (size_t)pl.slab_rows * D, 0, (size_t)pl.slab_rows * D * 4, aux.side));
     {
       cudaStream_t main_stream = stream;
       stream = aux.side;
@@ -524,15 +511,7 @@ pctc_status_t run_call(const pctc_problem_t* p, const void* hidden, const void* 
       e.out = d_dHacc;
       e.ld = D;
       e.accumulate = ci > 0;
-      if (pl.streamk) {
-        // a short last chunk may not qualify: it then runs tile by tile into the first slab
-        dh_slabs = 2;
-        if (umma_accum_streamk(M, D, Cc)) {
-          e.streamk = 1;
-          e.ksplit = 2;
-          e.ksplit_rows = pl.slab_rows;
-        }
-      } else if (pl.ksplit > 1) {
+      if (pl.ksplit > 1) {
         // the first chunk stores into (and so initialises) its slabs; a shorter chunk later on may
         // cut k into fewer ranges and then adds to the first slabs only
         int s = umma_accum_splits(M, D, Cc, DH_SPLIT_EXTRA_BYTES);

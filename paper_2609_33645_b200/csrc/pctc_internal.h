@@ -68,8 +68,6 @@ struct Epilogue {
   long long ld_colpart = 0;     //   each block of 32 rows of the rounded output (db_c = dZ_c^T 1), or null
   int ksplit = 1;               // EPI_ACCUM_F32 on the tensor-core path: the contraction is cut into this many
   int ksplit_rows = 0;          //   ranges of k; range s accumulates into rows [s * ksplit_rows, ...) of `out`
-  int streamk = 0;              // EPI_ACCUM_F32, tensor-core path: stream-K form (umma_accum_streamk); ksplit must be 2
-                                //   (two slabs, the second one zeroed by the caller before the first chunk)
   long long vocab = 0;          // V, for the index checks of the debug build
   int* status = nullptr;        //   ... and the status word they report to
 };
@@ -97,10 +95,6 @@ int umma_lse_splits(int m, int n);   // column splits (<= 32) for EPI_LSE_PARTIA
 // in total); and the slab height (m rounded up to whole row tiles) that goes with it.
 int umma_accum_splits(int m, int n, int k, size_t max_extra_bytes);
 int umma_accum_slab_rows(int m);
-// Whether the dX contraction of an [m, k] chunk into [m, n] runs in stream-K form on this library's plan (tall
-// tiles, equal shares of k-blocks per CTA pair, two accumulator slabs), and the slab height that goes with it.
-bool umma_accum_streamk(int m, int n, int k);
-int umma_accum_streamk_slab_rows(int m);
 int umma_lse_partials_per_split(int k);   // the kernel writes this many partials per split (1 or 2):
                                           // partial[(i*nsplit + sp)*pps + h]
 

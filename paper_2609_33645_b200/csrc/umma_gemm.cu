@@ -58,10 +58,6 @@ namespace {
 #define PCTC_TUNE_MT2 1           // 1: the dW contraction may use 512 x 256 tiles (see k_umma_gemm, MT)
 #endif
 
-#ifndef PCTC_TUNE_STREAMK
-#define PCTC_TUNE_STREAMK 1       // 1: the dX contraction of a wide head runs on 512 x 256 tiles whose k-blocks are
-#endif                            // dealt to the CTA pairs in equal contiguous shares (see umma_accum_streamk)
-
 #ifndef PCTC_TUNE_CTAS
 #define PCTC_TUNE_CTAS 2          // CTAs per tile: 2 = tcgen05 cta_group::2 pairs, 1 = independent CTAs
 #endif
@@ -124,9 +120,6 @@ struct UmmaArgs {
   int tile_mt;         // host only: 2 = launch the 512-row tile form (store epilogue, long contractions)
   int ksplit;          // EPI_ACCUM_F32: units per output tile, each contracting its own range of k
   int ksplit_rows;     //   ... and writing its own accumulator slab, this many rows further down
-  int streamk;         // EPI_ACCUM_F32: the k-blocks of all tiles, tile after tile, are dealt to the CTA groups in
-                       //   equal contiguous shares; the part of a tile that starts at k = 0 goes to slab 0, a part
-                       //   that starts inside the tile is added to slab 1 (at most one such part per tile)
   int* status;
   Epilogue e;
 };
@@ -495,35 +488,6 @@ k_umma_gemm(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
   const int ksplit = (EPI == EPI_ACCUM_F32) ? a.ksplit : 1;
   const int units = m_tiles * splits * ksplit;
   const int k_blocks = (a.k + BK - 1) / BK;
-  // The units of this CTA group: u = u_first, u_first + u_step, ... < u_end.  Usually every group takes every
-  // ngroups-th unit of the list above.  With stream-K a group owns k-blocks [sk_start, sk_end) of the
-  // sequence "all k-blocks of tile 0, all of tile 1, ..." and its unit u is its share of tile sk_tile0 + u.
-  const bool streamk = (EPI == EPI_ACCUM_F32) && a.streamk != 0;
-  int u_first = group, u_end = units, u_step = ngroups;
-  int sk_start = 0, sk_end = 0, sk_tile0 = 0;
-  if (streamk) {
-    const int total = m_tiles * n_tiles * k_blocks;
-    const int quota = (total + ngroups - 1) / ngroups;
-    sk_start = min(total, group * quota);
-    sk_end = min(total, sk_start + quota);
-    sk_tile0 = sk_start / k_blocks;
-    u_first = 0;
-    u_step = 1;
-    u_end = (sk_end > sk_start) ? ((sk_end - 1) / k_blocks - sk_tile0 + 1) : 0;
-  }
-  auto locate = [&](int u, int& mt, int& sp, int& ks, int& nt0, int& cnt, int& kb0, int& kcnt) {
-    if (streamk) {
-      const int tile = sk_tile0 + u;
-      decode_unit(tile, m_tiles, n_tiles, n_tiles, 1, a.raster_g, mt, sp, ks, nt0, cnt);
-      const int lo = max(sk_start, tile * k_blocks), hi = min(sk_end, (tile + 1) * k_blocks);
-      kb0 = lo - tile * k_blocks;
-      kcnt = hi - lo;
-      ks = kb0 ? 1 : 0;
-    } else {
-      decode_unit(u, m_tiles, n_tiles, splits, ksplit, a.raster_g, mt, sp, ks, nt0, cnt);
-      split_range(k_blocks, ksplit, ks, kb0, kcnt);      // this unit's share of the contraction
-    }
-  };
 
   if (threadIdx.x == 0) {
     for (int s = 0; s < STAGES; ++s) { mbar_init(&st->full[s], 1); mbar_init(&st->empty[s], 1); }
@@ -573,9 +537,10 @@ k_umma_gemm(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
         if (HINT_A) tma_load_2d_pair_hint(dst, map, c0, c1, bar, a_policy);
         else load(dst, map, c0, c1, bar);
       };
-      for (int u = u_first; u < u_end && ok; u += u_step) {
+      for (int u = group; u < units && ok; u += ngroups) {
         int mt, sp, ks, nt0, cnt, kb0, kcnt;
-        locate(u, mt, sp, ks, nt0, cnt, kb0, kcnt);
+        decode_unit(u, m_tiles, n_tiles, splits, ksplit, a.raster_g, mt, sp, ks, nt0, cnt);
+        split_range(k_blocks, ksplit, ks, kb0, kcnt);            // this unit's share of the contraction
         const int row_a = mt * TILE_M + rank * BM;               // this CTA's rows of A
         for (int nt = nt0; nt < nt0 + cnt && ok; ++nt) {
           const int row_b = nt * BN + rank * (BN / CTAS);        // this CTA's columns of the tile (rows of B)
@@ -629,9 +594,10 @@ k_umma_gemm(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
       const unsigned b_step = a.b_mn ? (2048u >> 4) : (32u >> 4);
       unsigned g = 0, it = 0;
       bool ok = true;
-      for (int u = u_first; u < u_end && ok; u += u_step) {
+      for (int u = group; u < units && ok; u += ngroups) {
         int mt, sp, ks, nt0, cnt, kb0, kcnt;
-        locate(u, mt, sp, ks, nt0, cnt, kb0, kcnt);
+        decode_unit(u, m_tiles, n_tiles, splits, ksplit, a.raster_g, mt, sp, ks, nt0, cnt);
+        split_range(k_blocks, ksplit, ks, kb0, kcnt);
         (void)mt;
         for (int nt = nt0; nt < nt0 + cnt && ok; ++nt, ++it) {
           // MT == 1: the two accumulators alternate between tiles.  MT == 2: both belong to this tile
@@ -707,9 +673,9 @@ k_umma_gemm(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
       }
     };
     if (EPI == EPI_DLOGITS && group < units) prefetch(group);
-    for (int u = u_first; u < u_end && ok; u += u_step) {
-      int mt, sp, ks, nt0, cnt, kb0_unused, kcnt_unused;
-      locate(u, mt, sp, ks, nt0, cnt, kb0_unused, kcnt_unused);
+    for (int u = group; u < units && ok; u += ngroups) {
+      int mt, sp, ks, nt0, cnt;
+      decode_unit(u, m_tiles, n_tiles, splits, ksplit, a.raster_g, mt, sp, ks, nt0, cnt);
       const int row0_cta = mt * TILE_M + rank * BM;      // first row of this CTA's half of the tile
       const int row0_out = row0_cta + ks * a.ksplit_rows; // ... and where it lands in the output (k-split slab)
       const int i = row0_cta + r;
@@ -883,8 +849,7 @@ k_umma_gemm(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
                   a.e.colpart[(long long)((row0_cta + q * 32) >> 5) * a.e.ld_colpart + j0 + col] = cs;
               }
               if (lane == 0) {
-                // (a stream-K part that starts inside its tile is always added: its slab starts at zero)
-                if ((EPI == EPI_ACCUM_F32 || EPI == EPI_STORE_OUT) && (a.e.accumulate || (streamk && ks == 1)))
+                if ((EPI == EPI_ACCUM_F32 || EPI == EPI_STORE_OUT) && a.e.accumulate)
                   tma_reduce_add_2d(&tmC, box, j0 + b * 16, row0_out + h * SUB_M + q * 32);
                 else if ((PCTC_TUNE_CHUNK_HINT & 1) && EPI == EPI_DLOGITS)
                   tma_store_2d_hint(&tmC, box, j0 + b * 16, row0_out + h * SUB_M + q * 32, make_evict_first_policy());
@@ -1123,7 +1088,7 @@ inline int epi_warps_for(int k) {
 template <int EPI>
 cudaError_t launch(const CUtensorMap& tmA, const CUtensorMap& tmB, const CUtensorMap& tmC, const UmmaArgs& a,
                    int grid, cudaStream_t stream) {
-  if constexpr ((EPI == EPI_STORE_OUT || EPI == EPI_ACCUM_F32) && CTAS_DEFAULT == 2) {
+  if constexpr (EPI == EPI_STORE_OUT && CTAS_DEFAULT == 2) {
     if (a.tile_mt == 2) return launch_ew<EPI, 4, 2>(tmA, tmB, tmC, a, grid, stream);
   }
   return epi_warps_for(a.k) == 8 ? launch_ew<EPI, 8>(tmA, tmB, tmC, a, grid, stream)
@@ -1177,18 +1142,6 @@ int umma_accum_splits(int m, int n, int k, size_t max_extra_bytes) {
   return best;
 }
 
-// Stream-K form of the dX contraction (EPI_ACCUM_F32): 512 x 256 tiles (25% fewer operand bytes per FLOP than
-// 256 x 256, as in the dW kernel), and instead of whole tiles every CTA pair gets the same number of k-blocks,
-// so no pair idles in a last partial wave.  It needs a long contraction (the epilogue of a tall tile is not
-// overlapped), at least as many tall tiles as CTA pairs (then a tile is shared by at most two pairs: one
-// extra accumulator slab), and is planned for a full B200 wherever it is computed.
-bool umma_accum_streamk(int m, int n, int k) {
-  if (!(PCTC_TUNE_STREAMK && PCTC_TUNE_MT2 && CTAS_DEFAULT == 2)) return false;
-  const long long tall_tiles = (long long)((m + 511) / 512) * ((n + BN - 1) / BN);
-  return k > EW_SWITCH_K && m >= 512 && tall_tiles >= 148 / CTAS_DEFAULT;
-}
-int umma_accum_streamk_slab_rows(int m) { return (m + 511) / 512 * 512; }
-
 cudaError_t umma_gemm(const __nv_bfloat16* A, long long lda, bool a_mn_major,
                       const __nv_bfloat16* B, long long ldb, bool b_mn_major,
                       int m, int n, int k, const Epilogue& e, int* status, cudaStream_t stream) {
@@ -1198,12 +1151,8 @@ cudaError_t umma_gemm(const __nv_bfloat16* A, long long lda, bool a_mn_major,
   bool ok = true;
   tmC = CUtensorMap{};
   // output boxes of the staged epilogues: 32 rows x 32 columns, clipped to the [m, n] extent
-  const bool streamk = e.kind == EPI_ACCUM_F32 && e.streamk != 0;
-  if (streamk && (!umma_accum_streamk(m, n, k) || e.ksplit != 2 || e.ksplit_rows < umma_accum_streamk_slab_rows(m)))
-    return cudaErrorInvalidValue;
-  const int ksplit = (e.kind == EPI_ACCUM_F32 && e.ksplit > 1) ? e.ksplit : 1;      // accumulator slabs
-  if (!streamk && ksplit > 1 && (ksplit > (k + BK - 1) / BK || e.ksplit_rows < umma_accum_slab_rows(m)))
-    return cudaErrorInvalidValue;
+  const int ksplit = (e.kind == EPI_ACCUM_F32 && e.ksplit > 1) ? e.ksplit : 1;
+  if (ksplit > 1 && (ksplit > (k + BK - 1) / BK || e.ksplit_rows < umma_accum_slab_rows(m))) return cudaErrorInvalidValue;
   if (e.kind == EPI_ACCUM_F32 || e.kind == EPI_SUBSET_LOGP) {
     if ((e.ld % 4) || ((size_t)e.out & 15)) return cudaErrorInvalidValue;
     const unsigned long long out_rows = (unsigned long long)(ksplit - 1) * e.ksplit_rows + m;   // k-split slabs stacked
@@ -1223,16 +1172,15 @@ cudaError_t umma_gemm(const __nv_bfloat16* A, long long lda, bool a_mn_major,
   a.a_mn = a_mn_major ? 1 : 0;
   a.b_mn = b_mn_major ? 1 : 0;
   a.nsplit = e.nsplit;
-  a.ksplit = streamk ? 1 : ksplit;
+  a.ksplit = ksplit;
   a.ksplit_rows = ksplit > 1 ? e.ksplit_rows : 0;
-  a.streamk = streamk ? 1 : 0;
   a.status = status;
   a.e = e;
   const int n_tiles = (n + BN - 1) / BN;
   const int groups = sm_count() / CTAS_DEFAULT;
   // 512-row tiles for the dW contraction when its main loop is long (the un-overlapped epilogue is then
   // a small share) and whole waves of the taller tiles cost no more than whole waves of the usual ones
-  a.tile_mt = streamk ? 2 : 1;
+  a.tile_mt = 1;
   if (PCTC_TUNE_MT2 && CTAS_DEFAULT == 2 && e.kind == EPI_STORE_OUT && k > EW_SWITCH_K && m >= 2 * BM * CTAS_DEFAULT) {
     const long long t1 = (long long)((m + 255) / 256) * n_tiles, t2 = (long long)((m + 511) / 512) * n_tiles;
     const long long w1 = (t1 + groups - 1) / groups, w2 = 2 * ((t2 + groups - 1) / groups);
@@ -1252,9 +1200,9 @@ cudaError_t umma_gemm(const __nv_bfloat16* A, long long lda, bool a_mn_major,
     const int bands = (int)((m_tiles + g - 1) / g);
     a.raster_g = (m_tiles + bands - 1) / bands;          // bands of equal height
   }
-  long long units = (long long)m_tiles * (walks ? e.nsplit : n_tiles) * (streamk ? 1 : ksplit);
+  long long units = (long long)m_tiles * (walks ? e.nsplit : n_tiles) * ksplit;
   if (walks && (e.nsplit < 1 || e.nsplit > n_tiles)) return cudaErrorInvalidValue;
-  const int grid = (int)(units < groups ? units : groups) * CTAS_DEFAULT;      // stream-K: units >= groups
+  const int grid = (int)(units < groups ? units : groups) * CTAS_DEFAULT;
   switch (e.kind) {
     case EPI_STORE_F32: return launch<EPI_STORE_F32>(tmA, tmB, tmC, a, grid, stream);
     case EPI_LSE_PARTIAL: return launch<EPI_LSE_PARTIAL>(tmA, tmB, tmC, a, grid, stream);

@@ -641,3 +641,19 @@ def test_more_utterances_than_one_length_slice(lib, path):
     fl = greedy["frame_labels"].cpu().numpy()
     for n in (0, 1023, 1024, 2047, 2048, 2099):
         assert np.all(fl[n, : batch.input_lengths[n]] >= 0) and np.all(fl[n, batch.input_lengths[n]:] == -1)
+
+
+@pytest.mark.parametrize("V,chunk", [(2 * 3072 + 520, 3072), (3 * 2560, 2560)])
+def test_wide_head_many_output_tiles_of_dx(lib, V, chunk):
+    """A head wide enough that dX += dZ_c W_c has more output tiles (11 x 13 of 256 x 256) than the GPU has CTA
+    pairs, with a ragged last chunk shorter than the others in the first case.  Three calls must agree bit
+    for bit."""
+    cfg = wl.Config("widehead", N=6, T_lo=400, T_hi=480, D=3328, V=V, dtype="bf16", U_lo=20, U_hi=60, zipf_s=1.1,
+                    rms_norm=True, seed=808)
+    batch = wl.make_batch(cfg, permute_ids=True, poison_padding=True)
+    runs = [H.run_gpu(lib, batch, chunk=chunk) for _ in range(3)]
+    ref = H.run_oracle(batch)
+    H.assert_parity(runs[0], ref, batch)
+    for other in runs[1:]:
+        for k in ("loss", "dH", "dW"):
+            np.testing.assert_array_equal(runs[0][k], other[k])

@@ -63,6 +63,10 @@ VARIANTS = {
     "probe_noepilogue": ("-DPCTC_PROBE=7",),      # no tensor-memory loads, no epilogue arithmetic, no chunk store
     "probe_nostore": ("-DPCTC_PROBE=4",),         # the dlogits chunk is computed but not written
     "probe_skipa": ("-DPCTC_PROBE=8",),           # the normaliser kernel reloads only its B operand per tile
+    "tune_walk_a": ("-DPCTC_TUNE_WALK_HINT=1",),  # L2 evict-last on the A rows of the column-walking kernels
+    "tune_walk_mb8": ("-DPCTC_TUNE_WALK_MB=8",),  # bands of the column-walking kernels whose A rows fill 8 / 16 / 66 MB
+    "tune_walk_mb16": ("-DPCTC_TUNE_WALK_MB=16",),
+    "tune_walk_mb66": ("-DPCTC_TUNE_WALK_MB=66",),
 }
 TEST_VARIANTS = ("shortwait", "bounds")           # the ones the test-suite loads
 

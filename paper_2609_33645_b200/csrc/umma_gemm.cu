@@ -80,6 +80,10 @@ constexpr bool PROBE_SKIP_A = (PCTC_PROBE & 8) != 0;
 #define PCTC_TUNE_CHUNK_HINT 0    // L2 eviction priority for the bf16 dlogits chunk: bit 0 evict-first on its stores
 #endif                            // (dlogits), bit 1 evict-first on its loads (A operand of the dX and dW kernels)
 
+#ifndef PCTC_TUNE_WALK_HINT
+#define PCTC_TUNE_WALK_HINT 0     // column-walking kernels (LSE, arg-max): bit 0 evict-last on the A rows (re-read for
+#endif                            // every column tile), bit 1 evict-first on the B panels (each used once per band)
+
 #ifndef PCTC_TUNE_PDL
 #define PCTC_TUNE_PDL 0           // 1: programmatic dependent launch: a contraction kernel's CTAs may start and set up
 #endif                            // (barriers, tensor memory) while the kernel before it in the stream drains
@@ -244,6 +248,11 @@ __device__ __forceinline__ void tma_store_2d(const CUtensorMap* map, const void*
 __device__ __forceinline__ unsigned long long make_evict_first_policy() {
   unsigned long long p;
   asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(p));
+  return p;
+}
+__device__ __forceinline__ unsigned long long make_evict_last_policy() {
+  unsigned long long p;
+  asm volatile("createpolicy.fractional.L2::evict_last.b64 %0, 1.0;" : "=l"(p));
   return p;
 }
 __device__ __forceinline__ void tma_store_2d_hint(const CUtensorMap* map, const void* smem_src, int c0, int c1,
@@ -531,10 +540,17 @@ k_umma_gemm(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
         else tma_load_2d(dst, map, c0, c1, bar);
       };
       // the A operand of the dX and dW contractions is the dlogits chunk
-      constexpr bool HINT_A = (PCTC_TUNE_CHUNK_HINT & 2) && CTAS == 2 && (EPI == EPI_ACCUM_F32 || EPI == EPI_STORE_OUT);
-      const unsigned long long a_policy = HINT_A ? make_evict_first_policy() : 0ull;
+      constexpr bool WALK_A = (PCTC_TUNE_WALK_HINT & 1) && CTAS == 2 && epi_walks_splits(EPI);
+      constexpr bool WALK_B = (PCTC_TUNE_WALK_HINT & 2) && CTAS == 2 && epi_walks_splits(EPI);
+      constexpr bool HINT_A = ((PCTC_TUNE_CHUNK_HINT & 2) && CTAS == 2 && (EPI == EPI_ACCUM_F32 || EPI == EPI_STORE_OUT)) || WALK_A;
+      const unsigned long long a_policy = WALK_A ? make_evict_last_policy() : (HINT_A ? make_evict_first_policy() : 0ull);
+      const unsigned long long b_policy = WALK_B ? make_evict_first_policy() : 0ull;
       auto load_a = [&](void* dst, const CUtensorMap* map, int c0, int c1, unsigned long long* bar) {
         if (HINT_A) tma_load_2d_pair_hint(dst, map, c0, c1, bar, a_policy);
+        else load(dst, map, c0, c1, bar);
+      };
+      auto load_b = [&](void* dst, const CUtensorMap* map, int c0, int c1, unsigned long long* bar) {
+        if (WALK_B) tma_load_2d_pair_hint(dst, map, c0, c1, bar, b_policy);
         else load(dst, map, c0, c1, bar);
       };
       for (int u = group; u < units && ok; u += ngroups) {
@@ -567,11 +583,11 @@ k_umma_gemm(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
               }
             }
             if (!a.b_mn) {
-              load(dB, &tmB, kb * BK, row_b, &st->full[s]);
+              load_b(dB, &tmB, kb * BK, row_b, &st->full[s]);
             } else {
 #pragma unroll
               for (int q = 0; q < BN / CTAS / 64; ++q)
-                load(dB + q * MN_GROUP_BYTES, &tmB, row_b + q * 64, kb * BK, &st->full[s]);
+                load_b(dB + q * MN_GROUP_BYTES, &tmB, row_b + q * 64, kb * BK, &st->full[s]);
             }
           }
         }

@@ -137,9 +137,11 @@ def _traced_call(binding, hidden, W, bias_dev, targets, il, tl, batch, res, trac
     return trace
 
 
-def time_config(binding, torch, dev, cfg, beam, steps, warmup, peaks):
+def time_config(binding, torch, dev, cfg, beam, steps, warmup, peaks, frozen_head=False, promise_k=False):
     """Device-resident timing of one configuration with the protocol of the headline run: inputs in HBM,
-    `warmup` untimed calls, `steps` timed calls between two CUDA events on the launching stream."""
+    `warmup` untimed calls, `steps` timed calls between two CUDA events on the launching stream.
+    frozen_head: dW is skipped (6 M D V FLOPs).  promise_k: max_K = the number of selected classes, counted on
+    the host as a data loader would."""
     batch = wl.make_batch(cfg)
     tdt = torch.bfloat16 if cfg.dtype == "bf16" else torch.float32
     hidden = torch.from_numpy(batch.hidden).to(tdt).to(dev)
@@ -148,32 +150,36 @@ def time_config(binding, torch, dev, cfg, beam, steps, warmup, peaks):
     il, tl = batch.input_lengths, batch.target_lengths
     M, D, V, N = batch.M, cfg.D, cfg.V, cfg.N
     dt = binding.PCTC_BF16 if cfg.dtype == "bf16" else binding.PCTC_FP32
-    prob = binding.make_problem(N, batch.T, D, V, dt, batch.blank, beam, 0, batch.targets.shape[1])
+    max_K = 0
+    if promise_k:
+        max_K = 1 + int(np.unique(np.concatenate([batch.targets[n, : tl[n]] for n in range(N)])).size)
+    prob = binding.make_problem(N, batch.T, D, V, dt, batch.blank, beam, 0, batch.targets.shape[1], max_K=max_K)
     ws_bytes = binding.workspace_bytes(prob, il, tl)
     chunk, nchunks = binding.chunk_width(prob, il, tl)
     half = binding.make_problem(N, batch.T, D, max(8, V // 2 // 8 * 8), dt, batch.blank, beam, chunk,
-                                batch.targets.shape[1])
+                                batch.targets.shape[1], max_K=max_K)
     ws_half = binding.workspace_bytes(half, il, tl)
-    res = binding.pruned_ctc_fwd_bwd(hidden, W, None, targets, il, tl, batch.blank, beam=beam, check_status=True)
+    kw = dict(beam=beam, skip_dW=frozen_head, max_K=max_K)
+    res = binding.pruned_ctc_fwd_bwd(hidden, W, None, targets, il, tl, batch.blank, check_status=True, **kw)
     for _ in range(max(0, warmup - 1)):
-        binding.pruned_ctc_fwd_bwd(hidden, W, None, targets, il, tl, batch.blank, beam=beam,
-                                   workspace=res["workspace"], out=res)
+        binding.pruned_ctc_fwd_bwd(hidden, W, None, targets, il, tl, batch.blank, workspace=res["workspace"], out=res,
+                                   **kw)
     trace = binding.Trace(binding.Trace.capacity_for(V, chunk))
     ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     torch.cuda.synchronize()
     ev0.record()
     for s in range(steps):
-        binding.pruned_ctc_fwd_bwd(hidden, W, None, targets, il, tl, batch.blank, beam=beam,
-                                   workspace=res["workspace"], out=res, trace=trace if s == steps - 1 else None)
+        binding.pruned_ctc_fwd_bwd(hidden, W, None, targets, il, tl, batch.blank, workspace=res["workspace"], out=res,
+                                   trace=trace if s == steps - 1 else None, **kw)
     ev1.record()
     torch.cuda.synchronize()
     if binding.workspace_status(res["workspace"]) != 0:
         raise SystemExit("device status word set while timing " + cfg.name)
     ms = ev0.elapsed_time(ev1) / steps
     dp_ms = sum(t for kind, t in trace.spans() if kind >= 0 and binding.PHASES[kind] == "dp")
-    flops = 8.0 * M * D * V
+    flops = (6.0 if frozen_head else 8.0) * M * D * V
     tfl = flops / (ms * 1e-3) / 1e12
-    out = dict(workload=cfg.name, dtype=cfg.dtype, beam=beam, M_frames=M, K_selected=int(res["K"].item()), D=D, V=V,
+    out = dict(workload=cfg.name, dtype=cfg.dtype, beam=beam, frozen_head=frozen_head, flops_per_step=flops, M_frames=M, K_selected=int(res["K"].item()), D=D, V=V,
                chunk=chunk, steps=steps, warmup=warmup, ms_per_step=round(ms, 4), frames_per_s=round(M / (ms * 1e-3), 1),
                tflops=round(tfl, 2),
                frac_of_bf16_peak=(dict(burst=round(tfl / peaks["bf16_tflops"], 4),
@@ -198,11 +204,12 @@ def print_table(path: str) -> int:
     if line is None:
         print("no bench line with an all_configs block in", path)
         return 1
-    print("| config | M | K | chunk | ms/step | frames/s | TFLOP/s (8MDV) | of measured burst / sustained bf16 peak "
+    print("| config | M | K | chunk | ms/step | frames/s | TFLOP/s | of measured burst / sustained bf16 peak "
           "| DP ms | workspace (at V/2; one fp32 M x V array) |")
     print("|---|---|---|---|---|---|---|---|---|---|")
     for r in line["all_configs"]:
-        name = r["workload"] + (", beam %g" % r["beam"] if r["beam"] else "")
+        name = r["workload"] + (", beam %g" % r["beam"] if r["beam"] else "") + (
+            ", frozen head (6MDV)" if r.get("frozen_head") else "")
         fr = r["frac_of_bf16_peak"]
         frac = "n/a (fp32 FMA path)" if fr is None else "%.1f%% / %.1f%%" % (100 * fr["burst"], 100 * fr["sustained"])
         print("| %s | %d | %d | %d | %.3f | %.0fk | %.1f | %s | %.2f | %.2f GB (%.2f GB; %.2f GB) |" % (
@@ -595,6 +602,10 @@ def main():
         for name, beams in (("c1", (0.0,)), ("c2", (0.0,)), ("c3", (0.0,)), ("c4", (0.0,)), ("c5", (0.0, 16.0, 8.0))):
             for b in beams:
                 all_cfg.append(time_config(binding, torch, dev, wl.CONFIGS[name], b, args.all_steps, 3, peaks))
+        # two more rows beyond the five configurations: the frozen-head setting of the paper's LLM-CTC runs on
+        # the headline shape, and the smallest workload of the paper's own benchmark grid
+        all_cfg.append(time_config(binding, torch, dev, wl.CONFIGS["c4"], 0.0, args.all_steps, 3, peaks, frozen_head=True))
+        all_cfg.append(time_config(binding, torch, dev, wl.CONFIGS["g16k"], 0.0, args.all_steps, 3, peaks, promise_k=True))
 
     line = dict(
         metric=METRIC, value=value, unit=UNIT, n_gpus=world, steps=args.steps, warmup=args.warmup,

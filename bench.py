@@ -208,6 +208,9 @@ def print_table(path: str) -> int:
           "| DP ms | workspace (at V/2; one fp32 M x V array) |")
     print("|---|---|---|---|---|---|---|---|---|---|")
     for r in line["all_configs"]:
+        if "error" in r:
+            print("| %s | failed: %s |" % (r["workload"], r["error"]))
+            continue
         name = r["workload"] + (", beam %g" % r["beam"] if r["beam"] else "") + (
             ", frozen head (6MDV)" if r.get("frozen_head") else "")
         fr = r["frac_of_bf16_peak"]
@@ -599,13 +602,17 @@ def main():
         del res, hidden, W, targets, traces
         torch.cuda.empty_cache()
         all_cfg = []
-        for name, beams in (("c1", (0.0,)), ("c2", (0.0,)), ("c3", (0.0,)), ("c4", (0.0,)), ("c5", (0.0, 16.0, 8.0))):
-            for b in beams:
-                all_cfg.append(time_config(binding, torch, dev, wl.CONFIGS[name], b, args.all_steps, 3, peaks))
-        # two more rows beyond the five configurations: the frozen-head setting of the paper's LLM-CTC runs on
-        # the headline shape, and the smallest workload of the paper's own benchmark grid
-        all_cfg.append(time_config(binding, torch, dev, wl.CONFIGS["c4"], 0.0, args.all_steps, 3, peaks, frozen_head=True))
-        all_cfg.append(time_config(binding, torch, dev, wl.CONFIGS["g16k"], 0.0, args.all_steps, 3, peaks, promise_k=True))
+        # the five configurations (c5 also at beams 16 and 8), then two more rows: the frozen-head setting of the
+        # paper's LLM-CTC runs on the headline shape, and the smallest workload of the paper's own benchmark grid
+        plan = [(n, b, {}) for n, beams in (("c1", (0.0,)), ("c2", (0.0,)), ("c3", (0.0,)), ("c4", (0.0,)),
+                                            ("c5", (0.0, 16.0, 8.0))) for b in beams]
+        plan += [("c4", 0.0, dict(frozen_head=True)), ("g16k", 0.0, dict(promise_k=True))]
+        for name, b, kw in plan:
+            try:
+                all_cfg.append(time_config(binding, torch, dev, wl.CONFIGS[name], b, args.all_steps, 3, peaks, **kw))
+            except Exception as exc:      # the headline line must not be lost to a side measurement
+                all_cfg.append(dict(workload=name, beam=b, error=repr(exc)[:300], **kw))
+                torch.cuda.empty_cache()
 
     line = dict(
         metric=METRIC, value=value, unit=UNIT, n_gpus=world, steps=args.steps, warmup=args.warmup,

@@ -67,6 +67,9 @@ VARIANTS = {
     "tune_walk_mb8": ("-DPCTC_TUNE_WALK_MB=8",),  # bands of the column-walking kernels whose A rows fill 8 / 16 / 66 MB
     "tune_walk_mb16": ("-DPCTC_TUNE_WALK_MB=16",),
     "tune_walk_mb66": ("-DPCTC_TUNE_WALK_MB=66",),
+    "tune_lse_s22": ("-DPCTC_TUNE_LSE_SPLITS=22",),   # forced column splits of the LSE kernel (c4: 594 = 22 x 27 tiles)
+    "tune_lse_s27": ("-DPCTC_TUNE_LSE_SPLITS=27",),
+    "tune_lse_s9": ("-DPCTC_TUNE_LSE_SPLITS=9",),
 }
 TEST_VARIANTS = ("shortwait", "bounds")           # the ones the test-suite loads
 

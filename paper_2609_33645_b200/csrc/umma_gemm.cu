@@ -1117,7 +1117,12 @@ bool umma_available() { return encode_fn() != nullptr; }
 
 int umma_lse_partials_per_split(int k) { return epi_warps_for(k) / 4; }
 
+#ifndef PCTC_TUNE_LSE_SPLITS
+#define PCTC_TUNE_LSE_SPLITS 0    // > 0: force this many column splits in the column-walking kernels (experiments)
+#endif
+
 int umma_lse_splits(int m, int n) {
+  if (PCTC_TUNE_LSE_SPLITS > 0) return PCTC_TUNE_LSE_SPLITS < (n + BN - 1) / BN ? PCTC_TUNE_LSE_SPLITS : (n + BN - 1) / BN;
   // column splits per row tile such that the (row tile, split) units fill whole waves of CTAs
   const int sms = sm_count() / CTAS_DEFAULT;       // CTA groups that run at once
   const int m_tiles = (m + BM * CTAS_DEFAULT - 1) / (BM * CTAS_DEFAULT), n_tiles = (n + BN - 1) / BN;
